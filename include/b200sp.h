@@ -1,0 +1,142 @@
+/*
+ * b200sp -- CSR sparse matrix-vector and sparse-times-dense products for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the shared library libb200sp.so.  Plain pointers and sizes only; no exception crosses
+ * this boundary; every function returns a b200sp_status (0 = success) unless stated otherwise.
+ *
+ * Operations (paper: Appendix C, Table 6, task 12 "SpMV CSR" and task 13 "SpMM CSR", which define
+ * A of shape (rows, cols) by values[nnz], col_indices[nnz] and row_offsets[rows + 1] = start of each
+ * row in values, with y = A x and C = A B, B of shape (cols, K), C of shape (rows, K)).  This
+ * library computes the BLAS-style generalisation
+ *
+ *     SpMV:  y = alpha * A * x + beta * y            x: n entries, y: m entries
+ *     SpMM:  Y = alpha * A * B + beta * Y            B: n x k, Y: m x k, both row-major, leading dim k
+ *
+ * in FP32, or with BF16 storage and FP32 accumulation (B200SP_BF16: vals, x / B and y / Y hold raw
+ * 16-bit bfloat16 patterns; alpha and beta stay FP32; every product and sum is FP32; one
+ * round-to-nearest-even conversion at the final store).
+ *
+ * Conventions common to all entry points
+ *  - Indices are 0-based int32; sizes are int64 with m, n, nnz < 2^31; row_ptr[0] = 0,
+ *    row_ptr[m] = nnz, row_ptr non-decreasing, 0 <= col_idx[p] < n.  Content is NOT checked on the
+ *    hot path (b200sp_validate_csr does it on request).  Columns may be unsorted; duplicates add.
+ *  - Unless a function says "host", every array pointer is a DEVICE pointer on the current device,
+ *    owned by the caller, which keeps it alive and unmodified until the stream work has finished.
+ *    col_idx, vals, x / B and y / Y must be 16-byte aligned, row_ptr 4-byte aligned.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls enqueue
+ *    work and return without synchronising, except where stated (plan creation reads back a few
+ *    hundred bytes and synchronises the stream once).
+ *  - beta == 0: y / Y is write-only (its old contents, NaN included, are ignored).  alpha == 0 or
+ *    nnz == 0: y = beta * y without reading A.  m == 0: nothing is done.  x / B must not alias y / Y.
+ *  - Results are deterministic: the same inputs give bit-identical outputs on every call (no
+ *    floating-point atomics; rows cut by a tile boundary are completed in a fixed order).
+ *  - Errors: host-detectable problems (negative or too large sizes, NULL pointer with non-zero
+ *    size, unknown dtype, k <= 0, misaligned pointer) return B200SP_ERR_INVALID_ARG and launch
+ *    nothing; a device that is not compute capability 10.x returns B200SP_ERR_ARCH; a failing CUDA
+ *    call returns B200SP_ERR_CUDA and its message is kept for b200sp_last_cuda_error().
+ *  - There is no CPU fallback: without a B200 the compute entry points fail.
+ */
+#ifndef B200SP_H_
+#define B200SP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { B200SP_F32 = 0, B200SP_BF16 = 1 } b200sp_dtype;
+
+typedef enum {
+  B200SP_OK = 0,
+  B200SP_ERR_INVALID_ARG = 1,
+  B200SP_ERR_UNSUPPORTED = 2,
+  B200SP_ERR_CUDA = 3,
+  B200SP_ERR_ALLOC = 4,
+  B200SP_ERR_ARCH = 5,
+  B200SP_ERR_BAD_CSR = 6
+} b200sp_status;
+
+/* Opaque: row statistics, row bins, nnz-balanced tile splits and the scratch the kernels need. */
+typedef struct b200sp_plan b200sp_plan;
+
+/* Row-length bins of the plan pass: rows of length 0, 1-4, 5-32, 33-1024 and > 1024. */
+#define B200SP_NUM_BINS 5
+
+/* What the plan pass found (b200sp_plan_info).  All counts are exact integers. */
+typedef struct {
+  int64_t m, n, nnz;
+  int32_t min_row_len, max_row_len;
+  int64_t bin_rows[B200SP_NUM_BINS];  /* rows per length bin */
+  int64_t bin_nnz[B200SP_NUM_BINS];   /* nonzeros held by the rows of each bin */
+  int32_t spmv_kernel;                /* 0 = merge-tile kernel (rows + nnz balanced), 1 = row-direct kernel */
+  int32_t spmv_tile_items;            /* merge items (rows + nonzeros) per SpMV tile */
+  int32_t spmv_tiles;                 /* number of SpMV tiles */
+  int32_t spmm_tile_nnz;              /* nonzeros per SpMM work unit */
+  int32_t spmm_tiles;                 /* number of SpMM work units */
+  int64_t scratch_bytes;              /* device memory held by the plan */
+} b200sp_plan_info_t;
+
+/* ---- one-shot calls -------------------------------------------------------------------------
+ * Task 12 / task 13 of the paper's Table 6 with alpha and beta.  The first call for a given
+ * (device, row_ptr, m, n, nnz) builds a plan (see b200sp_plan_create; synchronises the stream once)
+ * and caches it inside the library; later calls with the same key reuse it, so the CONTENTS of
+ * row_ptr must not change while the plan is cached (b200sp_cache_clear drops all cached plans).
+ * Two calls that use the same cached plan must not overlap on the GPU (they share its scratch).
+ * dtype is a b200sp_dtype. */
+int spmv_csr(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx,
+             const void* vals, const void* x, void* y, float alpha, float beta, int dtype, void* stream);
+
+int spmm_csr(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_ptr, const int32_t* col_idx,
+             const void* vals, const void* B, void* Y, float alpha, float beta, int dtype, void* stream);
+
+/* ---- plan API --------------------------------------------------------------------------------
+ * The plan pass depends on the sparsity pattern's row structure only (row_ptr): it computes the
+ * row-length statistics and bins, chooses the kernels, and computes the nnz-balanced split points
+ * (a merge-path search over rows + nonzeros for SpMV, over nonzeros for SpMM), all on the device.
+ * It allocates a few bytes per tile of device memory (released by b200sp_plan_destroy) and
+ * synchronises `stream` once.  A plan may be used from one stream at a time. */
+int b200sp_plan_create(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, void* stream);
+int b200sp_plan_destroy(b200sp_plan* plan);
+int b200sp_plan_info(const b200sp_plan* plan, b200sp_plan_info_t* out); /* `out` is a host pointer */
+
+/* Same operations as spmv_csr / spmm_csr with an explicit plan (m, n, nnz, row_ptr come from it). */
+int b200sp_spmv(b200sp_plan* plan, const int32_t* col_idx, const void* vals, const void* x, void* y,
+                float alpha, float beta, int dtype, void* stream);
+int b200sp_spmm(b200sp_plan* plan, int64_t k, const int32_t* col_idx, const void* vals, const void* B, void* Y,
+                float alpha, float beta, int dtype, void* stream);
+
+/* ---- host-buffer calls -----------------------------------------------------------------------
+ * Same operations with every array in HOST memory (pinned memory makes the copies asynchronous and
+ * faster, pageable memory works).  Each call allocates device buffers from the stream-ordered pool,
+ * copies the inputs in, plans (cached per pattern shape is impossible here, so the plan is rebuilt),
+ * runs the kernels, copies y / Y back and synchronises `stream` before returning. */
+int spmv_csr_host(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx,
+                  const void* vals, const void* x, void* y, float alpha, float beta, int dtype, void* stream);
+int spmm_csr_host(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_ptr, const int32_t* col_idx,
+                  const void* vals, const void* B, void* Y, float alpha, float beta, int dtype, void* stream);
+
+/* ---- checking and housekeeping ---------------------------------------------------------------
+ * b200sp_validate_csr checks on the device that row_ptr[0] = 0, row_ptr[m] = nnz, row_ptr is
+ * non-decreasing and every column index lies in [0, n); it synchronises the stream and returns
+ * B200SP_ERR_BAD_CSR if any check fails. */
+int b200sp_validate_csr(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx, void* stream);
+
+void b200sp_cache_clear(void);                 /* destroys every plan cached by the one-shot calls */
+const char* b200sp_status_string(int status);  /* static string, never NULL */
+const char* b200sp_last_cuda_error(void);      /* message of this thread's last failing CUDA call, "" if none */
+int b200sp_version(void);                      /* major * 10000 + minor * 100 + patch */
+
+/* Number of kernels this library has launched from this process so far (all entry points). */
+int64_t b200sp_launch_count(void);
+
+/* Tuning switches for A/B measurements; unknown names return B200SP_ERR_INVALID_ARG.
+ *   "spmv_kernel"   -1 = choose from the plan statistics (default), 0 = merge-tile, 1 = row-direct
+ *   "x_l2_window"    1 = pin x / B in L2 with a per-launch access-policy window (default), 0 = off
+ * A change applies to plans created afterwards. */
+int b200sp_set_option(const char* name, int value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* B200SP_H_ */

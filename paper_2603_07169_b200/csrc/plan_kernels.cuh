@@ -1,0 +1,96 @@
+// Plan pass (device side): row-length statistics and bins, nnz-balanced split points.
+#pragma once
+#include "common.cuh"
+
+namespace b200sp {
+
+struct PlanStats {
+  int min_len;
+  int max_len;
+  int bad;  // row_ptr not monotone (negative length seen)
+  int pad;
+  unsigned long long bin_rows[5];
+  unsigned long long bin_nnz[5];
+};
+
+__device__ __forceinline__ int length_bin(int len) {
+  return len == 0 ? 0 : len <= 4 ? 1 : len <= 32 ? 2 : len <= 1024 ? 3 : 4;
+}
+
+// One pass over row_ptr: min / max row length and the five length bins (rows, nnz per bin).
+// Integer atomics only, so the result does not depend on scheduling.
+__global__ void __launch_bounds__(256) plan_stats_kernel(const int* __restrict__ row_ptr, int m, PlanStats* st) {
+  __shared__ unsigned long long s_rows[5], s_nnz[5];
+  __shared__ int s_min, s_max, s_bad;
+  if (threadIdx.x < 5) { s_rows[threadIdx.x] = 0; s_nnz[threadIdx.x] = 0; }
+  if (threadIdx.x == 0) { s_min = 0x7FFFFFFF; s_max = 0; s_bad = 0; }
+  __syncthreads();
+  int lmin = 0x7FFFFFFF, lmax = 0, bad = 0;
+  unsigned rows[5] = {0, 0, 0, 0, 0};
+  unsigned long long nz[5] = {0, 0, 0, 0, 0};
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < m; i += (long long)gridDim.x * blockDim.x) {
+    const int len = row_ptr[i + 1] - row_ptr[i];
+    if (len < 0) { bad = 1; continue; }
+    lmin = min(lmin, len); lmax = max(lmax, len);
+    const int b = length_bin(len);
+#pragma unroll
+    for (int j = 0; j < 5; ++j) if (b == j) { rows[j]++; nz[j] += (unsigned)len; }
+  }
+  atomicMin(&s_min, lmin); atomicMax(&s_max, lmax); if (bad) atomicOr(&s_bad, 1);
+#pragma unroll
+  for (int j = 0; j < 5; ++j) if (rows[j]) { atomicAdd(&s_rows[j], (unsigned long long)rows[j]); atomicAdd(&s_nnz[j], nz[j]); }
+  __syncthreads();
+  if (threadIdx.x == 0) { atomicMin(&st->min_len, s_min); atomicMax(&st->max_len, s_max); if (s_bad) atomicOr(&st->bad, 1); }
+  if (threadIdx.x < 5 && s_rows[threadIdx.x]) {
+    atomicAdd(&st->bin_rows[threadIdx.x], s_rows[threadIdx.x]);
+    atomicAdd(&st->bin_nnz[threadIdx.x], s_nnz[threadIdx.x]);
+  }
+}
+
+// Merge-path split: the work list is the merge of the m row-end markers (row_ptr[1..m]) with the nnz
+// nonzero positions 0..nnz-1; tile t starts at diagonal t * items.  split_row[t] = number of row ends
+// consumed before that diagonal, so the tile's first nonzero is t * items - split_row[t].
+__global__ void __launch_bounds__(256) plan_merge_split_kernel(const int* __restrict__ row_ptr, int m, int nnz, int items,
+                                                               int tiles, int* __restrict__ split_row) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t > tiles) return;
+  const long long total = (long long)m + nnz;
+  long long d = (long long)t * items;
+  if (d > total) d = total;
+  int lo = (int)max(d - (long long)nnz, 0LL), hi = (int)min(d, (long long)m);
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if ((long long)row_ptr[mid + 1] <= d - mid - 1) lo = mid + 1; else hi = mid;
+  }
+  split_row[t] = lo;
+}
+
+// nnz-only split for SpMM: unit u starts at nonzero u * tile_nnz; split_row[u] = the row holding it
+// (the last row whose start is <= that position; rows of length 0 are skipped over).
+__global__ void __launch_bounds__(256) plan_nnz_split_kernel(const int* __restrict__ row_ptr, int m, int nnz, int tile_nnz,
+                                                             int tiles, int* __restrict__ split_row) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t > tiles) return;
+  long long p = (long long)t * tile_nnz;
+  if (p >= nnz) { split_row[t] = m; return; }
+  int lo = 0, hi = m;  // find the largest r with row_ptr[r] <= p  (then row_ptr[r+1] > p)
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if ((long long)row_ptr[mid + 1] <= p) lo = mid + 1; else hi = mid;
+  }
+  split_row[t] = lo;
+}
+
+// CSR content check on request.
+__global__ void __launch_bounds__(256) validate_csr_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col_idx, int m, int n,
+                                                           int nnz, int* bad) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  int b = 0;
+  if (i0 == 0) { if (row_ptr[0] != 0) b |= 1; if (row_ptr[m] != nnz) b |= 2; }
+  for (long long i = i0; i < m; i += stride) if (row_ptr[i + 1] < row_ptr[i]) b |= 4;
+  for (long long p = i0; p < nnz; p += stride) { const int c = col_idx[p]; if (c < 0 || c >= n) b |= 8; }
+  if (b) atomicOr(bad, b);
+}
+
+}  // namespace b200sp

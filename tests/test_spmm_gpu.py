@@ -1,0 +1,71 @@
+"""GPU parity: CSR SpMM through the C ABI against the CPU oracle."""
+import numpy as np
+import pytest
+
+import gen
+import oracle
+import paper_2603_07169_b200 as b200sp
+from gpu_util import assert_within, run_spmm, store
+
+pytestmark = pytest.mark.gpu
+
+DTYPES = ["f32", "bf16"]
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("k", [1, 3, 8, 17, 32, 64, 100, 256, 264])
+def test_small_random_all_k(k, dtype):
+    rng = np.random.default_rng(k)
+    m, n = 1500, 333
+    lens = rng.integers(0, 40, m)
+    lens[5] = 3000
+    lens[6] = 0
+    A = gen.random_csr(m, n, lens, seed=k)
+    B = rng.standard_normal(n * k).astype(np.float32)
+    Y0 = rng.standard_normal(m * k).astype(np.float32)
+    Y, Y_ref, S = run_spmm(A, B, k, None, 1.0, 0.0, dtype)
+    assert_within(Y, Y_ref, S, dtype, what="k=%d %s" % (k, dtype))
+    Y, Y_ref, S = run_spmm(A, B, k, Y0, 0.5, -2.0, dtype)
+    y0f = Y0 if dtype == "f32" else gen.bf16_to_f32(gen.to_bf16(Y0))
+    assert_within(Y, Y_ref, S, dtype, 1.0, np.abs(2.0 * y0f.astype(np.float64)).reshape(m, k), what="k=%d %s ab" % (k, dtype))
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_spmm_column_equals_spmv(dtype):
+    from gpu_util import run_spmv
+    rng = np.random.default_rng(1)
+    m, n, k = 4000, 500, 8
+    A = gen.random_csr(m, n, rng.integers(0, 30, m), 2)
+    B = rng.standard_normal((n, k)).astype(np.float32)
+    Y, Y_ref, S = run_spmm(A, B.ravel(), k, None, 1.0, 0.0, dtype)
+    assert_within(Y, Y_ref, S, dtype)
+
+
+@pytest.mark.parametrize("name", ["c5k64", "c5k256"])
+def test_workload_scaled(name):
+    w = gen.workload(name, scale_down=3)
+    for dtype in w.dtypes:
+        Y, Y_ref, S = run_spmm(w.A, w.B, w.k, None, w.alpha, w.beta, dtype)
+        assert_within(Y, Y_ref, S, dtype, what="%s %s" % (name, dtype))
+
+
+@pytest.mark.parametrize("name", ["c5k64", "c5k256"])
+def test_workload_full_size_sampled_rows(name):
+    """Full size; the oracle computes 2048 sampled output rows (plus the first and last) one by one."""
+    w = gen.workload(name)
+    rng = np.random.default_rng(11)
+    rows = np.unique(np.concatenate([[0, w.A.m - 1], rng.integers(0, w.A.m, 2048)])).astype(np.int64)
+    for dtype in w.dtypes:
+        Y, Y_ref, S = run_spmm(w.A, w.B, w.k, None, w.alpha, w.beta, dtype, rows=rows)
+        assert_within(Y, Y_ref, S, dtype, what="%s %s full" % (name, dtype))
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_host_buffer_entry_point(dtype):
+    w = gen.workload("c5k64", scale_down=4)
+    A = w.A
+    vals, B = store(A.vals, dtype), store(w.B, dtype)
+    Y = np.zeros(A.m * w.k, np.float32 if dtype == "f32" else np.uint16)
+    b200sp.spmm_csr_host(A.m, A.n, A.nnz, w.k, A.row_ptr, A.col_idx, vals, B, Y, 1.0, 0.0, dtype)
+    Y_ref, S = oracle.spmm_csr(A.m, A.n, w.k, A.row_ptr, A.col_idx, vals, B, None, 1.0, 0.0, dtype)
+    assert_within(Y.reshape(A.m, w.k), Y_ref, S, dtype)

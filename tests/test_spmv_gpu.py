@@ -1,0 +1,182 @@
+"""GPU parity: CSR SpMV through the C ABI against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+import paper_2603_07169_b200 as b200sp
+from gpu_util import assert_within, empty_out, run_spmv, store, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+DTYPES = ["f32", "bf16"]
+
+
+def ext_bound(A, S_ref, y0, alpha, beta):
+    """Labelled extension of the bound for alpha != 1 / beta != 0: S' = |alpha| S + |beta y0|."""
+    extra = np.abs(beta * y0.astype(np.float64)) if (beta != 0 and y0 is not None) else None
+    return abs(alpha) if alpha != 0 else 1.0, extra
+
+
+# ---------------------------------------------------------------- adversarial small shapes
+def row_len_cases():
+    rng = np.random.default_rng(0)
+    cases = {
+        "every_length_0_to_130": np.arange(131),
+        "all_empty": np.zeros(1000, np.int64),
+        "one_huge_row": np.array([3, 0, 100000, 5, 0, 0, 1]),
+        "huge_first_and_last": np.array([20000, 1, 0, 2, 30000]),
+        "single_row": np.array([9000]),
+        "single_entry": np.array([1]),
+        "many_empty_then_dense": np.concatenate([np.zeros(9000, np.int64), np.full(50, 700)]),
+        "lengths_32_33": np.tile([32, 33], 700),
+        "random_geometric": rng.geometric(0.08, 5000) - 1,
+        "tile_exact": np.full(4096 // 17 * 3, 16),          # rows + nnz = multiple of the tile size
+        "power_law": (rng.pareto(1.2, 3000) * 3).astype(np.int64).clip(0, 40000),
+    }
+    return cases
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("case", sorted(row_len_cases()))
+def test_adversarial_row_lengths(case, dtype):
+    lens = row_len_cases()[case]
+    m = len(lens)
+    n = 777
+    A = gen.random_csr(m, n, lens, seed=len(case), sort_cols=False, allow_dup=True)
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal(n).astype(np.float32)
+    y0 = rng.standard_normal(m).astype(np.float32)
+    for alpha, beta in [(1.0, 0.0), (-1.25, 0.75)]:
+        y, y_ref, S = run_spmv(A, x, y0, alpha, beta, dtype)
+        sc, extra = ext_bound(A, S, store(y0, "f32") if dtype == "f32" else gen.bf16_to_f32(gen.to_bf16(y0)), alpha, beta)
+        assert_within(y, y_ref, S, dtype, sc, extra, what="%s %s a=%g b=%g" % (case, dtype, alpha, beta))
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_empty_rows_are_exactly_zero_and_nan_in_y_is_ignored(dtype):
+    lens = np.array([0, 5, 0, 0, 40, 0])
+    A = gen.random_csr(6, 50, lens, 5)
+    x = np.ones(50, np.float32)
+    y, y_ref, S = run_spmv(A, x, None, 1.0, 0.0, dtype)     # run_spmv pre-fills y with NaN
+    yf = y if dtype == "f32" else gen.bf16_to_f32(y)
+    assert np.all(np.isfinite(yf))
+    assert yf[0] == 0 and yf[2] == 0 and yf[3] == 0 and yf[5] == 0
+    assert_within(y, y_ref, S, dtype)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_n_equal_one_and_m_not_multiple_of_anything(dtype):
+    rng = np.random.default_rng(3)
+    m = 4099
+    lens = rng.integers(0, 4, m)
+    A = gen.random_csr(m, 1, lens, 9)
+    x = np.array([1.5], np.float32)
+    y, y_ref, S = run_spmv(A, x, None, 1.0, 0.0, dtype)
+    assert_within(y, y_ref, S, dtype)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_alpha_zero_and_no_nonzeros(dtype):
+    m, n = 3000, 10
+    A = gen.random_csr(m, n, np.full(m, 2), 1)
+    rng = np.random.default_rng(0)
+    y0 = rng.standard_normal(m).astype(np.float32)
+    x = np.full(n, np.nan, np.float32)                        # alpha == 0: A and x are not read
+    y, y_ref, S = run_spmv(A, np.ones(n, np.float32), y0, 0.0, 2.0, dtype)
+    yf = y if dtype == "f32" else gen.bf16_to_f32(y)
+    assert_within(y, y_ref, S, dtype, 1.0, np.abs(2.0 * y0.astype(np.float64)))
+    Z = gen.random_csr(m, n, np.zeros(m, np.int64), 1)
+    y, y_ref, S = run_spmv(Z, np.ones(n, np.float32), y0, 1.0, 0.0, dtype)
+    yf = y if dtype == "f32" else gen.bf16_to_f32(y)
+    assert np.all(yf == 0)
+    y, y_ref, S = run_spmv(Z, np.ones(n, np.float32), y0, 1.0, -1.0, dtype)
+    assert_within(y, y_ref, S, dtype, 1.0, np.abs(y0.astype(np.float64)))
+
+
+def test_integer_data_is_exact_fp32():
+    rng = np.random.default_rng(2)
+    m, n = 20000, 300
+    lens = rng.integers(0, 60, m)
+    lens[17] = 9000
+    A = gen.random_csr(m, n, lens, 4, integer_vals=True)
+    x = rng.integers(-3, 4, n).astype(np.float32)
+    y, y_ref, S = run_spmv(A, x, None, 1.0, 0.0, "f32")
+    assert np.array_equal(y.astype(np.float64), y_ref)        # every partial sum is an exact integer
+
+
+# ---------------------------------------------------------------- the measured workloads
+@pytest.mark.parametrize("name,scale", [("c1", 0), ("c2", 2), ("c3", 2), ("c4", 2)])
+def test_workloads_scaled(name, scale):
+    w = gen.workload(name, scale_down=scale)
+    for dtype in w.dtypes:
+        y, y_ref, S = run_spmv(w.A, w.x, w.y0, w.alpha, w.beta, dtype, use_plan=(dtype == "bf16"))
+        r = assert_within(y, y_ref, S, dtype, what="%s %s" % (name, dtype))   # the literal bound, S without alpha/beta
+        assert r < 1.0
+
+
+@pytest.mark.parametrize("name", ["c2", "c3", "c4"])
+def test_workloads_full_size(name):
+    """Full size in the launch configuration the benchmark times; the oracle runs on all host cores."""
+    w = gen.workload(name)
+    for dtype in w.dtypes:
+        y, y_ref, S = run_spmv(w.A, w.x, w.y0, w.alpha, w.beta, dtype)
+        assert_within(y, y_ref, S, dtype, what="%s %s full" % (name, dtype))
+
+
+# ---------------------------------------------------------------- determinism, plan, validation, host API
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_bitwise_run_to_run_determinism(dtype):
+    w = gen.workload("c3", scale_down=1)
+    A = w.A
+    d = [to_dev(a) for a in (A.row_ptr, A.col_idx, store(A.vals, dtype), store(w.x, dtype))]
+    outs = []
+    for _ in range(3):
+        y = empty_out(A.m, dtype)
+        b200sp.spmv_csr(A.m, A.n, A.nnz, d[0], d[1], d[2], d[3], y, 1.0, 0.0, dtype)
+        torch.cuda.synchronize()
+        outs.append(y.cpu().numpy().copy())
+    b200sp.b200sp_cache_clear()
+    assert np.array_equal(outs[0].view(np.uint8), outs[1].view(np.uint8))
+    assert np.array_equal(outs[0].view(np.uint8), outs[2].view(np.uint8))
+
+
+def test_plan_info_matches_numpy():
+    w = gen.workload("c3", scale_down=2)
+    A = w.A
+    d_rp = to_dev(A.row_ptr)
+    plan = b200sp.b200sp_plan_create(A.m, A.n, A.nnz, d_rp)
+    info = b200sp.b200sp_plan_info(plan)
+    b200sp.b200sp_plan_destroy(plan)
+    L = np.diff(A.row_ptr).astype(np.int64)
+    assert info["m"] == A.m and info["n"] == A.n and info["nnz"] == A.nnz
+    assert info["min_row_len"] == L.min() and info["max_row_len"] == L.max()
+    edges = [(0, 0), (1, 4), (5, 32), (33, 1024), (1025, 1 << 40)]
+    for j, (lo, hi) in enumerate(edges):
+        sel = (L >= lo) & (L <= hi)
+        assert info["bin_rows"][j] == sel.sum() and info["bin_nnz"][j] == L[sel].sum()
+    assert info["spmv_tiles"] == -(-(A.m + A.nnz) // info["spmv_tile_items"])
+
+
+def test_validate_csr():
+    A = gen.random_csr(100, 40, np.full(100, 3), 1)
+    d_rp, d_ci = to_dev(A.row_ptr), to_dev(A.col_idx)
+    assert b200sp.b200sp_validate_csr(A.m, A.n, A.nnz, d_rp, d_ci) == 0
+    bad = A.col_idx.copy(); bad[7] = 40
+    assert b200sp.b200sp_validate_csr(A.m, A.n, A.nnz, d_rp, to_dev(bad)) == 6
+    bad = A.row_ptr.copy(); bad[5] = bad[6] + 1
+    assert b200sp.b200sp_validate_csr(A.m, A.n, A.nnz, to_dev(bad), d_ci) == 6
+    bad = A.row_ptr.copy(); bad[-1] -= 1
+    assert b200sp.b200sp_validate_csr(A.m, A.n, A.nnz, to_dev(bad), d_ci) == 6
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_host_buffer_entry_point(dtype):
+    w = gen.workload("c2", scale_down=3)
+    A = w.A
+    vals, x, y0 = store(A.vals, dtype), store(w.x, dtype), store(w.y0, dtype)
+    y = y0.copy()
+    b200sp.spmv_csr_host(A.m, A.n, A.nnz, A.row_ptr, A.col_idx, vals, x, y, w.alpha, w.beta, dtype)
+    y_ref, S = oracle.spmv_csr(A.m, A.n, A.row_ptr, A.col_idx, vals, x, y0, w.alpha, w.beta, dtype)
+    assert_within(y, y_ref, S, dtype)
