@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the CSR SpMV / SpMM hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extras]
+
+Headline (one JSON line on stdout): effective HBM GB/s of CSR SpMV on the uniform 16-nonzeros-per-row
+workload (m = n = 2^20, FP32, alpha 1.5, beta 0.5), i.e. algorithmic bytes per call divided by the
+device time per call, through the C ABI (spmv_csr) with a cached plan.  One "step" is one spmv_csr
+call (merge-tile kernel + carry fix-up kernel).  Inputs are resident in HBM; to keep every call
+cold, the steps rotate over R independent device copies of all operands whose total size is several
+times the L2 capacity, so no flush sits inside the timed region.  The same line carries the
+roofline fraction against the measured copy bandwidth, an end-to-end figure through spmv_csr_host
+(host buffers, copies inside the timed region), the CPU oracle timed on the host cores, the other
+workloads (BF16, R-MAT, 27-point stencil, SpMM) as extras, and the SM clocks sampled while running.
+
+With --gpus N > 1 (launched by torch.distributed.run) every rank runs an independent replica on its
+own GPU: the path is single-GPU by design, there is no data-path collective.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "SpMV/SpMM effective HBM GB/s (fraction of B200 peak); GFLOP/s at 2*nnz*k"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes (read + write) per launch of the dominant kernel from an ncu capture, keyed by
+# (workload, dtype); None where no capture has been made.  Sources: the summaries under profiles/.
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) from a background thread."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples = []
+        self.period = period_s
+        self._stop = threading.Event()
+        self._thread = None
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_sm = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as e:  # pragma: no cover
+            self.err = repr(e)
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                clk = int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                self.samples.append((time.perf_counter(), clk, reasons))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.ok:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread:
+            self._stop.set()
+            self._thread.join()
+
+    def summary(self, t0: float, t1: float):
+        if not self.ok:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml unavailable"]}
+        sel = [s for s in self.samples if t0 <= s[0] <= t1] or self.samples
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+                 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+        seen = 0
+        for s in sel:
+            seen |= s[2]
+        reasons = [n for bit, n in names.items() if seen & bit]
+        clk = sorted(s[1] for s in sel)
+        return {"sm_mhz": clk[len(clk) // 2] if clk else None, "sm_max_mhz": self.max_sm, "reasons": reasons,
+                "samples": len(sel)}
+
+
+# ------------------------------------------------------------------------------------------ helpers
+def stored(a, dtype):
+    import gen
+    if a is None:
+        return None
+    return gen.to_bf16(a) if dtype == "bf16" else np.ascontiguousarray(a, np.float32)
+
+
+def up(a, dev):
+    import torch
+    return torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).to(dev)
+
+
+class DeviceSet:
+    """One device copy of all operands of a workload."""
+
+    def __init__(self, w, dtype, dev):
+        import torch
+        A = w.A
+        self.rp, self.ci = up(A.row_ptr, dev), up(A.col_idx, dev)
+        self.va = up(stored(A.vals, dtype), dev)
+        dense = w.B if w.k else w.x
+        self.inp = up(stored(dense, dtype), dev)
+        kk = max(w.k, 1)
+        if w.beta != 0 and w.y0 is not None:
+            self.out = up(stored(w.y0, dtype), dev)
+        else:
+            self.out = torch.zeros(A.m * kk, dtype=torch.float32 if dtype == "f32" else torch.int16, device=dev)
+
+
+def measure(w, dtype, steps, warmup, dev, l2_bytes, barrier=None, min_copies=2, max_bytes=8 << 30):
+    """Times `steps` calls back to back with one CUDA-event pair on the launching stream; the calls rotate
+    over R device copies of all operands (R * bytes >= 4 * L2).  Returns a dict of figures."""
+    import torch
+    import gen
+    import paper_2603_07169_b200 as b200sp
+    A = w.A
+    e = 4 if dtype == "f32" else 2
+    abytes = gen.algorithmic_bytes(A.m, A.n, A.nnz, e, w.beta, w.k)
+    R = max(min_copies, -(-4 * l2_bytes // abytes))
+    R = max(1, min(R, max_bytes // max(abytes, 1), 256))
+    sets = [DeviceSet(w, dtype, dev) for _ in range(R)]
+    stream = torch.cuda.current_stream()
+
+    def call(s):
+        if w.k:
+            b200sp.spmm_csr(A.m, A.n, A.nnz, w.k, s.rp, s.ci, s.va, s.inp, s.out, w.alpha, w.beta, dtype, stream)
+        else:
+            b200sp.spmv_csr(A.m, A.n, A.nnz, s.rp, s.ci, s.va, s.inp, s.out, w.alpha, w.beta, dtype, stream)
+
+    t_plan0 = time.perf_counter()
+    call(sets[0])                       # first call builds and caches the plan for this row_ptr
+    torch.cuda.synchronize()
+    plan_ms = (time.perf_counter() - t_plan0) * 1e3
+    for s in sets[1:]:
+        call(s)
+    for i in range(max(warmup, 3)):
+        call(sets[i % R])
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    l0 = b200sp.b200sp_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    ev0.record(stream)
+    for i in range(steps):
+        call(sets[i % R])
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    t1 = time.perf_counter()
+    if barrier:
+        barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = b200sp.b200sp_launch_count() - l0
+    # isolated single calls (event pair around each, cold L2 by rotation): median
+    iso = []
+    for i in range(min(steps, 50)):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        call(sets[i % R])
+        b.record(stream)
+        b.synchronize()
+        iso.append(a.elapsed_time(b))
+    iso.sort()
+    ms_step = ms / steps
+    flops = 2.0 * A.nnz * max(w.k, 1)
+    res = {"ms_total": ms, "ms_per_step": ms_step, "ms_per_step_isolated_median": iso[len(iso) // 2], "gbs": abytes / ms_step * 1e-6,
+           "gflops": flops / ms_step * 1e-6, "algorithmic_bytes": abytes, "copies": R, "launches": launches,
+           "plan_ms_first_call": plan_ms, "t0": t0, "t1": t1, "nnz": A.nnz, "m": A.m}
+    res["_sets"] = sets
+    res["_call"] = call
+    return res
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores, on the headline workload (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import gen
+    import oracle
+    w = gen.workload("c2")
+    A = w.A
+    abytes = gen.algorithmic_bytes(A.m, A.n, A.nnz, 4, w.beta)
+    nt = oracle.max_threads()
+    run = lambda: oracle.spmv_csr(A.m, A.n, A.row_ptr, A.col_idx, A.vals, w.x, w.y0, w.alpha, w.beta, "f32", nthreads=nt)
+    t = time.perf_counter(); run(); first = time.perf_counter() - t
+    steps, warmup = args.steps, args.warmup
+    budget = 150.0
+    if first * (steps + warmup) > budget:      # keep the whole run within a few minutes
+        steps = max(1, int(budget / first) - warmup)
+    for _ in range(warmup):
+        run()
+    t = time.perf_counter()
+    for _ in range(steps):
+        run()
+    dt = (time.perf_counter() - t) / steps
+    val = abytes / dt * 1e-9
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus, "steps": steps,
+            "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "c2: CSR SpMV m=n=2^20, 16 nnz/row uniform, FP32 storage, alpha=1.5 beta=0.5",
+                       "gflops": 2.0 * A.nnz / dt * 1e-9},
+            "cpu_baseline": {"value": val, "unit": "GB/s", "cores": nt, "kind": "oracle",
+                             "sample": "whole workload per step (16.8 M nonzeros), OpenMP over rows"},
+            "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="only the headline workload")
+    ap.add_argument("--workload", default="c2", help="headline workload (default c2)")
+    ap.add_argument("--dtype", default="f32")
+    ap.add_argument("--profile", action="store_true",
+                    help="short run for a profiler: the timed loop of one workload only (no clock loop, e2e, extras, CPU baseline)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import gen
+    import paper_2603_07169_b200 as b200sp
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = "cuda:%d" % local
+    barrier = None
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+        barrier = lambda: (dist.barrier(), torch.cuda.synchronize())
+    peak, peak_kind = measured_peaks()
+    l2 = torch.cuda.get_device_properties(local).L2_cache_size
+    steps, warmup = max(args.steps, 1), max(args.warmup, 3)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    w = gen.workload(args.workload)
+    dtype = args.dtype
+    head = measure(w, dtype, steps, warmup, dev, l2, barrier)
+    if args.profile:
+        sampler.stop()
+        print(json.dumps({"profile_run": args.workload, "dtype": dtype, "ms_per_step": head["ms_per_step"], "gbs": head["gbs"],
+                          "frac": head["gbs"] / peak, "launches": head["launches"]}))
+        return
+    # keep the same loop running for about a second so that the clock sampler sees it under load
+    t_end = time.perf_counter() + 1.0
+    i = 0
+    while time.perf_counter() < t_end:
+        for _ in range(50):
+            head["_call"](head["_sets"][i % head["copies"]]); i += 1
+        torch.cuda.synchronize()
+    t_load_end = time.perf_counter()
+    clocks = sampler.summary(head["t0"], t_load_end)
+
+    # max over ranks of the timed region
+    ms_total = head["ms_total"]
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / steps
+    value = world * head["algorithmic_bytes"] / ms_step * 1e-6
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
+    A = w.A
+    hs = [torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+          for a in (A.row_ptr, A.col_idx, stored(A.vals, dtype), stored(w.B if w.k else w.x, dtype))]
+    kk = max(w.k, 1)
+    hy = (torch.from_numpy(stored(w.y0, dtype).view(np.int16) if dtype == "bf16" else stored(w.y0, dtype)).pin_memory()
+          if (w.beta != 0 and w.y0 is not None) else torch.zeros(A.m * kk, dtype=torch.float32 if dtype == "f32" else torch.int16).pin_memory())
+    stream = torch.cuda.current_stream()
+
+    def host_call():
+        if w.k:
+            b200sp.spmm_csr_host(A.m, A.n, A.nnz, w.k, hs[0], hs[1], hs[2], hs[3], hy, w.alpha, w.beta, dtype, stream)
+        else:
+            b200sp.spmv_csr_host(A.m, A.n, A.nnz, hs[0], hs[1], hs[2], hs[3], hy, w.alpha, w.beta, dtype, stream)
+
+    e2e_steps = max(3, min(steps, 10))
+    for _ in range(3):
+        host_call()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        host_call()
+    torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    el = 4 if dtype == "f32" else 2
+    h2d = sum(int(h.numel() * h.element_size()) for h in hs) + (A.m * kk * el if w.beta != 0 else 0)
+    d2h = A.m * kk * el
+    e2e = {"value": world * head["algorithmic_bytes"] / e2e_s * 1e-9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3, "steps": e2e_steps,
+           "note": "spmv_csr_host: pinned host buffers, H2D of all CSR arrays and operands, plan, kernels, D2H of y, sync"}
+
+    # ---- other workloads (bounded): same protocol, fewer steps
+    extras = {}
+    if not args.no_extras and rank == 0:
+        del head["_sets"], head["_call"]
+        torch.cuda.empty_cache()
+        todo = [("c2", "bf16"), ("c3", "f32"), ("c4", "bf16"), ("c1", "f32"), ("c5k64", "f32"), ("c5k64", "bf16"),
+                ("c5k256", "f32"), ("c5k256", "bf16")]
+        cache = {args.workload: w}
+        for name, dt in todo:
+            if (name, dt) == (args.workload, dtype):
+                continue
+            try:
+                ww = cache.get(name) or gen.workload(name)
+                cache = {name: ww}
+                r = measure(ww, dt, min(steps, 50), 5, dev, l2)
+                extras["%s_%s" % (name, dt)] = {
+                    "ms_per_step": round(r["ms_per_step"], 5), "ms_isolated_median": round(r["ms_per_step_isolated_median"], 5),
+                    "gbs": round(r["gbs"], 1), "frac_of_hbm": round(r["gbs"] / peak, 4), "gflops": round(r["gflops"], 1),
+                    "algorithmic_bytes": r["algorithmic_bytes"], "nnz": r["nnz"], "copies": r["copies"],
+                    "plan_ms_first_call": round(r["plan_ms_first_call"], 3)}
+                del r
+                b200sp.b200sp_cache_clear()
+                torch.cuda.empty_cache()
+            except Exception as ex:  # pragma: no cover
+                extras["%s_%s" % (name, dt)] = {"error": repr(ex)}
+    sampler.stop()
+
+    # ---- CPU baseline: the oracle on the host cores, same workload (rank 0, N = 1 only)
+    cpu = None
+    if rank == 0 and world == 1:
+        import oracle
+        nt = oracle.max_threads()
+        vals_s, in_s = stored(A.vals, dtype), stored(w.B if w.k else w.x, dtype)
+        y0_s = stored(w.y0, dtype) if w.beta != 0 else None
+        best, best1, y_ref, S_ref = 1e30, 1e30, None, None
+        if w.k:
+            rows = np.arange(0, A.m, max(1, A.m // 4096), dtype=np.int64)
+            run = lambda n_t: oracle.spmm_csr(A.m, A.n, w.k, A.row_ptr, A.col_idx, vals_s, in_s, y0_s, w.alpha, w.beta, dtype, rows=rows, nthreads=n_t)
+            frac_rows, sample = len(rows) / A.m, "%d sampled rows of the workload" % len(rows)
+        else:
+            run = lambda n_t: oracle.spmv_csr(A.m, A.n, A.row_ptr, A.col_idx, vals_s, in_s, y0_s, w.alpha, w.beta, dtype, nthreads=n_t)
+            frac_rows, sample = 1.0, "whole workload, best of 3, OpenMP over rows"
+        for _ in range(3):
+            t = time.perf_counter(); y_ref, S_ref = run(nt); best = min(best, time.perf_counter() - t)
+        t = time.perf_counter(); run(1); best1 = time.perf_counter() - t
+        cpu = {"value": head["algorithmic_bytes"] * frac_rows / best * 1e-9, "unit": "GB/s", "cores": nt, "kind": "oracle",
+               "sample": sample, "ms": best * 1e3, "ms_single_thread": best1 * 1e3}
+
+    if rank == 0:
+        config = {"workload": "%s: %s" % (args.workload, {
+            "c2": "CSR SpMV m=n=2^20, exactly 16 nnz/row uniform sorted columns, vals N(0,1), alpha=1.5 beta=0.5"}.get(args.workload, w.A.name)),
+            "m": A.m, "n": A.n, "nnz": A.nnz, "k": w.k, "alpha": w.alpha, "beta": w.beta,
+            "algorithmic_bytes_per_step": head["algorithmic_bytes"], "gflops": world * head["gflops"],
+            "l2": "steps rotate over %d device copies of all operands (%.0f MB in total, L2 is %.0f MB); no flush in the timed region"
+                  % (head["copies"], head["copies"] * head["algorithmic_bytes"] / 1e6, l2 / 1e6),
+            "plan": "cached per row_ptr; first call incl. plan %.3f ms (excluded)" % head["plan_ms_first_call"],
+            "ms_per_step_isolated_median": head["ms_per_step_isolated_median"],
+            "parallelism": "replicas only (single-GPU path)" if world > 1 else "1 GPU"}
+        achieved = head["algorithmic_bytes"] / (head["ms_total"] / steps) * 1e-6
+        line = {"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+                "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dtype,
+                "data": "synthetic", "config": config, "clocks": clocks, "e2e": e2e,
+                "gpu_launches": int(head["launches"]),
+                "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                             "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dtype)), "peak_kind": "of " + peak_kind,
+                             "note": "whole step (merge-tile kernel + carry fix-up) per call; algorithmic bytes per step over event time per step"},
+                "cpu_baseline": cpu, "extra": extras}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
