@@ -244,6 +244,7 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="only the headline workload")
     ap.add_argument("--workload", default="c2", help="headline workload (default c2)")
     ap.add_argument("--dtype", default="f32")
+    ap.add_argument("--opt", action="append", default=[], help="library tuning switch name=value (b200sp_set_option), repeatable")
     ap.add_argument("--profile", action="store_true",
                     help="short run for a profiler: the timed loop of one workload only (no clock loop, e2e, extras, CPU baseline)")
     args = ap.parse_args()
@@ -267,6 +268,9 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(dev))
         barrier = lambda: (dist.barrier(), torch.cuda.synchronize())
+    for o in args.opt:
+        name, val = o.split("=")
+        b200sp.b200sp_set_option(name, int(val))
     peak, peak_kind = measured_peaks()
     l2 = torch.cuda.get_device_properties(local).L2_cache_size
     steps, warmup = max(args.steps, 1), max(args.warmup, 3)

@@ -54,7 +54,8 @@ typedef enum {
   B200SP_ERR_CUDA = 3,
   B200SP_ERR_ALLOC = 4,
   B200SP_ERR_ARCH = 5,
-  B200SP_ERR_BAD_CSR = 6
+  B200SP_ERR_BAD_CSR = 6,
+  B200SP_ERR_TIMEOUT = 7
 } b200sp_status;
 
 /* Opaque: row statistics, row bins, nnz-balanced tile splits and the scratch the kernels need. */
@@ -69,9 +70,10 @@ typedef struct {
   int32_t min_row_len, max_row_len;
   int64_t bin_rows[B200SP_NUM_BINS];  /* rows per length bin */
   int64_t bin_nnz[B200SP_NUM_BINS];   /* nonzeros held by the rows of each bin */
-  int32_t spmv_kernel;                /* 0 = merge-tile kernel (rows + nnz balanced), 1 = row-direct kernel */
-  int32_t spmv_tile_items;            /* merge items (rows + nonzeros) per SpMV tile */
-  int32_t spmv_tiles;                 /* number of SpMV tiles */
+  int32_t spmv_kernel;                /* 0 = merge-tile kernel (rows + nnz balanced), 1 = row-direct kernel,
+                                         2 = uniform-row sub-warp kernel */
+  int32_t spmv_tile_items;            /* merge items (rows + nonzeros) per merge tile */
+  int32_t spmv_tiles;                 /* number of merge tiles */
   int32_t spmm_tile_nnz;              /* nonzeros per SpMM work unit */
   int32_t spmm_tiles;                 /* number of SpMM work units */
   int64_t scratch_bytes;              /* device memory held by the plan */
@@ -127,13 +129,25 @@ const char* b200sp_status_string(int status);  /* static string, never NULL */
 const char* b200sp_last_cuda_error(void);      /* message of this thread's last failing CUDA call, "" if none */
 int b200sp_version(void);                      /* major * 10000 + minor * 100 + patch */
 
+/* Synchronises `stream`, then reports whether any kernel of this library on the current device gave up
+ * on a bounded wait (a staged copy that never signalled its barrier): B200SP_ERR_TIMEOUT if so (the
+ * flag is cleared), else B200SP_OK.  The kernels never spin without a limit; a result produced by a
+ * launch that timed out is incomplete. */
+int b200sp_check(void* stream);
+
 /* Number of kernels this library has launched from this process so far (all entry points). */
 int64_t b200sp_launch_count(void);
 
 /* Tuning switches for A/B measurements; unknown names return B200SP_ERR_INVALID_ARG.
- *   "spmv_kernel"   -1 = choose from the plan statistics (default), 0 = merge-tile, 1 = row-direct
+ *   "spmv_kernel"   -1 = choose from the plan statistics (default), 0 = merge-tile, 1 = row-direct,
+ *                    2 = uniform-row; a kernel the matrix is not eligible for falls back to an eligible one
+ *   "uni_unroll"     groups of four nonzeros in flight per thread of the uniform-row kernel: 1, 2 or 4
+ *   "uni_ctas"       CTAs per SM for the uniform-row kernel, 0 = as many as fit
  *   "x_l2_window"    1 = pin x / B in L2 with a per-launch access-policy window (default), 0 = off
- * A change applies to plans created afterwards. */
+ *   "row_stages"     shared-memory stages per CTA of the row-direct kernel, 2..4
+ *   "row_ctas"       CTAs per SM the row-direct kernel sizes its tiles for, 1..4
+ *   "row_unroll"     gathers in flight per thread in the row-direct kernel: 4, 8 or 16
+ * "spmv_kernel" applies to plans created afterwards, the others to the next call. */
 int b200sp_set_option(const char* name, int value);
 
 #ifdef __cplusplus

@@ -3,6 +3,6 @@
 The Python layer only marshals arguments (see ``binding``); the product is the CUDA library built
 from ``csrc/`` and declared in ``include/b200sp.h``.
 """
-from .binding import (BF16, F32, B200spError, b200sp_cache_clear, b200sp_launch_count, b200sp_plan_create,  # noqa: F401
+from .binding import (BF16, F32, B200spError, b200sp_cache_clear, b200sp_check, b200sp_launch_count, b200sp_plan_create,  # noqa: F401
                       b200sp_plan_destroy, b200sp_plan_info, b200sp_set_option, b200sp_spmm, b200sp_spmv,
                       b200sp_validate_csr, b200sp_version, lib, spmm_csr, spmm_csr_host, spmv_csr, spmv_csr_host)

@@ -20,6 +20,7 @@ EXPORTS = (
     "spmv_csr", "spmm_csr", "b200sp_plan_create", "b200sp_plan_destroy", "b200sp_plan_info", "b200sp_spmv",
     "b200sp_spmm", "spmv_csr_host", "spmm_csr_host", "b200sp_validate_csr", "b200sp_cache_clear",
     "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_launch_count", "b200sp_set_option",
+    "b200sp_check",
 )
 
 
@@ -76,6 +77,8 @@ def lib() -> ctypes.CDLL:
         L.b200sp_version.restype = i32
         L.b200sp_launch_count.restype = i64
         L.b200sp_set_option.argtypes = [ctypes.c_char_p, i32]
+        L.b200sp_check.argtypes = [p]
+        L.b200sp_check.restype = i32
         for name in ("spmv_csr", "spmm_csr", "spmv_csr_host", "spmm_csr_host", "b200sp_plan_create", "b200sp_plan_destroy",
                      "b200sp_plan_info", "b200sp_spmv", "b200sp_spmm", "b200sp_validate_csr", "b200sp_set_option"):
             getattr(L, name).restype = i32
@@ -160,6 +163,11 @@ def b200sp_validate_csr(m, n, nnz, row_ptr, col_idx, stream=None) -> int:
     if rc not in (0, 6):
         raise B200spError(rc, "b200sp_validate_csr")
     return rc
+
+
+def b200sp_check(stream=None):
+    """Synchronises the stream; raises B200spError(status 7) if a kernel gave up on a bounded wait."""
+    _ck(lib().b200sp_check(_stream(stream)), "b200sp_check")
 
 
 def b200sp_cache_clear():

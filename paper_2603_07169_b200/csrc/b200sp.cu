@@ -14,6 +14,8 @@
 #include "common.cuh"
 #include "plan_kernels.cuh"
 #include "spmv_kernels.cuh"
+#include "spmv_row_kernels.cuh"
+#include "spmv_uniform_kernels.cuh"
 #include "spmm_kernels.cuh"
 
 using namespace b200sp;
@@ -26,6 +28,10 @@ constexpr int kVersion = 100;  // 0.1.0
 constexpr int kItems = 4096;
 constexpr int kThreads = 256;
 constexpr int kShortMax = 32;
+// SpMV row-direct kernel: eligibility and shared-memory budget (two CTAs per SM)
+constexpr int kRowThreads = 256;
+constexpr int kRowMaxLen = 64;
+constexpr int kSmemPerSm = 227 * 1024;   // usable shared memory per SM (each CTA also reserves 1 KB)
 // SpMM
 constexpr int kSpmmThreads = 256;
 constexpr int kSpmmTileNnz = 4096;
@@ -37,12 +43,20 @@ std::mutex g_mutex;
 struct Options {
   int spmv_kernel = -1;
   int x_l2_window = 1;
+  int row_stages = 3;   // shared-memory stages per CTA of the row-direct kernel (2..4)
+  int row_ctas = 2;     // CTAs per SM the row-direct kernel is sized for (1..4)
+  int row_unroll = 8;   // gathers in flight per thread (8 or 16)
+  int row_smem_kb = 220;  // shared memory per SM the row-direct kernel may use for its stages (the rest stays L1)
+  int row_threads = 256;  // threads per CTA of the row-direct kernel (128 or 256)
+  int uni_unroll = 2;     // groups of four nonzeros in flight per thread of the uniform-row kernel (1, 2 or 4)
+  int uni_ctas = 0;       // CTAs per SM for the uniform-row kernel (0 = as many as fit)
 } g_opt;
 
 struct DeviceInfo {
   bool known = false;
   int cc_major = 0, sms = 0, persist_max = 0, window_max = 0, l2_bytes = 0;
   size_t persist_set = 0;
+  int* err_flag = nullptr;  // device int: set by a kernel whose bounded wait ran out
 };
 DeviceInfo g_dev[64];
 
@@ -71,6 +85,8 @@ int device_info(DeviceInfo** out) {
     CU(cudaDeviceGetAttribute(&d.persist_max, cudaDevAttrMaxPersistingL2CacheSize, dev));
     CU(cudaDeviceGetAttribute(&d.window_max, cudaDevAttrMaxAccessPolicyWindowSize, dev));
     CU(cudaDeviceGetAttribute(&d.l2_bytes, cudaDevAttrL2CacheSize, dev));
+    CU(cudaMalloc(&d.err_flag, sizeof(int)));
+    CU(cudaMemset(d.err_flag, 0, sizeof(int)));
     d.known = true;
   }
   *out = &d;
@@ -79,12 +95,12 @@ int device_info(DeviceInfo** out) {
 
 // Launch with an optional L2 access-policy window (persisting hits) over the gathered operand.
 template <typename... KArgs, typename... Args>
-int launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream, const void* win_ptr, size_t win_bytes,
-           DeviceInfo* dev, Args... args) {
+int launch_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, const void* win_ptr,
+                size_t win_bytes, DeviceInfo* dev, Args... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
-  cfg.dynamicSmemBytes = 0;
+  cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   cfg.attrs = attr;
@@ -112,6 +128,12 @@ int launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream,
   CU(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return B200SP_OK;
+}
+
+template <typename... KArgs, typename... Args>
+int launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream, const void* win_ptr, size_t win_bytes,
+           DeviceInfo* dev, Args... args) {
+  return launch_smem(kernel, grid, block, 0, stream, win_ptr, win_bytes, dev, args...);
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -196,6 +218,19 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   if (h.bad) { plan_free(p); return B200SP_ERR_BAD_CSR; }
   I.min_row_len = h.min_len; I.max_row_len = h.max_len;
   for (int j = 0; j < B200SP_NUM_BINS; ++j) { I.bin_rows[j] = (int64_t)h.bin_rows[j]; I.bin_nnz[j] = (int64_t)h.bin_nnz[j]; }
+  // Kernel choice from the row statistics: when every row is short and the mean is not far below the
+  // maximum, a thread per row wastes little and rows never need splitting -> row-direct kernel.
+  // Anything with long or very uneven rows goes to the merge-tile kernel.
+  const bool row_direct_ok = nnz > 0 && h.max_len <= kRowMaxLen && aligned16(row_ptr) &&
+                             (h.max_len <= 8 || nnz * 4 >= (int64_t)h.max_len * m);
+  // Rows all of one length 4, 8, ..., 128: sub-warp-per-row kernel with 128-bit loads and no shared memory.
+  const bool uniform_ok = nnz > 0 && h.min_len == h.max_len && h.max_len >= 4 && h.max_len <= 128 && (h.max_len & (h.max_len - 1)) == 0;
+  const bool row_direct_possible = nnz > 0 && h.max_len <= kRowMaxLen && aligned16(row_ptr);
+  int choice = uniform_ok ? 2 : (row_direct_ok ? 1 : 0);
+  if (g_opt.spmv_kernel == 0) choice = 0;
+  if (g_opt.spmv_kernel == 1) choice = row_direct_possible ? 1 : 0;
+  if (g_opt.spmv_kernel == 2) choice = uniform_ok ? 2 : (row_direct_ok ? 1 : 0);
+  I.spmv_kernel = choice;
   *out = p;
   return B200SP_OK;
 }
@@ -209,12 +244,113 @@ int run_scale(long long count, T* y, float beta, cudaStream_t stream, DeviceInfo
   return launch(scale_kernel<T>, dim3((unsigned)blocks), dim3(256), stream, nullptr, 0, dev, count, y, beta);
 }
 
+int gcd_int(int a, int b) { while (b) { const int t = a % b; a = b; b = t; } return a; }
+
+template <typename T, int THREADS, int UNROLL, bool ROT>
+int launch_row_direct(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
+                      cudaStream_t stream, DeviceInfo* dev, int rot_lanes) {
+  const b200sp_plan_info_t& I = p->info;
+  const int max_len = I.max_row_len > 0 ? I.max_row_len : 1;
+  const int stages = g_opt.row_stages, ctas = g_opt.row_ctas;
+  int sm_budget = g_opt.row_smem_kb * 1024;
+  if (sm_budget > kSmemPerSm) sm_budget = kSmemPerSm;
+  const int cta_budget = sm_budget / ctas - 1024 - 256;
+  const int stage_budget = cta_budget / stages;
+  const int cap_max = (stage_budget - (THREADS + 4) * 4 - 64) / (4 + (int)sizeof(T));
+  int R = (cap_max - 16) / max_len;
+  if (R > THREADS) R = THREADS;
+  R &= ~3;
+  if (R < 4) return B200SP_ERR_UNSUPPORTED;
+  const int cap = (R * max_len + 16 + 7) & ~7;
+  const int tiles = (int)((I.m + R - 1) / R);
+  const size_t smem = (size_t)stages * row_tile_stage_bytes<T>(R, cap);
+  auto kernel = spmv_row_tile_kernel<T, THREADS, UNROLL, ROT>;
+  static int configured[64] = {};   // per instantiation and device: the carveout last set (percent + 1)
+  int carve = (int)(((size_t)ctas * (smem + 1024 + 128) * 100 + (size_t)kSmemPerSm) / ((size_t)kSmemPerSm + 1024)) + 1;
+  if (carve > 100) carve = 100;
+  if (configured[p->device] != carve + 1) {
+    CU(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerSm - 1024));
+    CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve));
+    configured[p->device] = carve + 1;
+  }
+  const int grid = tiles < ctas * dev->sms ? tiles : ctas * dev->sms;
+  return launch_smem(kernel, dim3(grid), dim3(THREADS), smem, stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz,
+                     p->row_ptr, col_idx, vals, x, y, alpha, beta, R, cap, tiles, stages, rot_lanes, dev->err_flag);
+}
+
+template <typename T>
+int run_spmv_row_direct(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
+                        cudaStream_t stream, DeviceInfo* dev) {
+  const b200sp_plan_info_t& I = p->info;
+  // equal-length rows: start each lane's walk at a different offset so that a warp's shared-memory reads spread over the banks
+  int rot_lanes = 0;
+  if (I.min_row_len == I.max_row_len && I.max_row_len > 1) {
+    const int g = gcd_int(I.max_row_len, 32);
+    if (g > 1) rot_lanes = 32 / g;
+  }
+#define ROW_DISPATCH(TH, U)                                                                                              \
+  return rot_lanes ? launch_row_direct<T, TH, U, true>(p, col_idx, vals, x, y, alpha, beta, stream, dev, rot_lanes)    \
+                   : launch_row_direct<T, TH, U, false>(p, col_idx, vals, x, y, alpha, beta, stream, dev, 0)
+  if (g_opt.row_threads == 128) {
+    if (g_opt.row_unroll == 16) { ROW_DISPATCH(128, 16); }
+    ROW_DISPATCH(128, 8);
+  }
+  if (g_opt.row_unroll == 16) { ROW_DISPATCH(256, 16); }
+  ROW_DISPATCH(256, 8);
+#undef ROW_DISPATCH
+}
+
+template <typename T, int LPR, int UNROLL>
+int launch_uniform(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
+                   cudaStream_t stream, DeviceInfo* dev) {
+  constexpr int THREADS = 256;
+  const b200sp_plan_info_t& I = p->info;
+  auto kernel = spmv_uniform_vec_kernel<T, LPR, UNROLL, THREADS>;
+  static int per_sm[64] = {};   // per instantiation and device
+  if (!per_sm[p->device]) {
+    CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 0));   // all of the unified cache as L1
+    int nb = 0;
+    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kernel, THREADS, 0));
+    per_sm[p->device] = nb > 0 ? nb : 1;
+  }
+  const int ctas = g_opt.uni_ctas > 0 && g_opt.uni_ctas < per_sm[p->device] ? g_opt.uni_ctas : per_sm[p->device];
+  const long long quads = I.nnz / 4;
+  long long blocks = (quads + (long long)THREADS * UNROLL - 1) / ((long long)THREADS * UNROLL);
+  const long long cap = (long long)dev->sms * ctas;
+  if (blocks > cap) blocks = cap;
+  return launch(kernel, dim3((unsigned)blocks), dim3(THREADS), stream, x, (size_t)I.n * sizeof(T), dev, quads, col_idx, vals, x, y, alpha, beta);
+}
+
+template <typename T, int LPR>
+int run_spmv_uniform_u(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
+                       cudaStream_t stream, DeviceInfo* dev) {
+  if (g_opt.uni_unroll == 1) return launch_uniform<T, LPR, 1>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  if (g_opt.uni_unroll == 4) return launch_uniform<T, LPR, 4>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  return launch_uniform<T, LPR, 2>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+}
+
+template <typename T>
+int run_spmv_uniform(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
+                     cudaStream_t stream, DeviceInfo* dev) {
+  switch (p->info.max_row_len / 4) {
+    case 1: return run_spmv_uniform_u<T, 1>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+    case 2: return run_spmv_uniform_u<T, 2>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+    case 4: return run_spmv_uniform_u<T, 4>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+    case 8: return run_spmv_uniform_u<T, 8>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+    case 16: return run_spmv_uniform_u<T, 16>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+    case 32: return run_spmv_uniform_u<T, 32>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  }
+  return B200SP_ERR_UNSUPPORTED;
+}
+
 template <typename T>
 int run_spmv(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
              cudaStream_t stream, DeviceInfo* dev) {
   const b200sp_plan_info_t& I = p->info;
   if (I.m == 0) return B200SP_OK;
   if (alpha == 0.0f || I.nnz == 0) return run_scale<T>(I.m, y, beta, stream, dev);
+  if (I.spmv_kernel == 2) return run_spmv_uniform<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  if (I.spmv_kernel == 1) return run_spmv_row_direct<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   const int tiles = I.spmv_tiles;
   int rc = launch(spmv_merge_tile_kernel<T, kItems, kThreads, kShortMax>, dim3(tiles), dim3(kThreads), stream, x,
                   (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx, vals, x, y, alpha, beta,
@@ -447,8 +583,21 @@ const char* b200sp_status_string(int s) {
     case B200SP_ERR_ALLOC: return "allocation failed";
     case B200SP_ERR_ARCH: return "device is not compute capability 10.x (B200)";
     case B200SP_ERR_BAD_CSR: return "CSR arrays are inconsistent";
+    case B200SP_ERR_TIMEOUT: return "a kernel gave up on a bounded wait";
     default: return "unknown status";
   }
+}
+
+int b200sp_check(void* stream_v) {
+  DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  int h = 0;
+  CU(cudaMemcpyAsync(&h, dev->err_flag, sizeof(int), cudaMemcpyDeviceToHost, stream));
+  CU(cudaStreamSynchronize(stream));
+  if (h) { CU(cudaMemsetAsync(dev->err_flag, 0, sizeof(int), stream)); CU(cudaStreamSynchronize(stream)); return B200SP_ERR_TIMEOUT; }
+  return B200SP_OK;
 }
 
 const char* b200sp_last_cuda_error(void) { return g_last_error.c_str(); }
@@ -458,8 +607,15 @@ int64_t b200sp_launch_count(void) { return g_launches.load(); }
 int b200sp_set_option(const char* name, int value) {
   if (!name) return B200SP_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
-  if (!strcmp(name, "spmv_kernel")) { if (value < -1 || value > 1) return B200SP_ERR_INVALID_ARG; g_opt.spmv_kernel = value; return B200SP_OK; }
+  if (!strcmp(name, "uni_unroll")) { if (value != 1 && value != 2 && value != 4) return B200SP_ERR_INVALID_ARG; g_opt.uni_unroll = value; return B200SP_OK; }
+  if (!strcmp(name, "uni_ctas")) { if (value < 0 || value > 32) return B200SP_ERR_INVALID_ARG; g_opt.uni_ctas = value; return B200SP_OK; }
+  if (!strcmp(name, "spmv_kernel")) { if (value < -1 || value > 2) return B200SP_ERR_INVALID_ARG; g_opt.spmv_kernel = value; return B200SP_OK; }
   if (!strcmp(name, "x_l2_window")) { g_opt.x_l2_window = value ? 1 : 0; return B200SP_OK; }
+  if (!strcmp(name, "row_stages")) { if (value < 2 || value > kRowMaxStages) return B200SP_ERR_INVALID_ARG; g_opt.row_stages = value; return B200SP_OK; }
+  if (!strcmp(name, "row_smem_kb")) { if (value < 16 || value > 227) return B200SP_ERR_INVALID_ARG; g_opt.row_smem_kb = value; return B200SP_OK; }
+  if (!strcmp(name, "row_threads")) { if (value != 128 && value != 256) return B200SP_ERR_INVALID_ARG; g_opt.row_threads = value; return B200SP_OK; }
+  if (!strcmp(name, "row_ctas")) { if (value < 1 || value > 8) return B200SP_ERR_INVALID_ARG; g_opt.row_ctas = value; return B200SP_OK; }
+  if (!strcmp(name, "row_unroll")) { if (value != 8 && value != 16) return B200SP_ERR_INVALID_ARG; g_opt.row_unroll = value; return B200SP_OK; }
   return B200SP_ERR_INVALID_ARG;
 }
 

@@ -1,0 +1,58 @@
+// Sub-warp-per-row CSR SpMV kernel for matrices whose rows all have the same length L = 4 * LPR,
+// LPR a power of two (plan: min row length == max row length):
+// y = alpha * A * x + beta * y  (paper, Appendix C, Table 6, task 12, with alpha/beta).
+//
+// With equal rows, row r starts at nonzero r * L, so row_ptr need not be read and every group of
+// four nonzeros is 16-byte aligned: each lane streams one int4 of col_idx and four vals with
+// 128-bit coalesced loads, gathers four x entries through the read-only path, and LPR adjacent lanes
+// combine their partial sums with __shfl_xor.  No shared memory is used, so the whole unified cache
+// serves as L1 for the gather (its capacity bounds the number of misses in flight, which is what
+// limits a gather over a vector much larger than L1).  UNROLL independent groups per thread keep
+// 4 * UNROLL gathers in flight.  The reduction order is fixed, so results are bit-reproducible.
+#pragma once
+#include "common.cuh"
+
+namespace b200sp {
+
+template <typename T, int LPR, int UNROLL, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+spmv_uniform_vec_kernel(long long quads, const int* __restrict__ col_idx, const T* __restrict__ vals,
+                        const T* __restrict__ x, T* __restrict__ y, float alpha, float beta) {
+  const long long stride = (long long)gridDim.x * THREADS;
+  long long g = (long long)blockIdx.x * THREADS + threadIdx.x;
+  // every lane of a warp runs the same number of iterations: quads is a multiple of LPR and warps start on multiples of 32
+  for (; g < quads; g += stride * UNROLL) {
+    int4 c[UNROLL];
+    float v[UNROLL][4];
+    bool ok[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const long long q = g + (long long)u * stride;
+      ok[u] = q < quads;
+      if (ok[u]) {
+        c[u] = ld_stream_i4(col_idx + q * 4);
+        ld_stream_vals4(vals + q * 4, v[u]);
+      }
+    }
+    float part[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      part[u] = 0.0f;
+      if (ok[u]) {
+        const float x0 = ld_gather(x + c[u].x), x1 = ld_gather(x + c[u].y), x2 = ld_gather(x + c[u].z), x3 = ld_gather(x + c[u].w);
+        part[u] = fmaf(v[u][3], x3, fmaf(v[u][2], x2, fmaf(v[u][1], x1, v[u][0] * x0)));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const long long q = g + (long long)u * stride;
+      // the lanes of one row either all pass `ok` or all fail it, and whole warps stay converged here
+      float s = part[u];
+#pragma unroll
+      for (int o = 1; o < LPR; o <<= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+      if (ok[u] && (q & (LPR - 1)) == 0) epilogue_store(y, q / LPR, s, alpha, beta);
+    }
+  }
+}
+
+}  // namespace b200sp

@@ -75,6 +75,7 @@ def test_invalid_arguments_are_rejected_on_the_host():
     assert L.b200sp_plan_info(None, None) == BAD
     assert L.b200sp_set_option(b"no_such_option", 1) == BAD
     assert L.b200sp_set_option(b"spmv_kernel", 5) == BAD
+    assert L.b200sp_set_option(b"row_unroll", 3) == BAD
 
 
 def test_empty_problem_is_a_no_op_without_a_device():

@@ -34,13 +34,31 @@ def row_len_cases():
         "random_geometric": rng.geometric(0.08, 5000) - 1,
         "tile_exact": np.full(4096 // 17 * 3, 16),          # rows + nnz = multiple of the tile size
         "power_law": (rng.pareto(1.2, 3000) * 3).astype(np.int64).clip(0, 40000),
+        "uniform_16": np.full(5003, 16),
+        "uniform_27_ragged_rows": np.full(1001, 27),
+        "uniform_64": np.full(777, 64),
+        "uniform_4": np.full(4001, 4),
+        "uniform_8": np.full(3001, 8),
+        "uniform_32": np.full(1501, 32),
+        "uniform_128": np.full(301, 128),
+        "short_mixed_0_to_8": rng.integers(0, 9, 10007),
+        "stencil_like": np.tile([8, 12, 18, 27, 27, 27, 27, 18], 500),
     }
     return cases
 
 
+@pytest.fixture(params=[-1, 0, 1, 2], ids=["auto", "merge_tile", "row_direct", "uniform"])
+def kernel_choice(request):
+    """Runs a test under each SpMV kernel selection (1 falls back to 0 inside the plan when rows are too long)."""
+    b200sp.b200sp_set_option("spmv_kernel", request.param)
+    yield request.param
+    b200sp.b200sp_set_option("spmv_kernel", -1)
+    b200sp.b200sp_check()
+
+
 @pytest.mark.parametrize("dtype", DTYPES)
 @pytest.mark.parametrize("case", sorted(row_len_cases()))
-def test_adversarial_row_lengths(case, dtype):
+def test_adversarial_row_lengths(case, dtype, kernel_choice):
     lens = row_len_cases()[case]
     m = len(lens)
     n = 777
@@ -67,7 +85,7 @@ def test_empty_rows_are_exactly_zero_and_nan_in_y_is_ignored(dtype):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
-def test_n_equal_one_and_m_not_multiple_of_anything(dtype):
+def test_n_equal_one_and_m_not_multiple_of_anything(dtype, kernel_choice):
     rng = np.random.default_rng(3)
     m = 4099
     lens = rng.integers(0, 4, m)
@@ -108,7 +126,7 @@ def test_integer_data_is_exact_fp32():
 
 # ---------------------------------------------------------------- the measured workloads
 @pytest.mark.parametrize("name,scale", [("c1", 0), ("c2", 2), ("c3", 2), ("c4", 2)])
-def test_workloads_scaled(name, scale):
+def test_workloads_scaled(name, scale, kernel_choice):
     w = gen.workload(name, scale_down=scale)
     for dtype in w.dtypes:
         y, y_ref, S = run_spmv(w.A, w.x, w.y0, w.alpha, w.beta, dtype, use_plan=(dtype == "bf16"))
@@ -157,6 +175,12 @@ def test_plan_info_matches_numpy():
         sel = (L >= lo) & (L <= hi)
         assert info["bin_rows"][j] == sel.sum() and info["bin_nnz"][j] == L[sel].sum()
     assert info["spmv_tiles"] == -(-(A.m + A.nnz) // info["spmv_tile_items"])
+    assert info["spmv_kernel"] == 0          # power-law rows: merge-tile kernel
+    w = gen.workload("c4", scale_down=2)
+    plan = b200sp.b200sp_plan_create(w.A.m, w.A.n, w.A.nnz, to_dev(w.A.row_ptr))
+    info = b200sp.b200sp_plan_info(plan)
+    b200sp.b200sp_plan_destroy(plan)
+    assert info["spmv_kernel"] == 1 and info["max_row_len"] == 27      # short regular rows: row-direct kernel
 
 
 def test_validate_csr():
