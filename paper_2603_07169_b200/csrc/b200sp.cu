@@ -43,8 +43,8 @@ std::mutex g_mutex;
 struct Options {
   int spmv_kernel = -1;
   int x_l2_window = 1;
-  int row_stages = 3;   // shared-memory stages per CTA of the row-direct kernel (2..4)
-  int row_ctas = 2;     // CTAs per SM the row-direct kernel is sized for (1..4)
+  int row_stages = 2;   // shared-memory stages per CTA of the row-direct kernel (2..4)
+  int row_ctas = 3;     // CTAs per SM the row-direct kernel is sized for (1..4)
   int row_unroll = 8;   // gathers in flight per thread (8 or 16)
   int row_smem_kb = 220;  // shared memory per SM the row-direct kernel may use for its stages (the rest stays L1)
   int row_threads = 256;  // threads per CTA of the row-direct kernel (128 or 256)
@@ -85,12 +85,20 @@ int device_info(DeviceInfo** out) {
     CU(cudaDeviceGetAttribute(&d.persist_max, cudaDevAttrMaxPersistingL2CacheSize, dev));
     CU(cudaDeviceGetAttribute(&d.window_max, cudaDevAttrMaxAccessPolicyWindowSize, dev));
     CU(cudaDeviceGetAttribute(&d.l2_bytes, cudaDevAttrL2CacheSize, dev));
-    CU(cudaMalloc(&d.err_flag, sizeof(int)));
-    CU(cudaMemset(d.err_flag, 0, sizeof(int)));
     d.known = true;
   }
   *out = &d;
   return d.cc_major == 10 ? B200SP_OK : B200SP_ERR_ARCH;
+}
+
+// The flag that kernels with bounded waits raise; allocated on first use (those kernels only).
+int ensure_err_flag(DeviceInfo* d) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!d->err_flag) {
+    CU(cudaMalloc(&d->err_flag, sizeof(int)));
+    CU(cudaMemset(d->err_flag, 0, sizeof(int)));
+  }
+  return B200SP_OK;
 }
 
 // Launch with an optional L2 access-policy window (persisting hits) over the gathered operand.
@@ -274,6 +282,8 @@ int launch_row_direct(b200sp_plan* p, const int32_t* col_idx, const T* vals, con
     configured[p->device] = carve + 1;
   }
   const int grid = tiles < ctas * dev->sms ? tiles : ctas * dev->sms;
+  const int rc_flag = ensure_err_flag(dev);
+  if (rc_flag != B200SP_OK) return rc_flag;
   return launch_smem(kernel, dim3(grid), dim3(THREADS), smem, stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz,
                      p->row_ptr, col_idx, vals, x, y, alpha, beta, R, cap, tiles, stages, rot_lanes, dev->err_flag);
 }
@@ -594,6 +604,7 @@ int b200sp_check(void* stream_v) {
   if (rc != B200SP_OK) return rc;
   cudaStream_t stream = (cudaStream_t)stream_v;
   int h = 0;
+  if (!dev->err_flag) { CU(cudaStreamSynchronize(stream)); return B200SP_OK; }   // no kernel with a bounded wait has run yet
   CU(cudaMemcpyAsync(&h, dev->err_flag, sizeof(int), cudaMemcpyDeviceToHost, stream));
   CU(cudaStreamSynchronize(stream));
   if (h) { CU(cudaMemsetAsync(dev->err_flag, 0, sizeof(int), stream)); CU(cudaStreamSynchronize(stream)); return B200SP_ERR_TIMEOUT; }
