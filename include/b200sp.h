@@ -55,7 +55,8 @@ typedef enum {
   B200SP_ERR_ALLOC = 4,
   B200SP_ERR_ARCH = 5,
   B200SP_ERR_BAD_CSR = 6,
-  B200SP_ERR_TIMEOUT = 7
+  B200SP_ERR_TIMEOUT = 7,
+  B200SP_ERR_TOO_LARGE = 8
 } b200sp_status;
 
 /* Opaque: row statistics, row bins, nnz-balanced tile splits and the scratch the kernels need. */
@@ -107,6 +108,30 @@ int b200sp_spmv(b200sp_plan* plan, const int32_t* col_idx, const void* vals, con
                 float alpha, float beta, int dtype, void* stream);
 int b200sp_spmm(b200sp_plan* plan, int64_t k, const int32_t* col_idx, const void* vals, const void* B, void* Y,
                 float alpha, float beta, int dtype, void* stream);
+
+/* ---- SpMV without any allocation ---------------------------------------------------------------
+ * (The paper has no counterpart for this entry point; it exists for callers of this library.)
+ *
+ * Some callers may not allocate device memory at all: code running inside a region where the
+ * allocator is off limits (a real-time or safety-certified loop whose memory was fixed at start-up,
+ * a plugin that must not touch its host's memory pools, a caller that has already handed every byte
+ * of the GPU to its own arena).  For them spmv_csr_noalloc computes the same y = alpha*A*x + beta*y
+ * as spmv_csr with the merge-tile kernel and its carry fix-up, but takes the scratch those kernels
+ * need (tile split points, carries, tails) from a fixed array compiled into the library instead of a
+ * plan: it calls no cudaMalloc / cudaFree and no allocating routine, builds no plan, caches nothing
+ * and never synchronises.  All pointers are device pointers, as for spmv_csr.
+ *
+ *  - Limit: m + nnz <= b200sp_noalloc_max_items() (268,435,456; the array is about 0.75 MB, held by
+ *    every GPU that loads the library until the process exits).  Larger problems are refused with
+ *    B200SP_ERR_TOO_LARGE and nothing is launched.
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *    that device current).  Make that first call before starting any stream capture.
+ *  - Every call uses the same array and finds the previous call's contents in it; each call rewrites
+ *    all the entries it later reads, so nothing needs clearing.  Two calls whose kernels overlap on the
+ *    GPU (different streams, no ordering between them) race on the array: order them. */
+int spmv_csr_noalloc(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx,
+                     const void* vals, const void* x, void* y, float alpha, float beta, int dtype, void* stream);
+int64_t b200sp_noalloc_max_items(void);   /* largest m + nnz that spmv_csr_noalloc accepts */
 
 /* ---- host-buffer calls -----------------------------------------------------------------------
  * Same operations with every array in HOST memory (pinned memory makes the copies asynchronous and

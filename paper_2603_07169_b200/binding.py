@@ -20,7 +20,7 @@ EXPORTS = (
     "spmv_csr", "spmm_csr", "b200sp_plan_create", "b200sp_plan_destroy", "b200sp_plan_info", "b200sp_spmv",
     "b200sp_spmm", "spmv_csr_host", "spmm_csr_host", "b200sp_validate_csr", "b200sp_cache_clear",
     "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_launch_count", "b200sp_set_option",
-    "b200sp_check",
+    "b200sp_check", "spmv_csr_noalloc", "b200sp_noalloc_max_items",
 )
 
 
@@ -62,6 +62,9 @@ def lib() -> ctypes.CDLL:
         L.spmv_csr.argtypes = [i64, i64, i64, p, p, p, p, p, f32, f32, i32, p]
         L.spmm_csr.argtypes = [i64, i64, i64, i64, p, p, p, p, p, f32, f32, i32, p]
         L.spmv_csr_host.argtypes = L.spmv_csr.argtypes
+        L.spmv_csr_noalloc.argtypes = L.spmv_csr.argtypes
+        L.spmv_csr_noalloc.restype = i32
+        L.b200sp_noalloc_max_items.restype = i64
         L.spmm_csr_host.argtypes = L.spmm_csr.argtypes
         L.b200sp_plan_create.argtypes = [ctypes.POINTER(p), i64, i64, i64, p, p]
         L.b200sp_plan_destroy.argtypes = [p]
@@ -121,6 +124,17 @@ def spmv_csr(m, n, nnz, row_ptr, col_idx, vals, x, y, alpha, beta, dtype, stream
 def spmm_csr(m, n, nnz, k, row_ptr, col_idx, vals, B, Y, alpha, beta, dtype, stream=None):
     _ck(lib().spmm_csr(m, n, nnz, k, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(B), _ptr(Y), alpha, beta, _dt(dtype),
                        _stream(stream)), "spmm_csr")
+
+
+def spmv_csr_noalloc(m, n, nnz, row_ptr, col_idx, vals, x, y, alpha, beta, dtype, stream=None):
+    """SpMV for callers that may not allocate device memory: scratch comes from a fixed array inside the
+    library (m + nnz <= b200sp_noalloc_max_items()); overlapping calls race on that array."""
+    _ck(lib().spmv_csr_noalloc(m, n, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype),
+                               _stream(stream)), "spmv_csr_noalloc")
+
+
+def b200sp_noalloc_max_items() -> int:
+    return lib().b200sp_noalloc_max_items()
 
 
 def spmv_csr_host(m, n, nnz, row_ptr, col_idx, vals, x, y, alpha, beta, dtype, stream=None):

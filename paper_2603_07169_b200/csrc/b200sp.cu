@@ -430,6 +430,49 @@ int get_cached_plan(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const 
 
 }  // namespace
 
+// ---- scratch for spmv_csr_noalloc: lives in the library image, one copy per GPU that loads it ----
+constexpr int kNoAllocMaxTiles = 65536;   // merge tiles of kItems items: m + nnz <= 65536 * 4096 = 268,435,456
+struct NoAllocScratch {
+  int32_t split_row[kNoAllocMaxTiles + 4];
+  float carry[kNoAllocMaxTiles];
+  float tail[kNoAllocMaxTiles];
+};
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+// In host code the name above is only a handle; the device address comes from cudaGetSymbolAddress,
+// looked up once per device with that device current.
+static NoAllocScratch* g_noalloc_ptr[64] = {};
+
+static int noalloc_scratch(NoAllocScratch** out) {
+  int dev = 0;
+  CU(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return B200SP_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!g_noalloc_ptr[dev]) {
+    void* ptr = nullptr;
+    CU(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+    g_noalloc_ptr[dev] = static_cast<NoAllocScratch*>(ptr);
+  }
+  *out = g_noalloc_ptr[dev];
+  return B200SP_OK;
+}
+
+template <typename T>
+static int run_spmv_noalloc(int64_t m, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx, const T* vals, const T* x, T* y,
+                            float alpha, float beta, cudaStream_t stream, DeviceInfo* dev, NoAllocScratch* sc) {
+  if (alpha == 0.0f || nnz == 0) return run_scale<T>(m, y, beta, stream, dev);
+  const int tiles = (int)((m + nnz + kItems - 1) / kItems);
+  int rc = launch(plan_merge_split_kernel, dim3((tiles + 1 + 255) / 256), dim3(256), stream, nullptr, 0, dev, row_ptr, (int)m, (int)nnz,
+                  kItems, tiles, (int*)sc->split_row);
+  if (rc != B200SP_OK) return rc;
+  rc = launch(spmv_merge_tile_kernel<T, kItems, kThreads, kShortMax>, dim3(tiles), dim3(kThreads), stream, nullptr, 0, dev, (int)m,
+              (int)nnz, row_ptr, col_idx, vals, x, y, alpha, beta, (const int*)sc->split_row, sc->carry, sc->tail);
+  if (rc != B200SP_OK) return rc;
+  if (tiles > 1)
+    rc = launch(spmv_carry_fixup_kernel<T, kItems>, dim3((tiles + 127) / 128), dim3(128), stream, nullptr, 0, dev, tiles, row_ptr,
+                (const int*)sc->split_row, (const float*)sc->carry, (const float*)sc->tail, y, alpha, beta);
+  return rc;
+}
+
 extern "C" {
 
 int b200sp_plan_create(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, void* stream) {
@@ -502,6 +545,29 @@ int spmm_csr(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_pt
   if (rc != B200SP_OK) return rc;
   return b200sp_spmm(p, k, col_idx, vals, B, Y, alpha, beta, dtype, stream);
 }
+
+int spmv_csr_noalloc(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx, const void* vals,
+                     const void* x, void* y, float alpha, float beta, int dtype, void* stream) {
+  int rc = check_sizes(m, n, nnz);
+  if (rc != B200SP_OK) return rc;
+  if (dtype != B200SP_F32 && dtype != B200SP_BF16) return B200SP_ERR_INVALID_ARG;
+  if (m > 0 && (!row_ptr || !y)) return B200SP_ERR_INVALID_ARG;
+  if (nnz > 0 && (!col_idx || !vals || !x)) return B200SP_ERR_INVALID_ARG;
+  if (!aligned4(row_ptr) || !aligned16(col_idx) || !aligned16(vals) || !aligned16(x) || !aligned16(y)) return B200SP_ERR_INVALID_ARG;
+  if (m + nnz > (int64_t)kNoAllocMaxTiles * kItems) return B200SP_ERR_TOO_LARGE;   // beyond the built-in scratch
+  if (m == 0) return B200SP_OK;
+  DeviceInfo* dev = nullptr;
+  rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  NoAllocScratch* sc = nullptr;
+  rc = noalloc_scratch(&sc);
+  if (rc != B200SP_OK) return rc;
+  if (dtype == B200SP_F32)
+    return run_spmv_noalloc<float>(m, nnz, row_ptr, col_idx, (const float*)vals, (const float*)x, (float*)y, alpha, beta, (cudaStream_t)stream, dev, sc);
+  return run_spmv_noalloc<bf16_t>(m, nnz, row_ptr, col_idx, (const bf16_t*)vals, (const bf16_t*)x, (bf16_t*)y, alpha, beta, (cudaStream_t)stream, dev, sc);
+}
+
+int64_t b200sp_noalloc_max_items(void) { return (int64_t)kNoAllocMaxTiles * kItems; }
 
 // ---- host-buffer entry points: copy in, plan, run, copy out, synchronise ----
 static int host_call(bool is_mm, int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_ptr, const int32_t* col_idx,
@@ -594,6 +660,7 @@ const char* b200sp_status_string(int s) {
     case B200SP_ERR_ARCH: return "device is not compute capability 10.x (B200)";
     case B200SP_ERR_BAD_CSR: return "CSR arrays are inconsistent";
     case B200SP_ERR_TIMEOUT: return "a kernel gave up on a bounded wait";
+    case B200SP_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }
