@@ -166,6 +166,13 @@ int64_t b200sp_launch_count(void);
 /* Tuning switches for A/B measurements; unknown names return B200SP_ERR_INVALID_ARG.
  *   "spmv_kernel"   -1 = choose from the plan statistics (default), 0 = merge-tile, 1 = row-direct,
  *                    2 = uniform-row; a kernel the matrix is not eligible for falls back to an eligible one
+ *   "spmm_sliced"    1 = SpMM walks k in 128-byte slices so that a slice of B stays in L2 (default), 0 = one pass
+ *   "merge_staged"   1 = persistent staged merge kernel, 0 = one tile per CTA (default)
+ *   "merge_threads"  threads per CTA of the one-tile-per-CTA merge kernel, 128 or 256
+ *   "merge_carve"    shared-memory carveout in percent requested for it (-1 = driver default)
+ *   "merge_items"    merge items per tile, 2048 or 4096 (applies to plans created afterwards)
+ *   "merge_stages"   shared-memory stages per CTA of the staged merge kernel, 2..4
+ *   "merge_ctas"     CTAs per SM of the staged merge kernel
  *   "uni_unroll"     groups of four nonzeros in flight per thread of the uniform-row kernel: 1, 2 or 4
  *   "uni_ctas"       CTAs per SM for the uniform-row kernel, 0 = as many as fit
  *   "x_l2_window"    1 = pin x / B in L2 with a per-launch access-policy window (default), 0 = off

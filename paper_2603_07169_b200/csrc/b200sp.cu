@@ -8,7 +8,9 @@
 #include <cstring>
 #include <map>
 #include <mutex>
+#include <algorithm>
 #include <string>
+#include <vector>
 #include <tuple>
 
 #include "common.cuh"
@@ -16,6 +18,7 @@
 #include "spmv_kernels.cuh"
 #include "spmv_row_kernels.cuh"
 #include "spmv_uniform_kernels.cuh"
+#include "spmv_merge_stage_kernels.cuh"
 #include "spmm_kernels.cuh"
 
 using namespace b200sp;
@@ -35,6 +38,7 @@ constexpr int kSmemPerSm = 227 * 1024;   // usable shared memory per SM (each CT
 // SpMM
 constexpr int kSpmmThreads = 256;
 constexpr int kSpmmTileNnz = 4096;
+constexpr int kLongRow = 1024;   // rows longer than this get a CTA of their own in SpMM (last length bin of the plan)
 
 thread_local std::string g_last_error;
 std::atomic<int64_t> g_launches{0};
@@ -50,6 +54,13 @@ struct Options {
   int row_threads = 256;  // threads per CTA of the row-direct kernel (128 or 256)
   int uni_unroll = 2;     // groups of four nonzeros in flight per thread of the uniform-row kernel (1, 2 or 4)
   int uni_ctas = 0;       // CTAs per SM for the uniform-row kernel (0 = as many as fit)
+  int merge_staged = 0;   // 1 = persistent staged merge kernel, 0 = one-tile-per-CTA merge kernel
+  int merge_items = 2048; // merge items per tile (2048 or 4096)
+  int merge_stages = 3;   // shared-memory stages per CTA of the staged merge kernel (2..4)
+  int merge_ctas = 2;     // CTAs per SM of the staged merge kernel
+  int merge_threads = 128; // threads per CTA of the one-tile-per-CTA merge kernel (128 or 256)
+  int spmm_sliced = 1;     // 1 = k-sliced SpMM kernel (default), 0 = one pass over all of k
+  int merge_carve = 30;    // shared-memory carveout (percent) requested for it, -1 = leave to the driver
 } g_opt;
 
 struct DeviceInfo {
@@ -164,6 +175,8 @@ struct b200sp_plan {
   float* carry = nullptr;             // spmv tiles
   float* tail = nullptr;              // spmv tiles
   int32_t* spmm_split_row = nullptr;  // spmm tiles + 1
+  int32_t* long_rows = nullptr;       // rows longer than kLongRow, ascending
+  int num_long = 0;
 };
 
 namespace {
@@ -173,7 +186,7 @@ std::map<std::tuple<int, const void*, int64_t, int64_t, int64_t>, b200sp_plan*> 
 int plan_free(b200sp_plan* p) {
   if (!p) return B200SP_OK;
   int rc = B200SP_OK;
-  for (void* q : {(void*)p->split_row, (void*)p->carry, (void*)p->tail, (void*)p->spmm_split_row})
+  for (void* q : {(void*)p->split_row, (void*)p->carry, (void*)p->tail, (void*)p->spmm_split_row, (void*)p->long_rows})
     if (q) { cudaError_t e = cudaFree(q); if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree"); }
   delete p;
   return rc;
@@ -188,8 +201,9 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   p->row_ptr = row_ptr;
   b200sp_plan_info_t& I = p->info;
   I.m = m; I.n = n; I.nnz = nnz;
-  I.spmv_tile_items = kItems;
-  I.spmv_tiles = (int32_t)((m + nnz + kItems - 1) / kItems);
+  const int items = g_opt.merge_items == 4096 ? 4096 : 2048;
+  I.spmv_tile_items = items;
+  I.spmv_tiles = (int32_t)((m + nnz + items - 1) / items);
   I.spmm_tile_nnz = kSpmmTileNnz;
   I.spmm_tiles = (int32_t)((nnz + kSpmmTileNnz - 1) / kSpmmTileNnz);
   I.spmv_kernel = g_opt.spmv_kernel >= 0 ? g_opt.spmv_kernel : 0;
@@ -214,7 +228,7 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   CUP(cudaMalloc(&p->tail, (nt + 1) * sizeof(float)));
   CUP(cudaMalloc(&p->spmm_split_row, (ns + 1) * sizeof(int32_t)));
   I.scratch_bytes = (int64_t)((nt + 1) * 12 + (ns + 1) * 4);
-  plan_merge_split_kernel<<<(unsigned)((nt + 1 + 255) / 256), 256, 0, stream>>>(row_ptr, (int)m, (int)nnz, kItems, (int)nt, p->split_row);
+  plan_merge_split_kernel<<<(unsigned)((nt + 1 + 255) / 256), 256, 0, stream>>>(row_ptr, (int)m, (int)nnz, items, (int)nt, p->split_row);
   plan_nnz_split_kernel<<<(unsigned)((ns + 1 + 255) / 256), 256, 0, stream>>>(row_ptr, (int)m, (int)nnz, kSpmmTileNnz, (int)ns, p->spmm_split_row);
   g_launches += 2;
   CUP(cudaGetLastError());
@@ -222,6 +236,28 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   CUP(cudaStreamSynchronize(stream));
   CUP(cudaFree(d_stats));
   d_stats = nullptr;
+  if (!h.bad && h.bin_rows[4] > 0) {   // list of the rows in the last length bin (> kLongRow), sorted on the host
+    const int cap = (int)h.bin_rows[4];
+    int* d_count = nullptr;
+    CUP(cudaMalloc(&p->long_rows, (size_t)cap * sizeof(int32_t)));
+    CUP(cudaMalloc(&d_count, sizeof(int)));
+    cudaError_t e = cudaMemsetAsync(d_count, 0, sizeof(int), stream);
+    if (e == cudaSuccess) {
+      const int blocks = (int)((m + 255) / 256);
+      plan_long_rows_kernel<<<blocks < dev->sms * 8 ? blocks : dev->sms * 8, 256, 0, stream>>>(row_ptr, (int)m, kLongRow, cap, p->long_rows, d_count);
+      g_launches++;
+      e = cudaGetLastError();
+    }
+    std::vector<int32_t> tmp((size_t)cap);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(tmp.data(), p->long_rows, (size_t)cap * sizeof(int32_t), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e == cudaSuccess) { std::sort(tmp.begin(), tmp.end()); e = cudaMemcpyAsync(p->long_rows, tmp.data(), (size_t)cap * sizeof(int32_t), cudaMemcpyHostToDevice, stream); }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    cudaFree(d_count);
+    if (e != cudaSuccess) return fail(cuda_fail(e, "plan long-row list"));
+    p->num_long = cap;
+    I.scratch_bytes += (int64_t)cap * 4;
+  }
 #undef CUP
   if (h.bad) { plan_free(p); return B200SP_ERR_BAD_CSR; }
   I.min_row_len = h.min_len; I.max_row_len = h.max_len;
@@ -353,6 +389,48 @@ int run_spmv_uniform(b200sp_plan* p, const int32_t* col_idx, const T* vals, cons
   return B200SP_ERR_UNSUPPORTED;
 }
 
+template <typename T, int ITEMS>
+int run_spmv_merge(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
+                   cudaStream_t stream, DeviceInfo* dev) {
+  const b200sp_plan_info_t& I = p->info;
+  const int tiles = I.spmv_tiles;
+  int rc;
+  if (g_opt.merge_staged) {
+    const int stages = g_opt.merge_stages, ctas = g_opt.merge_ctas;
+    auto kernel = spmv_merge_stage_kernel<T, ITEMS, kThreads, kShortMax>;
+    const size_t smem = (size_t)stages * merge_stage_bytes<T>(ITEMS);
+    if ((size_t)ctas * (smem + 2048) > (size_t)kSmemPerSm) return B200SP_ERR_UNSUPPORTED;
+    static int configured[64] = {};
+    int carve = (int)(((size_t)ctas * (smem + 2048) * 100 + (size_t)kSmemPerSm) / ((size_t)kSmemPerSm + 1024)) + 1;
+    if (carve > 100) carve = 100;
+    if (configured[p->device] != carve + 1) {
+      CU(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerSm - 2048));
+      CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve));
+      configured[p->device] = carve + 1;
+    }
+    rc = ensure_err_flag(dev);
+    if (rc != B200SP_OK) return rc;
+    const int grid = tiles < ctas * dev->sms ? tiles : ctas * dev->sms;
+    rc = launch_smem(kernel, dim3(grid), dim3(kThreads), smem, stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr,
+                     col_idx, vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail, tiles, stages, dev->err_flag);
+  } else if (g_opt.merge_threads == 128) {
+    auto kernel = spmv_merge_tile_kernel<T, ITEMS, 128, kShortMax>;
+    if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
+    rc = launch(kernel, dim3(tiles), dim3(128), stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx,
+                vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail);
+  } else {
+    auto kernel = spmv_merge_tile_kernel<T, ITEMS, kThreads, kShortMax>;
+    if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
+    rc = launch(kernel, dim3(tiles), dim3(kThreads), stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx,
+                vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail);
+  }
+  if (rc != B200SP_OK) return rc;
+  if (tiles > 1)
+    rc = launch(spmv_carry_fixup_kernel<T, ITEMS>, dim3((tiles + 127) / 128), dim3(128), stream, nullptr, 0, dev, tiles,
+                p->row_ptr, (const int*)p->split_row, (const float*)p->carry, (const float*)p->tail, y, alpha, beta);
+  return rc;
+}
+
 template <typename T>
 int run_spmv(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
              cudaStream_t stream, DeviceInfo* dev) {
@@ -361,15 +439,8 @@ int run_spmv(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, 
   if (alpha == 0.0f || I.nnz == 0) return run_scale<T>(I.m, y, beta, stream, dev);
   if (I.spmv_kernel == 2) return run_spmv_uniform<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (I.spmv_kernel == 1) return run_spmv_row_direct<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
-  const int tiles = I.spmv_tiles;
-  int rc = launch(spmv_merge_tile_kernel<T, kItems, kThreads, kShortMax>, dim3(tiles), dim3(kThreads), stream, x,
-                  (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx, vals, x, y, alpha, beta,
-                  (const int*)p->split_row, p->carry, p->tail);
-  if (rc != B200SP_OK) return rc;
-  if (tiles > 1)
-    rc = launch(spmv_carry_fixup_kernel<T, kItems>, dim3((tiles + 127) / 128), dim3(128), stream, nullptr, 0, dev, tiles,
-                p->row_ptr, (const int*)p->split_row, (const float*)p->carry, (const float*)p->tail, y, alpha, beta);
-  return rc;
+  if (I.spmv_tile_items == 4096) return run_spmv_merge<T, 4096>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  return run_spmv_merge<T, 2048>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
 }
 
 template <typename T, int VEC, int LANES, int NCH>
@@ -387,6 +458,18 @@ int run_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const
   const b200sp_plan_info_t& I = p->info;
   if (I.m == 0) return B200SP_OK;
   if (alpha == 0.0f || I.nnz == 0) return run_scale<T>((long long)I.m * k, Y, beta, stream, dev);
+  if (k % VEC == 0 && g_opt.spmm_sliced) {
+    constexpr int KS = 8 * VEC, GROUPS = kSpmmThreads / 8;
+    const int slices = (k + KS - 1) / KS;
+    const int row_blocks = (int)((I.m + GROUPS - 1) / GROUPS);
+    if ((long long)slices * row_blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+    int rc = launch(spmm_slice_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)(slices * row_blocks)), dim3(kSpmmThreads), stream,
+                    nullptr, 0, dev,
+                    (int)I.m, k, row_blocks, p->row_ptr, col_idx, vals, B, Y, alpha, beta, kLongRow);
+    if (rc != B200SP_OK || p->num_long == 0) return rc;
+    return launch(spmm_long_row_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)(slices * p->num_long)), dim3(kSpmmThreads), stream, nullptr, 0,
+                  dev, k, p->num_long, (const int*)p->long_rows, p->row_ptr, col_idx, vals, B, Y, alpha, beta);
+  }
   if (k % VEC != 0) {  // ragged k: scalar lanes
     if (k <= 8) return launch_spmm<T, 1, 8, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
     return launch_spmm<T, 1, 32, 2>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
@@ -685,6 +768,13 @@ int64_t b200sp_launch_count(void) { return g_launches.load(); }
 int b200sp_set_option(const char* name, int value) {
   if (!name) return B200SP_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
+  if (!strcmp(name, "spmm_sliced")) { g_opt.spmm_sliced = value ? 1 : 0; return B200SP_OK; }
+  if (!strcmp(name, "merge_threads")) { if (value != 128 && value != 256) return B200SP_ERR_INVALID_ARG; g_opt.merge_threads = value; return B200SP_OK; }
+  if (!strcmp(name, "merge_carve")) { if (value < -1 || value > 100) return B200SP_ERR_INVALID_ARG; g_opt.merge_carve = value; return B200SP_OK; }
+  if (!strcmp(name, "merge_staged")) { g_opt.merge_staged = value ? 1 : 0; return B200SP_OK; }
+  if (!strcmp(name, "merge_items")) { if (value != 2048 && value != 4096) return B200SP_ERR_INVALID_ARG; g_opt.merge_items = value; return B200SP_OK; }
+  if (!strcmp(name, "merge_stages")) { if (value < 2 || value > kMergeMaxStages) return B200SP_ERR_INVALID_ARG; g_opt.merge_stages = value; return B200SP_OK; }
+  if (!strcmp(name, "merge_ctas")) { if (value < 1 || value > 8) return B200SP_ERR_INVALID_ARG; g_opt.merge_ctas = value; return B200SP_OK; }
   if (!strcmp(name, "uni_unroll")) { if (value != 1 && value != 2 && value != 4) return B200SP_ERR_INVALID_ARG; g_opt.uni_unroll = value; return B200SP_OK; }
   if (!strcmp(name, "uni_ctas")) { if (value < 0 || value > 32) return B200SP_ERR_INVALID_ARG; g_opt.uni_ctas = value; return B200SP_OK; }
   if (!strcmp(name, "spmv_kernel")) { if (value < -1 || value > 2) return B200SP_ERR_INVALID_ARG; g_opt.spmv_kernel = value; return B200SP_OK; }

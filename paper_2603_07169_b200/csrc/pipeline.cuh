@@ -28,6 +28,9 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
+// Orders this thread's earlier generic-proxy accesses to shared memory (and, through a preceding CTA
+// barrier, those of the other threads) before the async-proxy writes of bulk copies issued after it.
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 // Global -> shared bulk copy; src and dst 16-byte aligned, bytes a positive multiple of 16.
 __device__ __forceinline__ void bulk_copy_g2s(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"

@@ -81,6 +81,17 @@ __global__ void __launch_bounds__(256) plan_nnz_split_kernel(const int* __restri
   split_row[t] = lo;
 }
 
+// Rows longer than `thresh`, appended to a list (order of the list only affects scheduling, never a value).
+__global__ void __launch_bounds__(256) plan_long_rows_kernel(const int* __restrict__ row_ptr, int m, int thresh, int capacity,
+                                                             int* __restrict__ list, int* __restrict__ count) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < m; i += (long long)gridDim.x * blockDim.x) {
+    if (row_ptr[i + 1] - row_ptr[i] > thresh) {
+      const int slot = atomicAdd(count, 1);
+      if (slot < capacity) list[slot] = (int)i;
+    }
+  }
+}
+
 // CSR content check on request.
 __global__ void __launch_bounds__(256) validate_csr_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col_idx, int m, int n,
                                                            int nnz, int* bad) {

@@ -119,4 +119,139 @@ spmm_row_group_kernel(int m, int k, const int* __restrict__ row_ptr, const int* 
   }
 }
 
+// Raw 16-byte pieces of a row of B, converted to FP32 only when they are consumed (keeps registers low).
+template <typename T, int VEC> struct RawVec;
+template <> struct RawVec<float, 4> {
+  typedef float4 type;
+  static __device__ __forceinline__ float4 ld(const float* p) { return __ldg((const float4*)p); }
+
+  static __device__ __forceinline__ void fma(const float4& b, float v, float (&acc)[4]) {
+    acc[0] = fmaf(v, b.x, acc[0]); acc[1] = fmaf(v, b.y, acc[1]); acc[2] = fmaf(v, b.z, acc[2]); acc[3] = fmaf(v, b.w, acc[3]);
+  }
+};
+template <> struct RawVec<bf16_t, 8> {
+  typedef uint4 type;
+  static __device__ __forceinline__ uint4 ld(const bf16_t* p) { return __ldg((const uint4*)p); }
+
+  static __device__ __forceinline__ void fma(const uint4& b, float v, float (&acc)[8]) {
+    acc[0] = fmaf(v, __uint_as_float(b.x << 16), acc[0]); acc[1] = fmaf(v, __uint_as_float(b.x & 0xFFFF0000u), acc[1]);
+    acc[2] = fmaf(v, __uint_as_float(b.y << 16), acc[2]); acc[3] = fmaf(v, __uint_as_float(b.y & 0xFFFF0000u), acc[3]);
+    acc[4] = fmaf(v, __uint_as_float(b.z << 16), acc[4]); acc[5] = fmaf(v, __uint_as_float(b.z & 0xFFFF0000u), acc[5]);
+    acc[6] = fmaf(v, __uint_as_float(b.w << 16), acc[6]); acc[7] = fmaf(v, __uint_as_float(b.w & 0xFFFF0000u), acc[7]);
+  }
+};
+
+// four consecutive (col, val) pairs with two broadcast vector loads (p a multiple of 4)
+__device__ __forceinline__ void ld_a4(const int* col_idx, const float* vals, int p, int (&c)[4], float (&v)[4]) {
+  const int4 cc = __ldg((const int4*)(col_idx + p));
+  const float4 vv = __ldg((const float4*)(vals + p));
+  c[0] = cc.x; c[1] = cc.y; c[2] = cc.z; c[3] = cc.w; v[0] = vv.x; v[1] = vv.y; v[2] = vv.z; v[3] = vv.w;
+}
+__device__ __forceinline__ void ld_a4(const int* col_idx, const bf16_t* vals, int p, int (&c)[4], float (&v)[4]) {
+  const int4 cc = __ldg((const int4*)(col_idx + p));
+  const uint2 vv = __ldg((const uint2*)(vals + p));
+  c[0] = cc.x; c[1] = cc.y; c[2] = cc.z; c[3] = cc.w;
+  v[0] = __uint_as_float(vv.x << 16); v[1] = __uint_as_float(vv.x & 0xFFFF0000u);
+  v[2] = __uint_as_float(vv.y << 16); v[3] = __uint_as_float(vv.y & 0xFFFF0000u);
+}
+
+// k-sliced kernel.  The dense dimension is cut into slices of 8 * VEC columns = 128 bytes per row of B,
+// one cache line.  blockIdx.x = slice * row_blocks + row block, so CTAs run slice by slice and the
+// part of B that a slice touches (n lines) can stay in L2 while every row of A passes over it; the
+// price is re-reading col_idx / vals once per slice.  Eight lanes own one row of A; all eight read the
+// row's (col, val) pairs with the same 128-bit loads (a broadcast, served by L1), and each lane keeps its
+// VEC columns of the slice in FP32 registers with four independent 16-byte reads of B in flight.
+// Rows longer than long_thresh are left to spmm_long_row_kernel.
+template <typename T, int VEC, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+spmm_slice_kernel(int m, int k, int row_blocks, const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
+                  const T* __restrict__ vals, const T* __restrict__ B, T* __restrict__ Y, float alpha, float beta, int long_thresh) {
+  constexpr int LANES = 8, GROUPS = THREADS / LANES, KS = LANES * VEC;
+  typedef typename RawVec<T, VEC>::type raw_t;
+  const int slice = blockIdx.x / row_blocks, rb = blockIdx.x - slice * row_blocks;
+  const int g = threadIdx.x / LANES, l8 = threadIdx.x % LANES;
+  const long long row = (long long)rb * GROUPS + g;
+  if (row >= m) return;
+  const int rs = __ldg(row_ptr + row), re = __ldg(row_ptr + row + 1);
+  if (re - rs > long_thresh) return;
+  const int col0 = slice * KS + l8 * VEC;
+  if (col0 >= k) return;
+  const T* Bc = B + col0;
+  float acc[VEC];
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
+  int p = rs;
+  for (; p < re && (p & 3); ++p) {   // up to the first multiple of four
+    const raw_t b = RawVec<T, VEC>::ld(Bc + (long long)__ldg(col_idx + p) * k);
+    RawVec<T, VEC>::fma(b, to_f32(__ldg(vals + p)), acc);
+  }
+  for (; p + 4 <= re; p += 4) {
+    int c[4]; float v[4];
+    ld_a4(col_idx, vals, p, c, v);
+    raw_t b[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) b[u] = RawVec<T, VEC>::ld(Bc + (long long)c[u] * k);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) RawVec<T, VEC>::fma(b[u], v[u], acc);
+  }
+  for (; p < re; ++p) {
+    const raw_t b = RawVec<T, VEC>::ld(Bc + (long long)__ldg(col_idx + p) * k);
+    RawVec<T, VEC>::fma(b, to_f32(__ldg(vals + p)), acc);
+  }
+  T* yp = Y + row * k + col0;
+  float out[VEC];
+  if (beta != 0.0f) {
+    float old[VEC];
+    VecLoad<T, VEC>::ld_plain(yp, old);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) out[j] = alpha * acc[j] + beta * old[j];
+  } else {
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) out[j] = alpha * acc[j];
+  }
+  VecLoad<T, VEC>::st(yp, out);
+}
+
+// One CTA per (long row, slice): the CTA's groups of eight lanes stride over the row's nonzeros, then the
+// per-group partial sums are added in group order through shared memory (fixed order: reproducible).
+template <typename T, int VEC, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+spmm_long_row_kernel(int k, int num_long, const int* __restrict__ long_rows, const int* __restrict__ row_ptr,
+                     const int* __restrict__ col_idx, const T* __restrict__ vals, const T* __restrict__ B, T* __restrict__ Y,
+                     float alpha, float beta) {
+  constexpr int LANES = 8, GROUPS = THREADS / LANES, KS = LANES * VEC;
+  __shared__ float part[GROUPS][KS];
+  const int slice = blockIdx.x / num_long;
+  const long long row = long_rows[blockIdx.x - slice * num_long];
+  const int g = threadIdx.x / LANES, l8 = threadIdx.x % LANES;
+  const int rs = __ldg(row_ptr + row), re = __ldg(row_ptr + row + 1);
+  const int col0 = slice * KS + l8 * VEC;
+  const bool active = col0 < k;
+  const T* Bc = B + col0;
+  float acc[VEC];
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
+  for (int p = rs + g; p < re; p += GROUPS) {
+    const int c = __ldg(col_idx + p);
+    const float v = to_f32(__ldg(vals + p));
+    if (active) {
+      float b[VEC];
+      VecLoad<T, VEC>::ld(Bc + (long long)c * k, b);
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) acc[j] = fmaf(v, b[j], acc[j]);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) part[g][l8 * VEC + j] = acc[j];
+  __syncthreads();
+  if (threadIdx.x < KS) {
+    const int col = slice * KS + threadIdx.x;
+    if (col < k) {
+      float s = 0.0f;
+      for (int gg = 0; gg < GROUPS; ++gg) s += part[gg][threadIdx.x];
+      epilogue_store(Y, row * k + col, s, alpha, beta);
+    }
+  }
+}
+
 }  // namespace b200sp

@@ -94,6 +94,7 @@ spmv_row_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const int*
     const int bulk_nz = max(a1 - a0, 0);
     for (int p = max(a1, a0); p < p1; ++p) { col_s[p - a0] = __ldg(col_idx + p); val_s[p - a0] = __ldg(vals + p); }
     const unsigned bytes = (unsigned)(max(bulk_rows, 0) * 4 + bulk_nz * (4 + (int)sizeof(T)));
+    fence_proxy_async_smem();
     mbar_arrive_expect_tx(bar, bytes);   // release: the plain stores above are visible to whoever observes the flip
     if (bulk_rows > 0) bulk_copy_g2s(smem_addr(rp_s), row_ptr + r0, (unsigned)bulk_rows * 4, bar);
     if (bulk_nz > 0) {

@@ -31,6 +31,27 @@ def test_small_random_all_k(k, dtype):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("sliced", [0, 1])
+def test_long_rows_and_both_kernels(sliced, dtype):
+    """Rows above and below the long-row threshold (1024), with the k-sliced and the one-pass kernel."""
+    b200sp.b200sp_set_option("spmm_sliced", sliced)
+    try:
+        rng = np.random.default_rng(3)
+        lens = np.array([1024, 1025, 0, 5000, 3, 1023, 20000] + [7] * 300)
+        A = gen.random_csr(len(lens), 900, lens, seed=11)
+        for k in (8, 64, 72, 256):
+            B = rng.standard_normal(900 * k).astype(np.float32)
+            Y0 = rng.standard_normal(len(lens) * k).astype(np.float32)
+            Y, Y_ref, S = run_spmm(A, B, k, None, 1.0, 0.0, dtype)
+            assert_within(Y, Y_ref, S, dtype, what="long rows k=%d" % k)
+            Y, Y_ref, S = run_spmm(A, B, k, Y0, -1.0, 0.5, dtype)
+            y0f = Y0 if dtype == "f32" else gen.bf16_to_f32(gen.to_bf16(Y0))
+            assert_within(Y, Y_ref, S, dtype, 1.0, np.abs(0.5 * y0f.astype(np.float64)).reshape(len(lens), k), what="long rows ab k=%d" % k)
+    finally:
+        b200sp.b200sp_set_option("spmm_sliced", 1)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
 def test_spmm_column_equals_spmv(dtype):
     from gpu_util import run_spmv
     rng = np.random.default_rng(1)

@@ -143,6 +143,28 @@ def test_workloads_full_size(name):
         assert_within(y, y_ref, S, dtype, what="%s %s full" % (name, dtype))
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("staged,items,stages", [(0, 2048, 3), (0, 4096, 3), (1, 2048, 2), (1, 2048, 4), (1, 4096, 3)])
+def test_merge_kernel_variants(staged, items, stages, dtype):
+    """Both merge kernels (one tile per CTA; persistent with staged copies) at both tile sizes."""
+    b200sp.b200sp_set_option("spmv_kernel", 0)
+    b200sp.b200sp_set_option("merge_staged", staged)
+    b200sp.b200sp_set_option("merge_items", items)
+    b200sp.b200sp_set_option("merge_stages", stages)
+    try:
+        rng = np.random.default_rng(items + stages)
+        for name, lens in (("power_law", (rng.pareto(1.1, 40000) * 2).astype(np.int64).clip(0, 60000)),
+                           ("every_length", np.arange(300)), ("empty_run", np.concatenate([np.zeros(20000, np.int64), [5000, 1, 0, 7]]))):
+            A = gen.random_csr(len(lens), 3001, lens, seed=7)
+            x = rng.standard_normal(3001).astype(np.float32)
+            y, y_ref, S = run_spmv(A, x, None, 1.0, 0.0, dtype)
+            assert_within(y, y_ref, S, dtype, what="%s staged=%d items=%d" % (name, staged, items))
+        b200sp.b200sp_check()
+    finally:
+        for k, v in (("spmv_kernel", -1), ("merge_staged", 1), ("merge_items", 2048), ("merge_stages", 3)):
+            b200sp.b200sp_set_option(k, v)
+
+
 # ---------------------------------------------------------------- determinism, plan, validation, host API
 @pytest.mark.parametrize("dtype", DTYPES)
 def test_bitwise_run_to_run_determinism(dtype):
@@ -174,7 +196,7 @@ def test_plan_info_matches_numpy():
     for j, (lo, hi) in enumerate(edges):
         sel = (L >= lo) & (L <= hi)
         assert info["bin_rows"][j] == sel.sum() and info["bin_nnz"][j] == L[sel].sum()
-    assert info["spmv_tiles"] == -(-(A.m + A.nnz) // info["spmv_tile_items"])
+    assert info["spmv_tiles"] == -(-(A.m + A.nnz) // info["spmv_tile_items"]) and info["spmv_tile_items"] in (2048, 4096)
     assert info["spmv_kernel"] == 0          # power-law rows: merge-tile kernel
     w = gen.workload("c4", scale_down=2)
     plan = b200sp.b200sp_plan_create(w.A.m, w.A.n, w.A.nnz, to_dev(w.A.row_ptr))
