@@ -36,7 +36,14 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) per launch of the dominant kernel from an ncu capture, keyed by
 # (workload, dtype); None where no capture has been made.  Sources: the summaries under profiles/.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    ("c2", "f32"): 147_020_288,     # profiles/spmv_uniform_vec_c2_f32.md
+    ("c2", "bf16"): 109_364_736,    # profiles/spmv_uniform_vec_c2_bf16.md
+    ("c3", "f32"): 305_818_112,     # profiles/spmv_merge_tile_c3_f32.md
+    ("c4", "bf16"): 690_968_832,    # profiles/spmv_row_tile_c4_bf16.md
+    ("c1", "f32"): 3_163_648,       # profiles/spmv_row_tile_c1_f32.md
+    ("c5k64", "f32"): 1_136_199_368,  # profiles/spmm_slice_c5k64_f32.md
+}
 
 
 def measured_peaks():
@@ -136,7 +143,7 @@ class DeviceSet:
             self.out = torch.zeros(A.m * kk, dtype=torch.float32 if dtype == "f32" else torch.int16, device=dev)
 
 
-def measure(w, dtype, steps, warmup, dev, l2_bytes, barrier=None, min_copies=2, max_bytes=8 << 30):
+def measure(w, dtype, steps, warmup, dev, l2_bytes, barrier=None, min_copies=2, max_bytes=8 << 30, cusparse=None):
     """Times `steps` calls back to back with one CUDA-event pair on the launching stream; the calls rotate
     over R device copies of all operands (R * bytes >= 4 * L2).  Returns a dict of figures."""
     import torch
@@ -195,9 +202,117 @@ def measure(w, dtype, steps, warmup, dev, l2_bytes, barrier=None, min_copies=2, 
     res = {"ms_total": ms, "ms_per_step": ms_step, "ms_per_step_isolated_median": iso[len(iso) // 2], "gbs": abytes / ms_step * 1e-6,
            "gflops": flops / ms_step * 1e-6, "algorithmic_bytes": abytes, "copies": R, "launches": launches,
            "plan_ms_first_call": plan_ms, "t0": t0, "t1": t1, "nnz": A.nnz, "m": A.m}
+    res["cusparse_ms"] = None
+    if cusparse is not None:
+        try:
+            res["cusparse_ms"] = cusparse.time(sets[0], w, dtype, min(steps, 20), stream)
+        except Exception as ex:  # pragma: no cover
+            res["cusparse_ms"] = "unavailable: %r" % (ex,)
     res["_sets"] = sets
     res["_call"] = call
     return res
+
+
+def aggregate_over_ranks(ms_local: float, bytes_per_step: int, steps: int, world: int, dist=None, device="cpu"):
+    """Whole-job figures for N independent replicas: time = max over ranks, work = sum over ranks.
+    Returns (ms_per_step, GB/s).  With world == 1 nothing is communicated."""
+    ms = ms_local
+    if world > 1:
+        import torch
+        t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_step = ms / steps
+    return ms_step, world * bytes_per_step / ms_step * 1e-6
+
+
+def probe_gather_rate(n_elems: int, dev) -> float:
+    """Random 4-byte gathers per second from a table of n_elems floats (rounded up to a power of two), L1-missing."""
+    import torch
+    import paper_2603_07169_b200 as b200sp
+    T = 1 << max(10, (n_elems - 1).bit_length())
+    table = torch.zeros(T, dtype=torch.float32, device=dev)
+    sink = torch.zeros(1, dtype=torch.float32, device=dev)
+    gathers = 1 << 26
+    stream = torch.cuda.current_stream()
+    for _ in range(3):
+        b200sp.b200sp_probe_gather(table, T, gathers, sink, stream)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(5):
+        b200sp.b200sp_probe_gather(table, T, gathers, sink, stream)
+    b.record(stream)
+    b.synchronize()
+    return 5 * gathers / (a.elapsed_time(b) * 1e-3)
+
+
+class CuSparse:
+    """cuSPARSE generic API through ctypes, timed on the same device buffers as a comparison point only."""
+    R_32F, R_16BF, IDX_32I, ORDER_ROW = 0, 14, 2, 2
+
+    def __init__(self):
+        import ctypes
+        self.c = ctypes
+        self.lib = None
+        for name in ("libcusparse.so.12", "libcusparse.so"):
+            try:
+                self.lib = ctypes.CDLL(name)
+                break
+            except OSError:
+                continue
+        if self.lib is None:
+            raise OSError("libcusparse not found")
+        self.h = ctypes.c_void_p()
+        self._ck(self.lib.cusparseCreate(ctypes.byref(self.h)))
+
+    def _ck(self, rc):
+        if rc != 0:
+            raise RuntimeError("cuSPARSE status %d" % rc)
+
+    def time(self, s, w, dtype, steps, stream):
+        """Median-free mean time per call (ms) of cusparseSpMV / cusparseSpMM on device set s (preprocess excluded)."""
+        import torch
+        c, L = self.c, self.lib
+        A = w.A
+        vt = self.R_32F if dtype == "f32" else self.R_16BF
+        vp = c.c_void_p
+        self._ck(L.cusparseSetStream(self.h, vp(stream.cuda_stream)))
+        mat = vp()
+        self._ck(L.cusparseCreateCsr(c.byref(mat), c.c_int64(A.m), c.c_int64(A.n), c.c_int64(A.nnz), vp(s.rp.data_ptr()), vp(s.ci.data_ptr()),
+                                     vp(s.va.data_ptr()), self.IDX_32I, self.IDX_32I, 0, vt))
+        alpha, beta = c.c_float(w.alpha), c.c_float(w.beta)
+        size = c.c_size_t(0)
+        out = s.out.clone()
+        if w.k:
+            dB, dC = vp(), vp()
+            self._ck(L.cusparseCreateDnMat(c.byref(dB), c.c_int64(A.n), c.c_int64(w.k), c.c_int64(w.k), vp(s.inp.data_ptr()), vt, self.ORDER_ROW))
+            self._ck(L.cusparseCreateDnMat(c.byref(dC), c.c_int64(A.m), c.c_int64(w.k), c.c_int64(w.k), vp(out.data_ptr()), vt, self.ORDER_ROW))
+            args = (self.h, 0, 0, c.byref(alpha), mat, dB, c.byref(beta), dC, self.R_32F, 0)
+            self._ck(L.cusparseSpMM_bufferSize(*args, c.byref(size)))
+            buf = torch.empty(max(size.value, 16), dtype=torch.uint8, device=s.va.device)
+            if hasattr(L, "cusparseSpMM_preprocess"):
+                self._ck(L.cusparseSpMM_preprocess(*args, vp(buf.data_ptr())))
+            run = lambda: L.cusparseSpMM(*args, vp(buf.data_ptr()))
+        else:
+            dX, dY = vp(), vp()
+            self._ck(L.cusparseCreateDnVec(c.byref(dX), c.c_int64(A.n), vp(s.inp.data_ptr()), vt))
+            self._ck(L.cusparseCreateDnVec(c.byref(dY), c.c_int64(A.m), vp(out.data_ptr()), vt))
+            args = (self.h, 0, c.byref(alpha), mat, dX, c.byref(beta), dY, self.R_32F, 0)
+            self._ck(L.cusparseSpMV_bufferSize(*args, c.byref(size)))
+            buf = torch.empty(max(size.value, 16), dtype=torch.uint8, device=s.va.device)
+            if hasattr(L, "cusparseSpMV_preprocess"):
+                self._ck(L.cusparseSpMV_preprocess(*args, vp(buf.data_ptr())))
+            run = lambda: L.cusparseSpMV(*args, vp(buf.data_ptr()))
+        for _ in range(3):
+            self._ck(run())
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(steps):
+            self._ck(run())
+        b.record(stream)
+        b.synchronize()
+        L.cusparseDestroySpMat(mat)
+        return a.elapsed_time(b) / steps
 
 
 def run_reference(args):
@@ -279,7 +394,11 @@ def main():
     sampler.start()
     w = gen.workload(args.workload)
     dtype = args.dtype
-    head = measure(w, dtype, steps, warmup, dev, l2, barrier)
+    try:
+        cusp = CuSparse() if (rank == 0 and not args.profile) else None
+    except Exception:  # pragma: no cover
+        cusp = None
+    head = measure(w, dtype, steps, warmup, dev, l2, barrier, cusparse=cusp)
     if args.profile:
         sampler.stop()
         print(json.dumps({"profile_run": args.workload, "dtype": dtype, "ms_per_step": head["ms_per_step"], "gbs": head["gbs"],
@@ -296,13 +415,8 @@ def main():
     clocks = sampler.summary(head["t0"], t_load_end)
 
     # max over ranks of the timed region
-    ms_total = head["ms_total"]
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-    ms_step = ms_total / steps
-    value = world * head["algorithmic_bytes"] / ms_step * 1e-6
+    ms_step, value = aggregate_over_ranks(head["ms_total"], head["algorithmic_bytes"], steps, world, dist if world > 1 else None, dev)
+    gather_rate = probe_gather_rate(w.A.n, dev) if not w.k else None
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     A = w.A
@@ -355,12 +469,15 @@ def main():
             try:
                 ww = cache.get(name) or gen.workload(name)
                 cache = {name: ww}
-                r = measure(ww, dt, min(steps, 50), 5, dev, l2)
+                r = measure(ww, dt, min(steps, 50), 5, dev, l2, cusparse=cusp)
                 extras["%s_%s" % (name, dt)] = {
                     "ms_per_step": round(r["ms_per_step"], 5), "ms_isolated_median": round(r["ms_per_step_isolated_median"], 5),
                     "gbs": round(r["gbs"], 1), "frac_of_hbm": round(r["gbs"] / peak, 4), "gflops": round(r["gflops"], 1),
                     "algorithmic_bytes": r["algorithmic_bytes"], "nnz": r["nnz"], "copies": r["copies"],
-                    "plan_ms_first_call": round(r["plan_ms_first_call"], 3)}
+                    "plan_ms_first_call": round(r["plan_ms_first_call"], 3),
+                    "cusparse_ms": round(r["cusparse_ms"], 5) if isinstance(r["cusparse_ms"], float) else r["cusparse_ms"]}
+                if not ww.k:   # SpMV: time at the measured L1-miss gather rate for this x
+                    extras["%s_%s" % (name, dt)]["gather_bound_ms"] = round(ww.A.nnz / probe_gather_rate(ww.A.n, dev) * 1e3, 5)
                 del r
                 b200sp.b200sp_cache_clear()
                 torch.cuda.empty_cache()
@@ -406,7 +523,12 @@ def main():
                 "gpu_launches": int(head["launches"]),
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                              "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dtype)), "peak_kind": "of " + peak_kind,
-                             "note": "whole step (merge-tile kernel + carry fix-up) per call; algorithmic bytes per step over event time per step"},
+                             "note": "algorithmic bytes per step over event time per step (the step is the SpMV kernel; plan cached)",
+                             "secondary": None if gather_rate is None else {
+                                 "bound": "L1-miss gather (one L2 request per random x read)", "gathers_per_s": gather_rate,
+                                 "ms_at_bound": A.nnz / gather_rate * 1e3, "frac_of_bound": (A.nnz / gather_rate * 1e3) / (head["ms_total"] / steps),
+                                 "note": "measured live with b200sp_probe_gather on a table the size of x"}},
+                "cusparse": {"ms_per_step": head["cusparse_ms"], "note": "cusparseSpMV/SpMM, default algorithm, preprocess excluded, warm (one operand set); comparison point only"},
                 "cpu_baseline": cpu, "extra": extras}
         print(json.dumps(line))
     if world > 1:

@@ -160,6 +160,13 @@ int b200sp_version(void);                      /* major * 10000 + minor * 100 + 
  * launch that timed out is incomplete. */
 int b200sp_check(void* stream);
 
+/* Measurement aid (no counterpart in the paper): enqueues `gathers` independent 4-byte reads of
+ * table[h(i) mod table_elems] (table_elems a power of two, h a hash computed in registers), eight in
+ * flight per thread, on as many CTAs as fit.  Timed by the caller with events it gives the rate at
+ * which the SMs take random reads that miss L1, i.e. the bound on gathering x from a vector much
+ * larger than L1.  `table` (table_elems floats) and `sink` (one float) are device pointers. */
+int b200sp_probe_gather(const float* table, int64_t table_elems, int64_t gathers, float* sink, void* stream);
+
 /* Number of kernels this library has launched from this process so far (all entry points). */
 int64_t b200sp_launch_count(void);
 

@@ -20,7 +20,7 @@ EXPORTS = (
     "spmv_csr", "spmm_csr", "b200sp_plan_create", "b200sp_plan_destroy", "b200sp_plan_info", "b200sp_spmv",
     "b200sp_spmm", "spmv_csr_host", "spmm_csr_host", "b200sp_validate_csr", "b200sp_cache_clear",
     "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_launch_count", "b200sp_set_option",
-    "b200sp_check", "spmv_csr_noalloc", "b200sp_noalloc_max_items",
+    "b200sp_check", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather",
 )
 
 
@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.spmv_csr_noalloc.argtypes = L.spmv_csr.argtypes
         L.spmv_csr_noalloc.restype = i32
         L.b200sp_noalloc_max_items.restype = i64
+        L.b200sp_probe_gather.argtypes = [p, i64, i64, p, p]
+        L.b200sp_probe_gather.restype = i32
         L.spmm_csr_host.argtypes = L.spmm_csr.argtypes
         L.b200sp_plan_create.argtypes = [ctypes.POINTER(p), i64, i64, i64, p, p]
         L.b200sp_plan_destroy.argtypes = [p]
@@ -131,6 +133,11 @@ def spmv_csr_noalloc(m, n, nnz, row_ptr, col_idx, vals, x, y, alpha, beta, dtype
     library (m + nnz <= b200sp_noalloc_max_items()); overlapping calls race on that array."""
     _ck(lib().spmv_csr_noalloc(m, n, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype),
                                _stream(stream)), "spmv_csr_noalloc")
+
+
+def b200sp_probe_gather(table, table_elems, gathers, sink, stream=None):
+    """Enqueues the random-gather probe (see include/b200sp.h); time it with CUDA events."""
+    _ck(lib().b200sp_probe_gather(_ptr(table), table_elems, gathers, _ptr(sink), _stream(stream)), "b200sp_probe_gather")
 
 
 def b200sp_noalloc_max_items() -> int:

@@ -650,6 +650,25 @@ int spmv_csr_noalloc(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, 
   return run_spmv_noalloc<bf16_t>(m, nnz, row_ptr, col_idx, (const bf16_t*)vals, (const bf16_t*)x, (bf16_t*)y, alpha, beta, (cudaStream_t)stream, dev, sc);
 }
 
+int b200sp_probe_gather(const float* table, int64_t table_elems, int64_t gathers, float* sink, void* stream) {
+  if (!table || !sink || table_elems <= 0 || (table_elems & (table_elems - 1)) != 0 || table_elems > ((int64_t)1 << 31) || gathers < 0)
+    return B200SP_ERR_INVALID_ARG;
+  DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  static int per_sm[64] = {};
+  int d = 0;
+  CU(cudaGetDevice(&d));
+  if (!per_sm[d]) {
+    CU(cudaFuncSetAttribute(probe_gather_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 0));
+    int nb = 0;
+    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, probe_gather_kernel, 256, 0));
+    per_sm[d] = nb > 0 ? nb : 1;
+  }
+  return launch(probe_gather_kernel, dim3((unsigned)(dev->sms * per_sm[d])), dim3(256), (cudaStream_t)stream, nullptr, 0, dev, table,
+                (unsigned)(table_elems - 1), (long long)gathers, sink);
+}
+
 int64_t b200sp_noalloc_max_items(void) { return (int64_t)kNoAllocMaxTiles * kItems; }
 
 // ---- host-buffer entry points: copy in, plan, run, copy out, synchronise ----
