@@ -60,6 +60,7 @@ struct Options {
   int merge_ctas = 2;     // CTAs per SM of the staged merge kernel
   int merge_threads = 128; // threads per CTA of the one-tile-per-CTA merge kernel (128 or 256)
   int spmm_sliced = 1;     // 1 = k-sliced SpMM kernel (default), 0 = one pass over all of k
+  int merge_short = 32;    // rows up to this many products are added by one thread (8, 16, 32, 64)
   int merge_carve = 30;    // shared-memory carveout (percent) requested for it, -1 = leave to the driver
 } g_opt;
 
@@ -389,7 +390,7 @@ int run_spmv_uniform(b200sp_plan* p, const int32_t* col_idx, const T* vals, cons
   return B200SP_ERR_UNSUPPORTED;
 }
 
-template <typename T, int ITEMS>
+template <typename T, int ITEMS, int SHORT = kShortMax>
 int run_spmv_merge(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
                    cudaStream_t stream, DeviceInfo* dev) {
   const b200sp_plan_info_t& I = p->info;
@@ -414,7 +415,7 @@ int run_spmv_merge(b200sp_plan* p, const int32_t* col_idx, const T* vals, const 
     rc = launch_smem(kernel, dim3(grid), dim3(kThreads), smem, stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr,
                      col_idx, vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail, tiles, stages, dev->err_flag);
   } else if (g_opt.merge_threads == 128) {
-    auto kernel = spmv_merge_tile_kernel<T, ITEMS, 128, kShortMax>;
+    auto kernel = spmv_merge_tile_kernel<T, ITEMS, 128, SHORT>;
     if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
     rc = launch(kernel, dim3(tiles), dim3(128), stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx,
                 vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail);
@@ -440,6 +441,9 @@ int run_spmv(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, 
   if (I.spmv_kernel == 2) return run_spmv_uniform<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (I.spmv_kernel == 1) return run_spmv_row_direct<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (I.spmv_tile_items == 4096) return run_spmv_merge<T, 4096>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  if (g_opt.merge_short == 8) return run_spmv_merge<T, 2048, 8>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  if (g_opt.merge_short == 16) return run_spmv_merge<T, 2048, 16>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  if (g_opt.merge_short == 64) return run_spmv_merge<T, 2048, 64>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   return run_spmv_merge<T, 2048>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
 }
 
@@ -789,6 +793,7 @@ int b200sp_set_option(const char* name, int value) {
   std::lock_guard<std::mutex> lock(g_mutex);
   if (!strcmp(name, "spmm_sliced")) { g_opt.spmm_sliced = value ? 1 : 0; return B200SP_OK; }
   if (!strcmp(name, "merge_threads")) { if (value != 128 && value != 256) return B200SP_ERR_INVALID_ARG; g_opt.merge_threads = value; return B200SP_OK; }
+  if (!strcmp(name, "merge_short")) { if (value != 8 && value != 16 && value != 32 && value != 64) return B200SP_ERR_INVALID_ARG; g_opt.merge_short = value; return B200SP_OK; }
   if (!strcmp(name, "merge_carve")) { if (value < -1 || value > 100) return B200SP_ERR_INVALID_ARG; g_opt.merge_carve = value; return B200SP_OK; }
   if (!strcmp(name, "merge_staged")) { g_opt.merge_staged = value ? 1 : 0; return B200SP_OK; }
   if (!strcmp(name, "merge_items")) { if (value != 2048 && value != 4096) return B200SP_ERR_INVALID_ARG; g_opt.merge_items = value; return B200SP_OK; }
