@@ -315,6 +315,107 @@ class CuSparse:
         return a.elapsed_time(b) / steps
 
 
+def paper_sweep(args, dev, l2_bytes):
+    """The experiment the paper ran for this operator (Table 6, tasks 12 / 13; Fig. 3a): its own sizes, speed-up over a
+    naive baseline kernel and the complexity-weighted score P = sum T(N_i) S_i / sum T(N_i) (Section 3.3, Eq. 1-2),
+    for this library and for cuSPARSE.  T(N) = nnz for SpMV and nnz * K for SpMM, as in the table."""
+    import torch
+    import gen
+    import paper_2603_07169_b200 as b200sp
+    stream = torch.cuda.current_stream()
+    try:
+        cusp = CuSparse()
+    except Exception:
+        cusp = None
+
+    def timed(fn, sets, steps):
+        for s_ in sets:          # every operand copy once: plans are built and cached here, not in the timed loop
+            fn(s_)
+        for i in range(3):
+            fn(sets[i % len(sets)])
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for i in range(steps):
+            fn(sets[i % len(sets)])
+        b.record(stream)
+        b.synchronize()
+        return a.elapsed_time(b) / steps * 1e3   # us
+
+    def timed_graph(fn, sets, calls=100, replays=5):
+        """Per-call device time (us) of `calls` back-to-back calls replayed from a CUDA graph: no host launch cost."""
+        for s_ in sets:
+            fn(s_)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            cap = torch.cuda.current_stream()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(calls):
+                    fn(sets[i % len(sets)], cap)
+        torch.cuda.current_stream().wait_stream(side)
+        g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(replays):
+            g.replay()
+        b.record()
+        b.synchronize()
+        return a.elapsed_time(b) / (replays * calls) * 1e3
+
+    out = {}
+    spmm_rows = [2 ** 10, 2 ** 12, 2 ** 14, 2 ** 16, 2 ** 18]
+    for op, rows_list, k in (("spmv", [2 ** e for e in range(10, 16)], 0), ("spmm", spmm_rows if not args.quick else spmm_rows[:3], 4096)):
+        for dtype in ("f32", "bf16"):
+            rec = {"rows": [], "nnz": [], "ours_us": [], "naive_us": [], "cusparse_us": []}
+            for rows in rows_list:
+                A = gen.paper_uniform(rows, 2048, 0.01, seed=rows + k)
+                w = gen.Workload("paper", A, x=gen.uniform(2048, -1.0, 1.0, 7, 1), B=(gen.normal(2048 * k, 7, 2) if k else None), k=k)
+                e = 4 if dtype == "f32" else 2
+                abytes = gen.algorithmic_bytes(A.m, A.n, A.nnz, e, 0.0, k)
+                R = int(max(2, min(64, -(-2 * l2_bytes // abytes), (6 << 30) // abytes)))
+                sets = [DeviceSet(w, dtype, dev) for _ in range(R)]
+                if k:
+                    ours = lambda s, st=stream: b200sp.spmm_csr(A.m, A.n, A.nnz, k, s.rp, s.ci, s.va, s.inp, s.out, 1.0, 0.0, dtype, st)
+                    naive = lambda s, st=stream: b200sp.b200sp_spmm_naive(A.m, A.n, A.nnz, k, s.rp, s.ci, s.va, s.inp, s.out, 1.0, 0.0, dtype, st)
+                else:
+                    ours = lambda s, st=stream: b200sp.spmv_csr(A.m, A.n, A.nnz, s.rp, s.ci, s.va, s.inp, s.out, 1.0, 0.0, dtype, st)
+                    naive = lambda s, st=stream: b200sp.b200sp_spmv_naive(A.m, A.n, A.nnz, s.rp, s.ci, s.va, s.inp, s.out, 1.0, 0.0, dtype, st)
+                steps = 200 if not k else max(5, min(100, int(2e11 / (A.nnz * k))))
+                rec["rows"].append(rows); rec["nnz"].append(A.nnz)
+                if k:
+                    rec["ours_us"].append(round(timed(ours, sets, steps), 3))
+                    rec["naive_us"].append(round(timed(naive, sets, max(3, steps // 4)), 3))
+                else:   # a few microseconds per call: replay from a CUDA graph so that the host launch path is not what is timed
+                    rec["ours_us"].append(round(timed_graph(ours, sets), 3))
+                    rec["naive_us"].append(round(timed_graph(naive, sets), 3))
+                    rec.setdefault("ours_host_launched_us", []).append(round(timed(ours, sets, steps), 3))
+                cu = None
+                if cusp is not None:
+                    try:
+                        cu = round(cusp.time(sets[0], w, dtype, steps, stream) * 1e3, 3)
+                    except Exception:
+                        cu = None
+                rec["cusparse_us"].append(cu)
+                del sets
+                b200sp.b200sp_cache_clear()
+                torch.cuda.empty_cache()
+            T = [n * max(k, 1) for n in rec["nnz"]]
+            S = [n / o for n, o in zip(rec["naive_us"], rec["ours_us"])]
+            rec["speedup_ours"] = [round(v, 3) for v in S]
+            rec["P_ours"] = round(sum(t * v for t, v in zip(T, S)) / sum(T), 3)
+            if all(c for c in rec["cusparse_us"]):
+                Sc = [n / c for n, c in zip(rec["naive_us"], rec["cusparse_us"])]
+                rec["speedup_cusparse"] = [round(v, 3) for v in Sc]
+                rec["P_cusparse"] = round(sum(t * v for t, v in zip(T, Sc)) / sum(T), 3)
+            out["%s_%s" % (op, dtype)] = rec
+    print(json.dumps({"paper_sweep": out, "note": "rows x 2048 at density 0.01 (K = 4096 for SpMM); speed-ups over the naive one-thread-per-row "
+                      "(per-entry) kernel; P per the paper's Eq. 1-2 with T = nnz (x K); operands rotate over independent copies; SpMV ours / naive are "
+                      "per-call device times of 100 calls replayed from a CUDA graph, cuSPARSE and SpMM are launched from the host"}))
+
+
 def run_reference(args):
     """The oracle, as it stands, on the host cores, on the headline workload (rank 0 only)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -359,6 +460,8 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="only the headline workload")
     ap.add_argument("--workload", default="c2", help="headline workload (default c2)")
     ap.add_argument("--dtype", default="f32")
+    ap.add_argument("--paper-sweep", action="store_true", help="the paper's own SpMV / SpMM sizes with speed-up over a naive kernel and its score P")
+    ap.add_argument("--quick", action="store_true", help="with --paper-sweep: skip the two largest SpMM sizes")
     ap.add_argument("--opt", action="append", default=[], help="library tuning switch name=value (b200sp_set_option), repeatable")
     ap.add_argument("--profile", action="store_true",
                     help="short run for a profiler: the timed loop of one workload only (no clock loop, e2e, extras, CPU baseline)")
@@ -390,6 +493,10 @@ def main():
     l2 = torch.cuda.get_device_properties(local).L2_cache_size
     steps, warmup = max(args.steps, 1), max(args.warmup, 3)
 
+    if args.paper_sweep:
+        if rank == 0:
+            paper_sweep(args, dev, l2)
+        return
     sampler = ClockSampler(local)
     sampler.start()
     w = gen.workload(args.workload)

@@ -154,6 +154,24 @@ def stencil27(N: int, seed: int, diag: float = 26.0, off: float = -1.0, sigma: f
     return CSR(m, m, rp, ci, va, "stencil27_%d" % N)
 
 
+def paper_uniform(rows: int, cols: int, density: float, seed: int) -> CSR:
+    """The paper's sparse inputs (Table 6, tasks 12 / 13): nnz = floor(rows * cols * density) positions drawn
+    uniformly without replacement over the whole matrix; values N(0, 1)."""
+    nnz = int(rows * cols * density)
+    rng = np.random.default_rng(seed)
+    total = rows * cols
+    pos = np.unique(rng.integers(0, total, int(nnz * 1.1) + 16))
+    while pos.shape[0] < nnz:
+        pos = np.unique(np.concatenate([pos, rng.integers(0, total, nnz)]))
+    pos = np.sort(rng.permutation(pos)[:nnz])
+    r, c = pos // cols, pos % cols
+    rp = np.zeros(rows + 1, np.int64)
+    np.add.at(rp, r + 1, 1)
+    np.cumsum(rp, out=rp)
+    va = rng.standard_normal(nnz).astype(np.float32)
+    return CSR(rows, cols, rp.astype(np.int32), c.astype(np.int32), va, "paper_%dx%d" % (rows, cols))
+
+
 def random_csr(m: int, n: int, row_lens, seed: int, sort_cols: bool = False, integer_vals: bool = False,
                allow_dup: bool = True) -> CSR:
     """Small adversarial matrix: given row lengths, columns uniform (duplicates allowed unless allow_dup

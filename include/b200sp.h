@@ -72,7 +72,7 @@ typedef struct {
   int64_t bin_rows[B200SP_NUM_BINS];  /* rows per length bin */
   int64_t bin_nnz[B200SP_NUM_BINS];   /* nonzeros held by the rows of each bin */
   int32_t spmv_kernel;                /* 0 = merge-tile kernel (rows + nnz balanced), 1 = row-direct kernel,
-                                         2 = uniform-row sub-warp kernel */
+                                         2 = uniform-row sub-warp kernel, 3 = sub-warp-per-row kernel (small problems) */
   int32_t spmv_tile_items;            /* merge items (rows + nonzeros) per merge tile */
   int32_t spmv_tiles;                 /* number of merge tiles */
   int32_t spmm_tile_nnz;              /* nonzeros per SpMM work unit */
@@ -160,6 +160,15 @@ int b200sp_version(void);                      /* major * 10000 + minor * 100 + 
  * launch that timed out is incomplete. */
 int b200sp_check(void* stream);
 
+/* Naive baselines: one thread per row (SpMV) / per output entry (SpMM), scalar loads, sequential sums.
+ * They play the role of the unoptimised baseline kernel that the paper's performance score (Section 3.3,
+ * Eq. 1-2: speed-up over the baseline, weighted by the baseline's complexity T(N)) is measured against.
+ * Same arguments and conventions as spmv_csr / spmm_csr, no plan, no alignment requirement; never used by them. */
+int b200sp_spmv_naive(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx, const void* vals,
+                      const void* x, void* y, float alpha, float beta, int dtype, void* stream);
+int b200sp_spmm_naive(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_ptr, const int32_t* col_idx, const void* vals,
+                      const void* B, void* Y, float alpha, float beta, int dtype, void* stream);
+
 /* Measurement aid (no counterpart in the paper): enqueues `gathers` independent 4-byte reads of
  * table[h(i) mod table_elems] (table_elems a power of two, h a hash computed in registers), eight in
  * flight per thread, on as many CTAs as fit.  Timed by the caller with events it gives the rate at
@@ -172,7 +181,9 @@ int64_t b200sp_launch_count(void);
 
 /* Tuning switches for A/B measurements; unknown names return B200SP_ERR_INVALID_ARG.
  *   "spmv_kernel"   -1 = choose from the plan statistics (default), 0 = merge-tile, 1 = row-direct,
- *                    2 = uniform-row; a kernel the matrix is not eligible for falls back to an eligible one
+ *                    2 = uniform-row, 3 = sub-warp per row; a kernel the matrix is not eligible for falls back
+ *   "sub_lanes"      lanes per row of the sub-warp kernel (1..32, power of two), 0 = from the mean row length
+ *   "spmm_bstage"    1 = SpMM keeps a slice of B in shared memory when A has few columns (default), 0 = never
  *   "spmm_sliced"    1 = SpMM walks k in 128-byte slices so that a slice of B stays in L2 (default), 0 = one pass
  *   "merge_staged"   1 = persistent staged merge kernel, 0 = one tile per CTA (default)
  *   "merge_threads"  threads per CTA of the one-tile-per-CTA merge kernel, 128 or 256
@@ -182,7 +193,8 @@ int64_t b200sp_launch_count(void);
  *   "merge_ctas"     CTAs per SM of the staged merge kernel
  *   "uni_unroll"     groups of four nonzeros in flight per thread of the uniform-row kernel: 1, 2 or 4
  *   "uni_ctas"       CTAs per SM for the uniform-row kernel, 0 = as many as fit
- *   "x_l2_window"    1 = pin x / B in L2 with a per-launch access-policy window (default), 0 = off
+ *   "x_l2_window"    1 = pin x in L2 with a per-launch access-policy window, 0 = off (default: measured to give
+ *                    nothing on large problems, where x stays in L2 anyway, and to cost 1.4 us per launch on tiny ones)
  *   "row_stages"     shared-memory stages per CTA of the row-direct kernel, 2..4
  *   "row_ctas"       CTAs per SM the row-direct kernel sizes its tiles for, 1..4
  *   "row_unroll"     gathers in flight per thread in the row-direct kernel: 4, 8 or 16

@@ -20,6 +20,7 @@
 #include "spmv_uniform_kernels.cuh"
 #include "spmv_merge_stage_kernels.cuh"
 #include "spmm_kernels.cuh"
+#include "spmm_bstage_kernels.cuh"
 
 using namespace b200sp;
 
@@ -38,6 +39,7 @@ constexpr int kSmemPerSm = 227 * 1024;   // usable shared memory per SM (each CT
 // SpMM
 constexpr int kSpmmThreads = 256;
 constexpr int kSpmmTileNnz = 4096;
+constexpr int kSmallNnz = 1 << 20;   // at or below this many nonzeros SpMV uses the sub-warp-per-row kernel
 constexpr int kLongRow = 1024;   // rows longer than this get a CTA of their own in SpMM (last length bin of the plan)
 
 thread_local std::string g_last_error;
@@ -46,7 +48,7 @@ std::mutex g_mutex;
 
 struct Options {
   int spmv_kernel = -1;
-  int x_l2_window = 1;
+  int x_l2_window = 0;   // measured: no gain on the large workloads (x stays in L2 anyway), +1.4 us per launch on tiny ones
   int row_stages = 2;   // shared-memory stages per CTA of the row-direct kernel (2..4)
   int row_ctas = 3;     // CTAs per SM the row-direct kernel is sized for (1..4)
   int row_unroll = 8;   // gathers in flight per thread (8 or 16)
@@ -59,7 +61,11 @@ struct Options {
   int merge_stages = 3;   // shared-memory stages per CTA of the staged merge kernel (2..4)
   int merge_ctas = 2;     // CTAs per SM of the staged merge kernel
   int merge_threads = 128; // threads per CTA of the one-tile-per-CTA merge kernel (128 or 256)
+  int bstage_threads = 1024; // threads per CTA of that kernel (256, 512 or 1024)
+  int bstage_nnz = 131072;   // nonzeros per CTA it aims for
+  int spmm_bstage = 1;     // 1 = hold the slice of B in shared memory when A has few columns (default), 0 = never
   int spmm_sliced = 1;     // 1 = k-sliced SpMM kernel (default), 0 = one pass over all of k
+  int sub_lanes = 0;       // lanes per row of the sub-warp kernel (0 = from the mean row length)
   int merge_short = 32;    // rows up to this many products are added by one thread (8, 16, 32, 64)
   int merge_carve = 30;    // shared-memory carveout (percent) requested for it, -1 = leave to the driver
 } g_opt;
@@ -272,6 +278,9 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   const bool uniform_ok = nnz > 0 && h.min_len == h.max_len && h.max_len >= 4 && h.max_len <= 128 && (h.max_len & (h.max_len - 1)) == 0;
   const bool row_direct_possible = nnz > 0 && h.max_len <= kRowMaxLen && aligned16(row_ptr);
   int choice = uniform_ok ? 2 : (row_direct_ok ? 1 : 0);
+  // Small problems (launch-latency regime): one sub-warp per row, no scratch, maximum spread over the SMs.
+  if (nnz > 0 && nnz <= kSmallNnz && h.max_len <= 4096) choice = 3;
+  if (g_opt.spmv_kernel == 3) choice = h.max_len <= 65536 ? 3 : 0;
   if (g_opt.spmv_kernel == 0) choice = 0;
   if (g_opt.spmv_kernel == 1) choice = row_direct_possible ? 1 : 0;
   if (g_opt.spmv_kernel == 2) choice = uniform_ok ? 2 : (row_direct_ok ? 1 : 0);
@@ -432,12 +441,42 @@ int run_spmv_merge(b200sp_plan* p, const int32_t* col_idx, const T* vals, const 
   return rc;
 }
 
+template <typename T, int LPR>
+int launch_subwarp(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
+                   cudaStream_t stream, DeviceInfo* dev) {
+  constexpr int THREADS = 128;
+  const b200sp_plan_info_t& I = p->info;
+  const long long groups_per_cta = THREADS / LPR;
+  const long long blocks = (I.m + groups_per_cta - 1) / groups_per_cta;
+  if (blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+  return launch(spmv_subwarp_kernel<T, LPR, THREADS>, dim3((unsigned)blocks), dim3(THREADS), stream, x, (size_t)I.n * sizeof(T), dev,
+                (int)I.m, p->row_ptr, col_idx, vals, x, y, alpha, beta);
+}
+
+template <typename T>
+int run_spmv_subwarp(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
+                     cudaStream_t stream, DeviceInfo* dev) {
+  const b200sp_plan_info_t& I = p->info;
+  const double mean = I.m > 0 ? (double)I.nnz / (double)I.m : 0.0;
+  int lpr = g_opt.sub_lanes;
+  if (lpr <= 0) lpr = mean <= 3 ? 1 : mean <= 6 ? 2 : mean <= 12 ? 4 : mean <= 24 ? 8 : mean <= 64 ? 16 : 32;
+  switch (lpr) {
+    case 1: return launch_subwarp<T, 1>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+    case 2: return launch_subwarp<T, 2>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+    case 4: return launch_subwarp<T, 4>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+    case 8: return launch_subwarp<T, 8>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+    case 16: return launch_subwarp<T, 16>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+    default: return launch_subwarp<T, 32>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  }
+}
+
 template <typename T>
 int run_spmv(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
              cudaStream_t stream, DeviceInfo* dev) {
   const b200sp_plan_info_t& I = p->info;
   if (I.m == 0) return B200SP_OK;
   if (alpha == 0.0f || I.nnz == 0) return run_scale<T>(I.m, y, beta, stream, dev);
+  if (I.spmv_kernel == 3) return run_spmv_subwarp<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (I.spmv_kernel == 2) return run_spmv_uniform<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (I.spmv_kernel == 1) return run_spmv_row_direct<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (I.spmv_tile_items == 4096) return run_spmv_merge<T, 4096>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
@@ -456,12 +495,93 @@ int launch_spmm(const b200sp_plan_info_t& I, const int32_t* row_ptr, int k, cons
                 (size_t)I.n * k * sizeof(T), dev, (int)I.m, k, row_ptr, col_idx, vals, B, Y, alpha, beta);
 }
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn tensor_map_encoder() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    else
+      (void)cudaGetLastError();
+  }
+  return fn;
+}
+
+// B slice in shared memory: used when A has few enough columns and every row of B is re-used often enough.
+template <typename T, int VEC, int LANES, int THREADS = 1024>
+int launch_spmm_bstage(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const T* B, T* Y, float alpha, float beta,
+                       cudaStream_t stream, DeviceInfo* dev, EncodeTiledFn encode) {
+  const b200sp_plan_info_t& I = p->info;
+  constexpr int KS = LANES * VEC, ROW_BYTES = LANES * 16;
+  const int box_rows = I.n < 256 ? (int)I.n : 256;
+  const int boxes = (int)((I.n + box_rows - 1) / box_rows);
+  const size_t smem = (size_t)boxes * box_rows * ROW_BYTES;
+  CUtensorMap map;
+  const cuuint64_t gdim[2] = {(cuuint64_t)k, (cuuint64_t)I.n};
+  const cuuint64_t gstride[1] = {(cuuint64_t)k * sizeof(T)};
+  const cuuint32_t box[2] = {(cuuint32_t)KS, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult cr = encode(&map, sizeof(T) == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<T*>(B), gdim,
+                             gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (cr != CUDA_SUCCESS) return B200SP_ERR_UNSUPPORTED;
+  auto kernel = spmm_bstage_kernel<T, VEC, LANES, THREADS>;
+  static bool configured[64] = {};
+  if (!configured[p->device]) {
+    CU(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerSm - 2048));
+    configured[p->device] = true;
+  }
+  const int slices = (k + KS - 1) / KS;
+  long long chunks = (I.nnz + g_opt.bstage_nnz - 1) / g_opt.bstage_nnz;   // a given number of nonzeros per CTA ...
+  const long long fill = (2LL * dev->sms + slices - 1) / slices;   // ... but at least two CTAs per SM over the grid
+  if (chunks < fill) chunks = fill;
+  if (chunks > I.m) chunks = I.m;
+  if (chunks < 1) chunks = 1;
+  const int rows_per_chunk = (int)((I.m + chunks - 1) / chunks);
+  const int row_chunks = (int)((I.m + rows_per_chunk - 1) / rows_per_chunk);
+  if ((long long)slices * row_chunks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+  int rc = ensure_err_flag(dev);
+  if (rc != B200SP_OK) return rc;
+  return launch_smem(kernel, dim3((unsigned)(slices * row_chunks)), dim3(THREADS), smem, stream, nullptr, 0, dev, map, (int)I.m, (int)I.n,
+                     k, row_chunks, rows_per_chunk, box_rows, p->row_ptr, col_idx, vals, Y, alpha, beta, dev->err_flag);
+}
+
 template <typename T, int VEC>
 int run_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const T* B, T* Y, float alpha, float beta,
              cudaStream_t stream, DeviceInfo* dev) {
   const b200sp_plan_info_t& I = p->info;
   if (I.m == 0) return B200SP_OK;
   if (alpha == 0.0f || I.nnz == 0) return run_scale<T>((long long)I.m * k, Y, beta, stream, dev);
+  if (k % VEC == 0 && g_opt.spmm_bstage && I.nnz >= 4 * I.n && ((size_t)k * sizeof(T)) % 16 == 0) {
+    // widest slice of B (128, 64 or 32 bytes per row) whose n rows fit in one SM's shared memory
+    const size_t budget = (size_t)kSmemPerSm - 4096;
+    const size_t n_pad = (size_t)((I.n + 255) / 256) * 256;
+    EncodeTiledFn encode = tensor_map_encoder();
+    if (encode && n_pad * 32 <= budget) {
+      int rc;
+      if (g_opt.bstage_threads == 256) {
+        if (n_pad * 128 <= budget) rc = launch_spmm_bstage<T, VEC, 8, 256>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+        else if (n_pad * 64 <= budget) rc = launch_spmm_bstage<T, VEC, 4, 256>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+        else rc = launch_spmm_bstage<T, VEC, 2, 256>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+      } else if (g_opt.bstage_threads == 512) {
+        if (n_pad * 128 <= budget) rc = launch_spmm_bstage<T, VEC, 8, 512>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+        else if (n_pad * 64 <= budget) rc = launch_spmm_bstage<T, VEC, 4, 512>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+        else rc = launch_spmm_bstage<T, VEC, 2, 512>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+      } else {
+        if (n_pad * 128 <= budget) rc = launch_spmm_bstage<T, VEC, 8>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+        else if (n_pad * 64 <= budget) rc = launch_spmm_bstage<T, VEC, 4>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+        else rc = launch_spmm_bstage<T, VEC, 2>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+      }
+      if (rc != B200SP_ERR_UNSUPPORTED) return rc;   // unsupported shape for the tensor map: fall through to the sliced kernel
+    }
+  }
   if (k % VEC == 0 && g_opt.spmm_sliced) {
     constexpr int KS = 8 * VEC, GROUPS = kSpmmThreads / 8;
     const int slices = (k + KS - 1) / KS;
@@ -654,6 +774,46 @@ int spmv_csr_noalloc(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, 
   return run_spmv_noalloc<bf16_t>(m, nnz, row_ptr, col_idx, (const bf16_t*)vals, (const bf16_t*)x, (bf16_t*)y, alpha, beta, (cudaStream_t)stream, dev, sc);
 }
 
+int b200sp_spmv_naive(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx, const void* vals,
+                      const void* x, void* y, float alpha, float beta, int dtype, void* stream) {
+  int rc = check_sizes(m, n, nnz);
+  if (rc != B200SP_OK) return rc;
+  if (dtype != B200SP_F32 && dtype != B200SP_BF16) return B200SP_ERR_INVALID_ARG;
+  if (m > 0 && (!row_ptr || !y)) return B200SP_ERR_INVALID_ARG;
+  if (nnz > 0 && (!col_idx || !vals || !x)) return B200SP_ERR_INVALID_ARG;
+  if (m == 0) return B200SP_OK;
+  DeviceInfo* dev = nullptr;
+  rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  const unsigned blocks = (unsigned)((m + 255) / 256);
+  if (dtype == B200SP_F32)
+    return launch(spmv_naive_kernel<float>, dim3(blocks), dim3(256), (cudaStream_t)stream, nullptr, 0, dev, (int)m, row_ptr, col_idx,
+                  (const float*)vals, (const float*)x, (float*)y, alpha, beta);
+  return launch(spmv_naive_kernel<bf16_t>, dim3(blocks), dim3(256), (cudaStream_t)stream, nullptr, 0, dev, (int)m, row_ptr, col_idx,
+                (const bf16_t*)vals, (const bf16_t*)x, (bf16_t*)y, alpha, beta);
+}
+
+int b200sp_spmm_naive(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_ptr, const int32_t* col_idx, const void* vals,
+                      const void* B, void* Y, float alpha, float beta, int dtype, void* stream) {
+  int rc = check_sizes(m, n, nnz);
+  if (rc != B200SP_OK) return rc;
+  if (dtype != B200SP_F32 && dtype != B200SP_BF16) return B200SP_ERR_INVALID_ARG;
+  if (k <= 0 || k >= ((int64_t)1 << 31)) return B200SP_ERR_INVALID_ARG;
+  if (m > 0 && (!row_ptr || !Y)) return B200SP_ERR_INVALID_ARG;
+  if (nnz > 0 && (!col_idx || !vals || !B)) return B200SP_ERR_INVALID_ARG;
+  if (m == 0) return B200SP_OK;
+  DeviceInfo* dev = nullptr;
+  rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  const long long blocks = (m * k + 255) / 256;
+  if (blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+  if (dtype == B200SP_F32)
+    return launch(spmm_naive_kernel<float>, dim3((unsigned)blocks), dim3(256), (cudaStream_t)stream, nullptr, 0, dev, (long long)m, (int)k,
+                  row_ptr, col_idx, (const float*)vals, (const float*)B, (float*)Y, alpha, beta);
+  return launch(spmm_naive_kernel<bf16_t>, dim3((unsigned)blocks), dim3(256), (cudaStream_t)stream, nullptr, 0, dev, (long long)m, (int)k,
+                row_ptr, col_idx, (const bf16_t*)vals, (const bf16_t*)B, (bf16_t*)Y, alpha, beta);
+}
+
 int b200sp_probe_gather(const float* table, int64_t table_elems, int64_t gathers, float* sink, void* stream) {
   if (!table || !sink || table_elems <= 0 || (table_elems & (table_elems - 1)) != 0 || table_elems > ((int64_t)1 << 31) || gathers < 0)
     return B200SP_ERR_INVALID_ARG;
@@ -791,8 +951,12 @@ int64_t b200sp_launch_count(void) { return g_launches.load(); }
 int b200sp_set_option(const char* name, int value) {
   if (!name) return B200SP_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
+  if (!strcmp(name, "bstage_threads")) { if (value != 256 && value != 512 && value != 1024) return B200SP_ERR_INVALID_ARG; g_opt.bstage_threads = value; return B200SP_OK; }
+  if (!strcmp(name, "bstage_nnz")) { if (value < 1024) return B200SP_ERR_INVALID_ARG; g_opt.bstage_nnz = value; return B200SP_OK; }
+  if (!strcmp(name, "spmm_bstage")) { g_opt.spmm_bstage = value ? 1 : 0; return B200SP_OK; }
   if (!strcmp(name, "spmm_sliced")) { g_opt.spmm_sliced = value ? 1 : 0; return B200SP_OK; }
   if (!strcmp(name, "merge_threads")) { if (value != 128 && value != 256) return B200SP_ERR_INVALID_ARG; g_opt.merge_threads = value; return B200SP_OK; }
+  if (!strcmp(name, "sub_lanes")) { if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != 16 && value != 32) return B200SP_ERR_INVALID_ARG; g_opt.sub_lanes = value; return B200SP_OK; }
   if (!strcmp(name, "merge_short")) { if (value != 8 && value != 16 && value != 32 && value != 64) return B200SP_ERR_INVALID_ARG; g_opt.merge_short = value; return B200SP_OK; }
   if (!strcmp(name, "merge_carve")) { if (value < -1 || value > 100) return B200SP_ERR_INVALID_ARG; g_opt.merge_carve = value; return B200SP_OK; }
   if (!strcmp(name, "merge_staged")) { g_opt.merge_staged = value ? 1 : 0; return B200SP_OK; }
@@ -801,7 +965,7 @@ int b200sp_set_option(const char* name, int value) {
   if (!strcmp(name, "merge_ctas")) { if (value < 1 || value > 8) return B200SP_ERR_INVALID_ARG; g_opt.merge_ctas = value; return B200SP_OK; }
   if (!strcmp(name, "uni_unroll")) { if (value != 1 && value != 2 && value != 4) return B200SP_ERR_INVALID_ARG; g_opt.uni_unroll = value; return B200SP_OK; }
   if (!strcmp(name, "uni_ctas")) { if (value < 0 || value > 32) return B200SP_ERR_INVALID_ARG; g_opt.uni_ctas = value; return B200SP_OK; }
-  if (!strcmp(name, "spmv_kernel")) { if (value < -1 || value > 2) return B200SP_ERR_INVALID_ARG; g_opt.spmv_kernel = value; return B200SP_OK; }
+  if (!strcmp(name, "spmv_kernel")) { if (value < -1 || value > 3) return B200SP_ERR_INVALID_ARG; g_opt.spmv_kernel = value; return B200SP_OK; }
   if (!strcmp(name, "x_l2_window")) { g_opt.x_l2_window = value ? 1 : 0; return B200SP_OK; }
   if (!strcmp(name, "row_stages")) { if (value < 2 || value > kRowMaxStages) return B200SP_ERR_INVALID_ARG; g_opt.row_stages = value; return B200SP_OK; }
   if (!strcmp(name, "row_smem_kb")) { if (value < 16 || value > 227) return B200SP_ERR_INVALID_ARG; g_opt.row_smem_kb = value; return B200SP_OK; }

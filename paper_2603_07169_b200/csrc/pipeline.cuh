@@ -5,7 +5,7 @@
 
 namespace b200sp {
 
-constexpr int kSpinLimit = 1 << 22;  // polls of try_wait (each may block for a hardware-defined time slice)
+constexpr int kSpinLimit = 1 << 20;  // polls of try_wait (each may block for a hardware-defined time slice)
 
 __device__ __forceinline__ unsigned smem_addr(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 

@@ -52,6 +52,27 @@ def test_long_rows_and_both_kernels(sliced, dtype):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("n,k", [(2048, 4096), (2048, 40), (1500, 72), (300, 264), (5000, 64), (100, 8)])
+def test_b_slice_in_shared_memory(n, k, dtype):
+    """Few columns: the kernel that holds a slice of B in shared memory (the paper's SpMM shape is n = 2048, K = 4096).
+    Covers all three slice widths, n not a multiple of the copy box, k not a multiple of the slice, long rows, beta != 0."""
+    rng = np.random.default_rng(n + k)
+    m = 3000
+    lens = rng.integers(0, 40, m)
+    lens[7] = min(n, 2500)
+    lens[8] = 0
+    A = gen.random_csr(m, n, lens, seed=n)
+    B = rng.standard_normal(n * k).astype(np.float32)
+    Y0 = rng.standard_normal(m * k).astype(np.float32)
+    Y, Y_ref, S = run_spmm(A, B, k, None, 1.0, 0.0, dtype)
+    assert_within(Y, Y_ref, S, dtype, what="bstage n=%d k=%d" % (n, k))
+    Y, Y_ref, S = run_spmm(A, B, k, Y0, 2.0, -0.5, dtype)
+    y0f = Y0 if dtype == "f32" else gen.bf16_to_f32(gen.to_bf16(Y0))
+    assert_within(Y, Y_ref, S, dtype, 2.0, np.abs(0.5 * y0f.astype(np.float64)).reshape(m, k), what="bstage ab n=%d k=%d" % (n, k))
+    b200sp.b200sp_check()
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
 def test_spmm_column_equals_spmv(dtype):
     from gpu_util import run_spmv
     rng = np.random.default_rng(1)

@@ -47,7 +47,7 @@ def row_len_cases():
     return cases
 
 
-@pytest.fixture(params=[-1, 0, 1, 2], ids=["auto", "merge_tile", "row_direct", "uniform"])
+@pytest.fixture(params=[-1, 0, 1, 2, 3], ids=["auto", "merge_tile", "row_direct", "uniform", "subwarp"])
 def kernel_choice(request):
     """Runs a test under each SpMV kernel selection (1 falls back to 0 inside the plan when rows are too long)."""
     b200sp.b200sp_set_option("spmv_kernel", request.param)
@@ -163,6 +163,40 @@ def test_merge_kernel_variants(staged, items, stages, dtype):
     finally:
         for k, v in (("spmv_kernel", -1), ("merge_staged", 1), ("merge_items", 2048), ("merge_stages", 3)):
             b200sp.b200sp_set_option(k, v)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_naive_baseline_kernels(dtype):
+    """The baselines of the speed-up metric are held to the same bound as the product kernels."""
+    rng = np.random.default_rng(4)
+    A = gen.paper_uniform(1500, 2048, 0.01, seed=3)
+    x = rng.standard_normal(2048).astype(np.float32)
+    vals_s, x_s = store(A.vals, dtype), store(x, dtype)
+    d = [to_dev(a) for a in (A.row_ptr, A.col_idx, vals_s, x_s)]
+    y = empty_out(A.m, dtype)
+    b200sp.b200sp_spmv_naive(A.m, A.n, A.nnz, d[0], d[1], d[2], d[3], y, 1.0, 0.0, dtype)
+    torch.cuda.synchronize()
+    y_ref, S = oracle.spmv_csr(A.m, A.n, A.row_ptr, A.col_idx, vals_s, x_s, None, 1.0, 0.0, dtype)
+    assert_within(to_host(y, dtype), y_ref, S, dtype, what="naive spmv")
+    k = 24
+    B = rng.standard_normal(2048 * k).astype(np.float32)
+    B_s = store(B, dtype)
+    Y = empty_out(A.m * k, dtype)
+    b200sp.b200sp_spmm_naive(A.m, A.n, A.nnz, k, d[0], d[1], d[2], to_dev(B_s), Y, 1.0, 0.0, dtype)
+    torch.cuda.synchronize()
+    Y_ref, S = oracle.spmm_csr(A.m, A.n, k, A.row_ptr, A.col_idx, vals_s, B_s, None, 1.0, 0.0, dtype)
+    assert_within(to_host(Y, dtype).reshape(A.m, k), Y_ref, S, dtype, what="naive spmm")
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("rows", [1024, 4096, 32768])
+def test_paper_sized_spmv(rows, dtype):
+    """The paper's own SpMV CSR sizes (Table 6, task 12): rows x 2048 at density 0.01."""
+    A = gen.paper_uniform(rows, 2048, 0.01, seed=rows)
+    assert A.nnz == int(rows * 2048 * 0.01)
+    x = gen.uniform(2048, -1.0, 1.0, 5, 1)
+    y, y_ref, S = run_spmv(A, x, None, 1.0, 0.0, dtype)
+    assert_within(y, y_ref, S, dtype, what="paper rows=%d" % rows)
 
 
 # ---------------------------------------------------------------- determinism, plan, validation, host API
