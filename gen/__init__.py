@@ -201,6 +201,26 @@ def random_csr(m: int, n: int, row_lens, seed: int, sort_cols: bool = False, int
     return CSR(m, n, rp.astype(np.int32), ci, va, "random")
 
 
+def csr_to_coo(A: CSR):
+    """(row_idx, col_idx, vals) of a CSR matrix, entries in CSR order (sorted by row)."""
+    rows = np.repeat(np.arange(A.m, dtype=np.int32), np.diff(A.row_ptr))
+    return rows, A.col_idx.copy(), A.vals.copy()
+
+
+def csr_to_ell(A: CSR, width: Optional[int] = None, pad_value: float = -1.0):
+    """(width, col_ids, vals), row-major m x width, padding marked with col_id = -1 (value -1 as in the paper's task text)."""
+    L = np.diff(A.row_ptr)
+    W = int(L.max()) if width is None else int(width)
+    assert W >= (int(L.max()) if A.m else 0)
+    col = np.full((A.m, W), -1, np.int32)
+    val = np.full((A.m, W), pad_value, np.float32)
+    j = np.arange(A.nnz, dtype=np.int64) - np.repeat(A.row_ptr[:-1].astype(np.int64), L)
+    r = np.repeat(np.arange(A.m, dtype=np.int64), L)
+    col[r, j] = A.col_idx
+    val[r, j] = A.vals
+    return W, col.ravel(), val.ravel()
+
+
 # ------------------------------------------------------------------ the five measured workloads
 @dataclass
 class Workload:

@@ -48,6 +48,10 @@ def _L():
         lib.oracle_spmv_csr.restype = i32
         lib.oracle_spmm_csr_rows.argtypes = [i64, i64, i64, i64, p, p, p, p, p, f64, f64, i32, p, i64, p, p, i32]
         lib.oracle_spmm_csr_rows.restype = i32
+        lib.oracle_spmm_coo.argtypes = [i64, i64, i64, i64, p, p, p, p, p, f64, f64, i32, p, p]
+        lib.oracle_spmm_coo.restype = i32
+        lib.oracle_spmm_ell.argtypes = [i64, i64, i64, i64, p, p, p, p, f64, f64, i32, p, p]
+        lib.oracle_spmm_ell.restype = i32
         lib.oracle_bf16_to_double.argtypes = [ctypes.c_uint16]
         lib.oracle_bf16_to_double.restype = f64
         lib.oracle_max_threads.restype = i32
@@ -111,6 +115,36 @@ def spmm_csr(m, n, k, row_ptr, col_idx, vals, B, Y0=None, alpha=1.0, beta=0.0, d
                                    float(alpha), float(beta), _DT[dtype], _p(rows), nr, _p(Y), _p(S), nthreads)
     if rc != 0:
         raise RuntimeError("oracle_spmm_csr failed")
+    return Y, S
+
+
+def spmm_coo(m, n, k, row_idx, col_idx, vals, B, Y0=None, alpha=1.0, beta=0.0, dtype="f32"):
+    """COO form (entries in any order; duplicates add): (Y_ref, S_ref) of shape (m, k).  k = 1 with B = x is SpMV."""
+    _check(dtype, vals, B, Y0)
+    row_idx = np.ascontiguousarray(row_idx, np.int32)
+    col_idx = np.ascontiguousarray(col_idx, np.int32)
+    assert B.size == n * k and row_idx.shape == col_idx.shape
+    if beta != 0.0 and Y0 is None:
+        raise ValueError("beta != 0 needs Y0")
+    Y, S = np.empty((m, k), np.float64), np.empty((m, k), np.float64)
+    rc = _L().oracle_spmm_coo(m, n, col_idx.shape[0], k, _p(row_idx), _p(col_idx), _p(vals), _p(B), _p(Y0), float(alpha), float(beta),
+                              _DT[dtype], _p(Y), _p(S))
+    if rc != 0:
+        raise RuntimeError("oracle_spmm_coo failed")
+    return Y, S
+
+
+def spmm_ell(m, n, width, k, col_ids, vals, B, Y0=None, alpha=1.0, beta=0.0, dtype="f32"):
+    """ELL form (row-major m x width, padding where col_ids < 0): (Y_ref, S_ref) of shape (m, k)."""
+    _check(dtype, vals, B, Y0)
+    col_ids = np.ascontiguousarray(col_ids, np.int32)
+    assert col_ids.size == m * width and vals.size == m * width and B.size == n * k
+    if beta != 0.0 and Y0 is None:
+        raise ValueError("beta != 0 needs Y0")
+    Y, S = np.empty((m, k), np.float64), np.empty((m, k), np.float64)
+    rc = _L().oracle_spmm_ell(m, n, width, k, _p(col_ids), _p(vals), _p(B), _p(Y0), float(alpha), float(beta), _DT[dtype], _p(Y), _p(S))
+    if rc != 0:
+        raise RuntimeError("oracle_spmm_ell failed")
     return Y, S
 
 

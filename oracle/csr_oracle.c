@@ -113,3 +113,49 @@ int oracle_spmm_csr(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t*
   return oracle_spmm_csr_rows(m, n, nnz, k, row_ptr, col_idx, vals, B, Y0, alpha, beta, dtype, 0, m, Y_ref,
                               S_ref, nthreads);
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * COO and ELL forms of the same products (paper, Appendix C, Table 6: tasks 8 / 9 "SpMV / SpMM COO" --
+ * values[nnz], row_indices[nnz], col_indices[nnz] -- and tasks 14 / 15 "SpMV / SpMM ELL" -- values and
+ * col_ids of size rows x max_nnz_per_row, padding positions marked with -1).  Readings: COO entries may
+ * come in any order for the oracle (duplicates add; the sum is taken in storage order); ELL is row-major
+ * (row i occupies [i*width, (i+1)*width)) and an entry is padding when its col_id is negative, whatever
+ * its value holds.  k = 1 with B = x gives SpMV.
+ * ---------------------------------------------------------------------------------------------- */
+int oracle_spmm_coo(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_idx, const int32_t* col_idx,
+                    const void* vals, const void* B, const void* Y0, double alpha, double beta, int dtype,
+                    double* Y_ref, double* S_ref) {
+  (void)n;
+  if (dtype != ORACLE_F32 && dtype != ORACLE_BF16) return -1;
+  for (int64_t i = 0; i < m * k; ++i) { Y_ref[i] = 0.0; if (S_ref) S_ref[i] = 0.0; }
+  for (int64_t p = 0; p < nnz; ++p) {
+    const int64_t i = row_idx[p];
+    for (int64_t c = 0; c < k; ++c) {
+      const double t = load(vals, p, dtype) * load(B, (int64_t)col_idx[p] * k + c, dtype);
+      Y_ref[i * k + c] += t;
+      if (S_ref) S_ref[i * k + c] += fabs(t);
+    }
+  }
+  for (int64_t i = 0; i < m * k; ++i) Y_ref[i] = alpha * Y_ref[i] + (beta == 0.0 ? 0.0 : beta * load(Y0, i, dtype));
+  return 0;
+}
+
+int oracle_spmm_ell(int64_t m, int64_t n, int64_t width, int64_t k, const int32_t* col_ids, const void* vals,
+                    const void* B, const void* Y0, double alpha, double beta, int dtype, double* Y_ref, double* S_ref) {
+  (void)n;
+  if (dtype != ORACLE_F32 && dtype != ORACLE_BF16) return -1;
+  for (int64_t i = 0; i < m; ++i)
+    for (int64_t c = 0; c < k; ++c) {
+      double acc = 0.0, S = 0.0;
+      for (int64_t j = 0; j < width; ++j) {
+        const int64_t p = i * width + j;
+        if (col_ids[p] < 0) continue; /* padding */
+        const double t = load(vals, p, dtype) * load(B, (int64_t)col_ids[p] * k + c, dtype);
+        acc += t;
+        S += fabs(t);
+      }
+      Y_ref[i * k + c] = alpha * acc + (beta == 0.0 ? 0.0 : beta * load(Y0, i * k + c, dtype));
+      if (S_ref) S_ref[i * k + c] = S;
+    }
+  return 0;
+}

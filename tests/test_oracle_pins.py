@@ -341,3 +341,51 @@ def test_tolerance_ratio_helper():
     assert r > 1 and i == 1               # an empty row must be exactly zero
     yb = gen.to_bf16(np.array([1.0, 0.0, -2.0], np.float32))
     assert oracle.tolerance_ratio(yb, y_ref, S, "bf16")[0] == 0.0
+
+
+# ---------------------------------------------------------------- COO and ELL forms
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_coo_and_ell_oracles_vs_exact_dense(dtype):
+    rng = np.random.default_rng(31)
+    m, n, k = 9, 6, 4
+    A = gen.random_csr(m, n, [0, 3, 1, 0, 5, 2, 2, 0, 4], 5)
+    B = rng.standard_normal(n * k).astype(np.float32)
+    Y0 = rng.standard_normal(m * k).astype(np.float32)
+    v_s, v_f = stored(A.vals, dtype)
+    B_s, B_f = stored(B, dtype)
+    Y_s, Y_f = stored(Y0, dtype)
+    alpha, beta = 1.5, -0.25
+    D = dense_exact(A, v_f)
+    exact = [[Fraction(alpha) * sum(D[i][j] * frac(B_f[j * k + c]) for j in range(n)) + Fraction(beta) * frac(Y_f[i * k + c])
+              for c in range(k)] for i in range(m)]
+    # COO, entries shuffled (any order is legal for the definition)
+    r, c, _ = gen.csr_to_coo(A)
+    perm = rng.permutation(A.nnz)
+    Yc, Sc = oracle.spmm_coo(m, n, k, r[perm], c[perm], np.ascontiguousarray(v_s[perm]), B_s, Y_s, alpha, beta, dtype)
+    # ELL with extra padding columns; padded values are garbage on purpose
+    W, ci, va = gen.csr_to_ell(A, width=7, pad_value=123.0)
+    va_s, _ = stored(va, dtype)
+    Ye, Se = oracle.spmm_ell(m, n, W, k, ci, va_s, B_s, Y_s, alpha, beta, dtype)
+    Yr, Sr = oracle.spmm_csr(m, n, k, A.row_ptr, A.col_idx, v_s, B_s, Y_s, alpha, beta, dtype)
+    for i in range(m):
+        for cc in range(k):
+            tol = Fraction(float(Sr[i, cc]) * 2.0 ** -48 + abs(float(exact[i][cc])) * 2.0 ** -50)
+            assert abs(Fraction(float(Yc[i, cc])) - exact[i][cc]) <= tol
+            assert abs(Fraction(float(Ye[i, cc])) - exact[i][cc]) <= tol
+    assert np.array_equal(Ye, Yr) and np.array_equal(Se, Sr)          # ELL walks the entries in CSR order: bit-identical
+    assert np.allclose(Sc, Sr, rtol=1e-14, atol=0)
+
+
+def test_coo_ell_hand_worked_fixture():
+    g = _read_golden(os.path.join(GOLDEN, "spmv_hand_worked.txt"))
+    m, n = int(g["m"][0]), int(g["n"][0])
+    rp = np.array(g["row_ptr"], np.int32)
+    A = gen.CSR(m, n, rp, np.array(g["col_idx"], np.int32), np.array(g["vals"], np.float32))
+    x = np.array(g["x"], np.float32)
+    r, c, v = gen.csr_to_coo(A)
+    y, S = oracle.spmm_coo(m, n, 1, r, c, v, x)
+    assert list(y[:, 0]) == g["Ax"] and list(S[:, 0]) == g["S"]
+    W, ci, va = gen.csr_to_ell(A)
+    assert W == 4 and list(ci[:4]) == [0, 3, -1, -1] and list(ci[4:8]) == [-1] * 4
+    y, S = oracle.spmm_ell(m, n, W, 1, ci, va, x)
+    assert list(y[:, 0]) == g["Ax"] and list(S[:, 0]) == g["S"]
