@@ -20,7 +20,7 @@ EXPORTS = (
     "spmv_csr", "spmm_csr", "b200sp_plan_create", "b200sp_plan_destroy", "b200sp_plan_info", "b200sp_spmv",
     "b200sp_spmm", "spmv_csr_host", "spmm_csr_host", "b200sp_validate_csr", "b200sp_cache_clear",
     "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_launch_count", "b200sp_set_option",
-    "b200sp_check", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_spmv_naive", "b200sp_spmm_naive",
+    "b200sp_check", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell",
 )
 
 
@@ -67,6 +67,12 @@ def lib() -> ctypes.CDLL:
         L.b200sp_spmv_naive.restype = i32
         L.b200sp_spmm_naive.argtypes = L.spmm_csr.argtypes
         L.b200sp_spmm_naive.restype = i32
+        L.spmv_coo.argtypes = L.spmv_csr.argtypes
+        L.spmm_coo.argtypes = L.spmm_csr.argtypes
+        L.spmv_ell.argtypes = [i64, i64, i64, p, p, p, p, f32, f32, i32, p]
+        L.spmm_ell.argtypes = [i64, i64, i64, i64, p, p, p, p, f32, f32, i32, p]
+        for name in ("spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell"):
+            getattr(L, name).restype = i32
         L.spmv_csr_noalloc.restype = i32
         L.b200sp_noalloc_max_items.restype = i64
         L.b200sp_probe_gather.argtypes = [p, i64, i64, p, p]
@@ -137,6 +143,22 @@ def spmv_csr_noalloc(m, n, nnz, row_ptr, col_idx, vals, x, y, alpha, beta, dtype
     library (m + nnz <= b200sp_noalloc_max_items()); overlapping calls race on that array."""
     _ck(lib().spmv_csr_noalloc(m, n, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype),
                                _stream(stream)), "spmv_csr_noalloc")
+
+
+def spmv_coo(m, n, nnz, row_idx, col_idx, vals, x, y, alpha, beta, dtype, stream=None):
+    _ck(lib().spmv_coo(m, n, nnz, _ptr(row_idx), _ptr(col_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype), _stream(stream)), "spmv_coo")
+
+
+def spmm_coo(m, n, nnz, k, row_idx, col_idx, vals, B, Y, alpha, beta, dtype, stream=None):
+    _ck(lib().spmm_coo(m, n, nnz, k, _ptr(row_idx), _ptr(col_idx), _ptr(vals), _ptr(B), _ptr(Y), alpha, beta, _dt(dtype), _stream(stream)), "spmm_coo")
+
+
+def spmv_ell(m, n, width, col_ids, vals, x, y, alpha, beta, dtype, stream=None):
+    _ck(lib().spmv_ell(m, n, width, _ptr(col_ids), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype), _stream(stream)), "spmv_ell")
+
+
+def spmm_ell(m, n, width, k, col_ids, vals, B, Y, alpha, beta, dtype, stream=None):
+    _ck(lib().spmm_ell(m, n, width, k, _ptr(col_ids), _ptr(vals), _ptr(B), _ptr(Y), alpha, beta, _dt(dtype), _stream(stream)), "spmm_ell")
 
 
 def b200sp_spmv_naive(m, n, nnz, row_ptr, col_idx, vals, x, y, alpha, beta, dtype, stream=None):

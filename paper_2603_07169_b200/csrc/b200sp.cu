@@ -21,6 +21,7 @@
 #include "spmv_merge_stage_kernels.cuh"
 #include "spmm_kernels.cuh"
 #include "spmm_bstage_kernels.cuh"
+#include "format_kernels.cuh"
 
 using namespace b200sp;
 
@@ -835,6 +836,168 @@ int b200sp_probe_gather(const float* table, int64_t table_elems, int64_t gathers
 
 int64_t b200sp_noalloc_max_items(void) { return (int64_t)kNoAllocMaxTiles * kItems; }
 
+// ---- COO front end: row offsets from sorted row indices, then the CSR path ----
+struct CooEntry { int32_t* row_ptr = nullptr; };
+static std::map<std::tuple<int, const void*, int64_t, int64_t, int64_t>, CooEntry> g_coo_cache;
+
+static int coo_row_ptr(const int32_t** out, int64_t m, int64_t n, int64_t nnz, const int32_t* row_idx, cudaStream_t stream) {
+  DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  int d = 0;
+  CU(cudaGetDevice(&d));
+  const auto key = std::make_tuple(d, (const void*)row_idx, m, n, nnz);
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    auto it = g_coo_cache.find(key);
+    if (it != g_coo_cache.end()) { *out = it->second.row_ptr; return B200SP_OK; }
+  }
+  int32_t* rp = nullptr;
+  int* d_bad = nullptr;
+  int h_bad = 0;
+  CU(cudaMalloc(&rp, (size_t)(m + 1) * sizeof(int32_t)));
+  cudaError_t e = cudaMalloc(&d_bad, sizeof(int));
+  if (e == cudaSuccess) e = cudaMemsetAsync(d_bad, 0, sizeof(int), stream);
+  if (e == cudaSuccess) {
+    const long long work = (m + 1 > nnz ? m + 1 : nnz);
+    long long blocks = (work + 255) / 256;
+    if (blocks > (long long)dev->sms * 16) blocks = (long long)dev->sms * 16;
+    coo_row_ptr_kernel<<<(unsigned)blocks, 256, 0, stream>>>(row_idx, (int)nnz, (int)m, rp, d_bad);
+    g_launches++;
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&h_bad, d_bad, sizeof(int), cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  if (d_bad) cudaFree(d_bad);
+  if (e != cudaSuccess) { cudaFree(rp); return cuda_fail(e, "COO row offsets"); }
+  if (h_bad) { cudaFree(rp); return B200SP_ERR_UNSUPPORTED; }   // entries not sorted by row, or a row index out of range
+  std::lock_guard<std::mutex> lock(g_mutex);
+  auto ins = g_coo_cache.emplace(key, CooEntry{rp});
+  if (!ins.second) { cudaFree(rp); rp = ins.first->second.row_ptr; }
+  *out = rp;
+  return B200SP_OK;
+}
+
+int spmv_coo(int64_t m, int64_t n, int64_t nnz, const int32_t* row_idx, const int32_t* col_idx, const void* vals, const void* x,
+             void* y, float alpha, float beta, int dtype, void* stream) {
+  int rc = check_sizes(m, n, nnz);
+  if (rc != B200SP_OK) return rc;
+  if (nnz > 0 && !row_idx) return B200SP_ERR_INVALID_ARG;
+  if (m == 0) return B200SP_OK;
+  const int32_t* rp = nullptr;
+  rc = coo_row_ptr(&rp, m, n, nnz, row_idx, (cudaStream_t)stream);
+  if (rc != B200SP_OK) return rc;
+  return spmv_csr(m, n, nnz, rp, col_idx, vals, x, y, alpha, beta, dtype, stream);
+}
+
+int spmm_coo(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_idx, const int32_t* col_idx, const void* vals,
+             const void* B, void* Y, float alpha, float beta, int dtype, void* stream) {
+  int rc = check_sizes(m, n, nnz);
+  if (rc != B200SP_OK) return rc;
+  if (nnz > 0 && !row_idx) return B200SP_ERR_INVALID_ARG;
+  if (k <= 0) return B200SP_ERR_INVALID_ARG;
+  if (m == 0) return B200SP_OK;
+  const int32_t* rp = nullptr;
+  rc = coo_row_ptr(&rp, m, n, nnz, row_idx, (cudaStream_t)stream);
+  if (rc != B200SP_OK) return rc;
+  return spmm_csr(m, n, nnz, k, rp, col_idx, vals, B, Y, alpha, beta, dtype, stream);
+}
+
+// ---- ELL front end ----
+static int check_ell(int64_t m, int64_t n, int64_t width, const void* col_ids, const void* vals, const void* in, const void* out, int dtype) {
+  if (m < 0 || n < 0 || width < 0 || n >= ((int64_t)1 << 31) || m >= ((int64_t)1 << 31) - 1) return B200SP_ERR_INVALID_ARG;
+  if (m * width >= ((int64_t)1 << 31)) return B200SP_ERR_INVALID_ARG;
+  if (dtype != B200SP_F32 && dtype != B200SP_BF16) return B200SP_ERR_INVALID_ARG;
+  if (m > 0 && !out) return B200SP_ERR_INVALID_ARG;
+  if (m * width > 0 && (!col_ids || !vals || !in)) return B200SP_ERR_INVALID_ARG;
+  if (!aligned16(col_ids) || !aligned16(vals) || !aligned16(in) || !aligned16(out)) return B200SP_ERR_INVALID_ARG;
+  return B200SP_OK;
+}
+
+}  // extern "C"
+
+template <typename T, int LPR, int VECW>
+static int launch_ell_spmv(int64_t m, int width, const int32_t* col_ids, const T* vals, const T* x, T* y, float alpha, float beta,
+                           cudaStream_t stream, DeviceInfo* dev) {
+  constexpr int THREADS = 128;
+  const long long blocks = (m * LPR + THREADS - 1) / THREADS;
+  if (blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+  return launch(spmv_ell_kernel<T, LPR, VECW, THREADS>, dim3((unsigned)blocks), dim3(THREADS), stream, nullptr, 0, dev, (int)m, width, col_ids,
+                vals, x, y, alpha, beta);
+}
+
+template <typename T>
+static int run_ell_spmv(int64_t m, int width, const int32_t* col_ids, const T* vals, const T* x, T* y, float alpha, float beta,
+                        cudaStream_t stream, DeviceInfo* dev) {
+  if (m == 0) return B200SP_OK;
+  if (alpha == 0.0f || width == 0) return run_scale<T>(m, y, beta, stream, dev);
+  if (width % 4 == 0) {   // 128-bit loads: lanes per row = largest power of two not above width / 4 (at most 32)
+    const int q = width / 4;
+    if (q >= 32) return launch_ell_spmv<T, 32, 4>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);
+    if (q >= 16) return launch_ell_spmv<T, 16, 4>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);
+    if (q >= 8) return launch_ell_spmv<T, 8, 4>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);
+    if (q >= 4) return launch_ell_spmv<T, 4, 4>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);
+    if (q >= 2) return launch_ell_spmv<T, 2, 4>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);
+    return launch_ell_spmv<T, 1, 4>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);
+  }
+  if (width >= 32) return launch_ell_spmv<T, 16, 1>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);
+  if (width >= 12) return launch_ell_spmv<T, 8, 1>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);
+  if (width >= 6) return launch_ell_spmv<T, 4, 1>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);
+  if (width >= 3) return launch_ell_spmv<T, 2, 1>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);
+  return launch_ell_spmv<T, 1, 1>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);
+}
+
+extern "C" {
+
+int spmv_ell(int64_t m, int64_t n, int64_t width, const int32_t* col_ids, const void* vals, const void* x, void* y, float alpha, float beta,
+             int dtype, void* stream) {
+  int rc = check_ell(m, n, width, col_ids, vals, x, y, dtype);
+  if (rc != B200SP_OK) return rc;
+  if (m == 0) return B200SP_OK;
+  DeviceInfo* dev = nullptr;
+  rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  if (dtype == B200SP_F32) return run_ell_spmv<float>(m, (int)width, col_ids, (const float*)vals, (const float*)x, (float*)y, alpha, beta, (cudaStream_t)stream, dev);
+  return run_ell_spmv<bf16_t>(m, (int)width, col_ids, (const bf16_t*)vals, (const bf16_t*)x, (bf16_t*)y, alpha, beta, (cudaStream_t)stream, dev);
+}
+
+}  // extern "C"
+
+template <typename T, int VEC>
+static int run_ell_spmm(int64_t m, int width, int k, const int32_t* col_ids, const T* vals, const T* B, T* Y, float alpha, float beta,
+                        cudaStream_t stream, DeviceInfo* dev) {
+  if (m == 0) return B200SP_OK;
+  if (alpha == 0.0f || width == 0) return run_scale<T>((long long)m * k, Y, beta, stream, dev);
+  if (k % VEC == 0) {
+    constexpr int KS = 8 * VEC, GROUPS = kSpmmThreads / 8;
+    const int slices = (k + KS - 1) / KS;
+    const int row_blocks = (int)((m + GROUPS - 1) / GROUPS);
+    if ((long long)slices * row_blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+    return launch(spmm_ell_slice_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)(slices * row_blocks)), dim3(kSpmmThreads), stream, nullptr, 0, dev,
+                  (int)m, k, width, row_blocks, col_ids, vals, B, Y, alpha, beta);
+  }
+  const long long blocks = ((long long)m * k + 255) / 256;
+  if (blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+  return launch(spmm_ell_entry_kernel<T>, dim3((unsigned)blocks), dim3(256), stream, nullptr, 0, dev, (long long)m, k, width, col_ids, vals, B, Y,
+                alpha, beta);
+}
+
+extern "C" {
+
+int spmm_ell(int64_t m, int64_t n, int64_t width, int64_t k, const int32_t* col_ids, const void* vals, const void* B, void* Y, float alpha,
+             float beta, int dtype, void* stream) {
+  int rc = check_ell(m, n, width, col_ids, vals, B, Y, dtype);
+  if (rc != B200SP_OK) return rc;
+  if (k <= 0 || k >= ((int64_t)1 << 31) || m * k >= ((int64_t)1 << 40)) return B200SP_ERR_INVALID_ARG;
+  if (m == 0) return B200SP_OK;
+  DeviceInfo* dev = nullptr;
+  rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  if (dtype == B200SP_F32)
+    return run_ell_spmm<float, 4>(m, (int)width, (int)k, col_ids, (const float*)vals, (const float*)B, (float*)Y, alpha, beta, (cudaStream_t)stream, dev);
+  return run_ell_spmm<bf16_t, 8>(m, (int)width, (int)k, col_ids, (const bf16_t*)vals, (const bf16_t*)B, (bf16_t*)Y, alpha, beta, (cudaStream_t)stream, dev);
+}
+
 // ---- host-buffer entry points: copy in, plan, run, copy out, synchronise ----
 static int host_call(bool is_mm, int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_ptr, const int32_t* col_idx,
                      const void* vals, const void* in, void* out, float alpha, float beta, int dtype, void* stream_v) {
@@ -914,6 +1077,8 @@ void b200sp_cache_clear(void) {
   std::lock_guard<std::mutex> lock(g_mutex);
   for (auto& kv : g_cache) plan_free(kv.second);
   g_cache.clear();
+  for (auto& kv : g_coo_cache) cudaFree(kv.second.row_ptr);
+  g_coo_cache.clear();
 }
 
 const char* b200sp_status_string(int s) {
