@@ -332,7 +332,42 @@ int launch_row_direct(b200sp_plan* p, const int32_t* col_idx, const T* vals, con
   const int rc_flag = ensure_err_flag(dev);
   if (rc_flag != B200SP_OK) return rc_flag;
   return launch_smem(kernel, dim3(grid), dim3(THREADS), smem, stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz,
-                     p->row_ptr, col_idx, vals, x, y, alpha, beta, R, cap, tiles, stages, rot_lanes, dev->err_flag);
+                     p->row_ptr, col_idx, vals, x, y, alpha, beta, R, cap, tiles, stages, rot_lanes, dev->err_flag, 0);
+}
+
+// The same kernel on an ELL matrix of at most kRowMaxLen slots per row (implicit row offsets, padding skipped).
+template <typename T>
+int launch_row_direct_ell(int64_t m, int width, const int32_t* col_ids, const T* vals, const T* x, T* y, float alpha, float beta,
+                          cudaStream_t stream, DeviceInfo* dev) {
+  constexpr int THREADS = kRowThreads, UNROLL = 8;
+  const int stages = g_opt.row_stages, ctas = g_opt.row_ctas;
+  int sm_budget = g_opt.row_smem_kb * 1024;
+  if (sm_budget > kSmemPerSm) sm_budget = kSmemPerSm;
+  const int stage_budget = (sm_budget / ctas - 1024 - 256) / stages;
+  const int cap_max = (stage_budget - (THREADS + 4) * 4 - 64) / (4 + (int)sizeof(T));
+  int R = (cap_max - 16) / width;
+  if (R > THREADS) R = THREADS;
+  R &= ~3;
+  if (R < 4) return B200SP_ERR_UNSUPPORTED;
+  const int cap = (R * width + 16 + 7) & ~7;
+  const int tiles = (int)((m + R - 1) / R);
+  const size_t smem = (size_t)stages * row_tile_stage_bytes<T>(R, cap);
+  auto kernel = spmv_row_tile_kernel<T, THREADS, UNROLL, false, true>;
+  int d = 0;
+  CU(cudaGetDevice(&d));
+  static int configured[64] = {};
+  int carve = (int)(((size_t)ctas * (smem + 1024 + 128) * 100 + (size_t)kSmemPerSm) / ((size_t)kSmemPerSm + 1024)) + 1;
+  if (carve > 100) carve = 100;
+  if (configured[d] != carve + 1) {
+    CU(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerSm - 1024));
+    CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve));
+    configured[d] = carve + 1;
+  }
+  const int grid = tiles < ctas * dev->sms ? tiles : ctas * dev->sms;
+  const int rc_flag = ensure_err_flag(dev);
+  if (rc_flag != B200SP_OK) return rc_flag;
+  return launch_smem(kernel, dim3(grid), dim3(THREADS), smem, stream, nullptr, 0, dev, (int)m, (int)(m * width), (const int*)nullptr, col_ids,
+                     vals, x, y, alpha, beta, R, cap, tiles, stages, 0, dev->err_flag, width);
 }
 
 template <typename T>
@@ -931,6 +966,8 @@ static int run_ell_spmv(int64_t m, int width, const int32_t* col_ids, const T* v
                         cudaStream_t stream, DeviceInfo* dev) {
   if (m == 0) return B200SP_OK;
   if (alpha == 0.0f || width == 0) return run_scale<T>(m, y, beta, stream, dev);
+  if (width % 4 != 0 && width <= kRowMaxLen)   // odd widths (stencils): the staged row-direct kernel with implicit row offsets
+    return launch_row_direct_ell<T>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);
   if (width % 4 == 0) {   // 128-bit loads: lanes per row = largest power of two not above width / 4 (at most 32)
     const int q = width / 4;
     if (q >= 32) return launch_ell_spmv<T, 32, 4>(m, width, col_ids, vals, x, y, alpha, beta, stream, dev);

@@ -26,7 +26,7 @@ __host__ __device__ __forceinline__ int row_tile_stage_bytes(int R, int cap) {
 constexpr int kRowMaxStages = 4;
 
 // One batch of UNROLL nonzeros of a row: shared-memory reads, then all gathers, then the FMA chain.
-template <typename T, int UNROLL, bool ROT, bool FULL>
+template <typename T, int UNROLL, bool ROT, bool FULL, bool ELL = false>
 __device__ __forceinline__ float row_batch(const int* __restrict__ cp, const T* __restrict__ vp, const T* __restrict__ x,
                                            int j, int len, int rot, float acc) {
   int c[UNROLL];
@@ -40,17 +40,23 @@ __device__ __forceinline__ float row_batch(const int* __restrict__ cp, const T* 
     v[u] = ok ? to_f32(vp[q]) : 0.0f;
   }
 #pragma unroll
-  for (int u = 0; u < UNROLL; ++u) xv[u] = (FULL || c[u] >= 0) ? ld_gather(x + c[u]) : 0.0f;
+  for (int u = 0; u < UNROLL; ++u) xv[u] = ((FULL && !ELL) || c[u] >= 0) ? ld_gather(x + c[u]) : 0.0f;   // ELL: negative col_id = padding
+  if (ELL) {
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) if (c[u] < 0) v[u] = 0.0f;   // a padded value may hold anything
+  }
 #pragma unroll
   for (int u = 0; u < UNROLL; ++u) acc = fmaf(v[u], xv[u], acc);
   return acc;
 }
 
-template <typename T, int THREADS, int UNROLL, bool ROT>
+// ELL = true: the matrix is ELL (row-major m x ell_width, padding col_id < 0): row i starts at i * ell_width,
+// row_ptr is not read (the pointer may be null) and padded entries are skipped.
+template <typename T, int THREADS, int UNROLL, bool ROT, bool ELL = false>
 __global__ void __launch_bounds__(THREADS)
 spmv_row_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
                      const T* __restrict__ vals, const T* __restrict__ x, T* __restrict__ y, float alpha, float beta,
-                     int R, int cap, int num_tiles, int stages, int rot_lanes, int* __restrict__ err) {
+                     int R, int cap, int num_tiles, int stages, int rot_lanes, int* __restrict__ err, int ell_width = 0) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ __align__(8) unsigned long long full_bar[kRowMaxStages];
   const int tid = threadIdx.x;
@@ -71,8 +77,8 @@ spmv_row_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const int*
   auto load_bounds = [&](int i) {
     if (i < my_tiles) {
       const int r0 = ((int)blockIdx.x + i * (int)gridDim.x) * R;
-      nb0 = __ldg(row_ptr + r0);
-      nb1 = __ldg(row_ptr + min(r0 + R, m));
+      if (ELL) { nb0 = r0 * ell_width; nb1 = min(r0 + R, m) * ell_width; }
+      else { nb0 = __ldg(row_ptr + r0); nb1 = __ldg(row_ptr + min(r0 + R, m)); }
     }
   };
   auto issue = [&](int i, int s) {
@@ -85,8 +91,8 @@ spmv_row_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const int*
     const int r1 = min(r0 + R, m);
     const int p0 = nb0, p1 = nb1;
     // row_ptr entries r0 .. r1 (inclusive)
-    const int want = r1 - r0 + 1;
-    const int bulk_rows = min((want + 3) & ~3, rows4 - r0);   // r0 is a multiple of 4
+    const int want = ELL ? 0 : r1 - r0 + 1;
+    const int bulk_rows = ELL ? 0 : min((want + 3) & ~3, rows4 - r0);   // r0 is a multiple of 4
     for (int j = max(bulk_rows, 0); j < want; ++j) rp_s[j] = __ldg(row_ptr + r0 + j);
     // nonzeros [a0, a1) with a0, a1 multiples of 8 around [p0, p1)
     const int a0 = p0 & ~7;
@@ -134,16 +140,16 @@ spmv_row_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const int*
       return;
     }
     if (tid < rows) {
-      const int a0 = rp_s[0] & ~7;
-      const int sft = rp_s[tid] - a0;
-      const int len = rp_s[tid + 1] - a0 - sft;
+      const int a0 = (ELL ? r0 * ell_width : rp_s[0]) & ~7;
+      const int sft = (ELL ? (r0 + tid) * ell_width : rp_s[tid]) - a0;
+      const int len = ELL ? ell_width : rp_s[tid + 1] - a0 - sft;
       const int* cp = col_s + sft;
       const T* vp = val_s + sft;
       const int rot = (ROT && rot0 < len) ? rot0 : 0;
       float acc = 0.0f;
       int j = 0;
-      for (; j + UNROLL <= len; j += UNROLL) acc = row_batch<T, UNROLL, ROT, true>(cp, vp, x, j, len, rot, acc);
-      if (j < len) acc = row_batch<T, UNROLL, ROT, false>(cp, vp, x, j, len, rot, acc);
+      for (; j + UNROLL <= len; j += UNROLL) acc = row_batch<T, UNROLL, ROT, true, ELL>(cp, vp, x, j, len, rot, acc);
+      if (j < len) acc = row_batch<T, UNROLL, ROT, false, ELL>(cp, vp, x, j, len, rot, acc);
       float r = alpha * acc;
       if (beta != 0.0f) r += beta * yold;
       store_elem(y + r0 + tid, r);
