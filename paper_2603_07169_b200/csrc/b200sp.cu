@@ -279,8 +279,9 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   const bool uniform_ok = nnz > 0 && h.min_len == h.max_len && h.max_len >= 4 && h.max_len <= 128 && (h.max_len & (h.max_len - 1)) == 0;
   const bool row_direct_possible = nnz > 0 && h.max_len <= kRowMaxLen && aligned16(row_ptr);
   int choice = uniform_ok ? 2 : (row_direct_ok ? 1 : 0);
-  // Small problems (launch-latency regime): one sub-warp per row, no scratch, maximum spread over the SMs.
-  if (nnz > 0 && nnz <= kSmallNnz && h.max_len <= 4096) choice = 3;
+  // Small problems (launch-latency regime): one sub-warp per row, no scratch, maximum spread over the SMs -- unless the
+  // rows are uniform (the uniform-row kernel is as flat) or the row-direct kernel would still get a tile for every SM.
+  if (nnz > 0 && nnz <= kSmallNnz && h.max_len <= 4096 && !uniform_ok && !(row_direct_ok && m >= (int64_t)kRowThreads * dev->sms)) choice = 3;
   if (g_opt.spmv_kernel == 3) choice = h.max_len <= 65536 ? 3 : 0;
   if (g_opt.spmv_kernel == 0) choice = 0;
   if (g_opt.spmv_kernel == 1) choice = row_direct_possible ? 1 : 0;
