@@ -97,6 +97,9 @@ int spmm_csr(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_pt
  * The plan pass depends on the sparsity pattern's row structure only (row_ptr): it computes the
  * row-length statistics and bins, chooses the kernels, and computes the nnz-balanced split points
  * (a merge-path search over rows + nonzeros for SpMV, over nonzeros for SpMM), all on the device.
+ * When the row statistics select the row-direct SpMV kernel, the first b200sp_spmv / spmv_csr call with a given
+ * col_idx additionally samples how local the columns are (one small kernel and one synchronisation of the stream)
+ * and falls back to the merge-tile kernel for matrices with scattered columns.
  * It allocates a few bytes per tile of device memory (released by b200sp_plan_destroy) and
  * synchronises `stream` once.  A plan may be used from one stream at a time. */
 int b200sp_plan_create(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, void* stream);

@@ -185,6 +185,8 @@ struct b200sp_plan {
   int32_t* spmm_split_row = nullptr;  // spmm tiles + 1
   int32_t* long_rows = nullptr;       // rows longer than kLongRow, ascending
   int num_long = 0;
+  const void* probed_col_idx = nullptr;   // col_idx the column-locality probe last ran on
+  bool cols_local = true;                 // its verdict: adjacent rows share most of their lines of x
 };
 
 namespace {
@@ -507,12 +509,45 @@ int run_spmv_subwarp(b200sp_plan* p, const int32_t* col_idx, const T* vals, cons
   }
 }
 
+// The row-direct kernel gives its shared memory to stages and leaves little L1; that pays only when the gather of x is
+// local (adjacent rows share lines).  The first call with a given col_idx samples that property (one small kernel, one
+// synchronisation); matrices with scattered columns go to the merge-tile kernel instead.
+int probe_col_locality(b200sp_plan* p, const int32_t* col_idx, cudaStream_t stream) {
+  if (p->probed_col_idx == (const void*)col_idx) return B200SP_OK;
+  const b200sp_plan_info_t& I = p->info;
+  unsigned long long* d_out = nullptr;
+  unsigned long long h[2] = {0, 0};
+  CU(cudaMalloc(&d_out, sizeof h));
+  cudaError_t e = cudaMemsetAsync(d_out, 0, sizeof h, stream);
+  const int samples = I.m - 1 < 8192 ? (int)(I.m - 1) : 8192;
+  if (e == cudaSuccess && samples > 0) {
+    plan_col_locality_kernel<<<(samples + 127) / 128, 128, 0, stream>>>(p->row_ptr, col_idx, (int)I.m, samples, d_out);
+    g_launches++;
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(h, d_out, sizeof h, cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  cudaFree(d_out);
+  if (e != cudaSuccess) return cuda_fail(e, "column-locality probe");
+  p->cols_local = h[1] == 0 || 2 * h[0] >= h[1];   // at least half of the sampled entries re-use a line of the row above
+  p->probed_col_idx = col_idx;
+  return B200SP_OK;
+}
+
 template <typename T>
 int run_spmv(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
              cudaStream_t stream, DeviceInfo* dev) {
   const b200sp_plan_info_t& I = p->info;
   if (I.m == 0) return B200SP_OK;
   if (alpha == 0.0f || I.nnz == 0) return run_scale<T>(I.m, y, beta, stream, dev);
+  if (I.spmv_kernel == 1 && g_opt.spmv_kernel != 1) {   // chosen from the row statistics, not forced: confirm with the column probe
+    const int rc = probe_col_locality(p, col_idx, stream);
+    if (rc != B200SP_OK) return rc;
+    if (!p->cols_local) {
+      if (I.spmv_tile_items == 4096) return run_spmv_merge<T, 4096>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+      return run_spmv_merge<T, 2048>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+    }
+  }
   if (I.spmv_kernel == 3) return run_spmv_subwarp<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (I.spmv_kernel == 2) return run_spmv_uniform<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (I.spmv_kernel == 1) return run_spmv_row_direct<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);

@@ -92,6 +92,28 @@ __global__ void __launch_bounds__(256) plan_long_rows_kernel(const int* __restri
   }
 }
 
+// Column-locality probe for matrices with short rows: for `samples` evenly spaced pairs of adjacent rows (r, r + 1),
+// counts the entries of row r + 1 whose 128-byte line of x (32 four-byte entries) is also touched by row r.
+// Banded / stencil / mesh matrices score near 1, matrices with random columns near 0.  out[0] += hits, out[1] += entries.
+__global__ void __launch_bounds__(128) plan_col_locality_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col_idx, int m,
+                                                                int samples, unsigned long long* __restrict__ out) {
+  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= samples || m < 2) return;
+  const long long r = (long long)s * (m - 1) / samples;
+  const int a0 = row_ptr[r], a1 = row_ptr[r + 1], b1 = row_ptr[r + 2];
+  const int la = a1 - a0, lb = b1 - a1;
+  if (la <= 0 || lb <= 0 || la > 64 || lb > 64) return;
+  unsigned hits = 0;
+  for (int j = 0; j < lb; ++j) {
+    const int line = col_idx[a1 + j] >> 5;
+    bool found = false;
+    for (int i = 0; i < la; ++i) found |= (col_idx[a0 + i] >> 5) == line;
+    hits += found;
+  }
+  atomicAdd(&out[0], (unsigned long long)hits);
+  atomicAdd(&out[1], (unsigned long long)lb);
+}
+
 // CSR content check on request.
 __global__ void __launch_bounds__(256) validate_csr_kernel(const int* __restrict__ row_ptr, const int* __restrict__ col_idx, int m, int n,
                                                            int nnz, int* bad) {

@@ -199,6 +199,39 @@ def test_paper_sized_spmv(rows, dtype):
     assert_within(y, y_ref, S, dtype, what="paper rows=%d" % rows)
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_short_rows_with_scattered_columns_take_the_merge_kernel(dtype):
+    """Short irregular rows select the row-direct kernel from row_ptr alone; the column probe must send random columns to the
+    merge-tile kernel (2 launches per call) and keep a banded matrix on the row-direct kernel (1 launch)."""
+    rng = np.random.default_rng(12)
+    m = 1 << 17                                       # > 2^20 nonzeros so that the small-problem kernel is not chosen
+    lens = rng.poisson(12, m).clip(0, 40)
+    A = gen.random_csr(m, m, lens, seed=4)            # uniform random columns
+    x = rng.standard_normal(m).astype(np.float32)
+    vals_s, x_s = store(A.vals, dtype), store(x, dtype)
+    d = [to_dev(a) for a in (A.row_ptr, A.col_idx, vals_s, x_s)]
+    y = empty_out(m, dtype)
+    b200sp.spmv_csr(m, m, A.nnz, d[0], d[1], d[2], d[3], y, 1.0, 0.0, dtype)      # plan + probe
+    n0 = b200sp.b200sp_launch_count()
+    b200sp.spmv_csr(m, m, A.nnz, d[0], d[1], d[2], d[3], y, 1.0, 0.0, dtype)
+    torch.cuda.synchronize()
+    assert b200sp.b200sp_launch_count() - n0 == 2     # merge-tile kernel + carry fix-up
+    y_ref, S = oracle.spmv_csr(m, m, A.row_ptr, A.col_idx, vals_s, x_s, None, 1.0, 0.0, dtype, nthreads=oracle.max_threads())
+    assert_within(to_host(y, dtype), y_ref, S, dtype, what="scattered short rows")
+    b200sp.b200sp_cache_clear()
+    w = gen.workload("c4", scale_down=1)              # 80^3 stencil: banded
+    B = w.A
+    vals_s, x_s = store(B.vals, dtype), store(w.x, dtype)
+    d = [to_dev(a) for a in (B.row_ptr, B.col_idx, vals_s, x_s)]
+    y = empty_out(B.m, dtype)
+    b200sp.spmv_csr(B.m, B.n, B.nnz, d[0], d[1], d[2], d[3], y, 1.0, 0.0, dtype)
+    n0 = b200sp.b200sp_launch_count()
+    b200sp.spmv_csr(B.m, B.n, B.nnz, d[0], d[1], d[2], d[3], y, 1.0, 0.0, dtype)
+    torch.cuda.synchronize()
+    assert b200sp.b200sp_launch_count() - n0 == 1     # row-direct kernel, no fix-up
+    b200sp.b200sp_cache_clear()
+
+
 # ---------------------------------------------------------------- determinism, plan, validation, host API
 @pytest.mark.parametrize("dtype", DTYPES)
 def test_bitwise_run_to_run_determinism(dtype):
