@@ -207,6 +207,16 @@ def csr_to_coo(A: CSR):
     return rows, A.col_idx.copy(), A.vals.copy()
 
 
+def csr_to_csc(A: CSR):
+    """(col_ptr, row_idx, vals) of the same matrix in CSC; entries of a column in ascending row order."""
+    rows = np.repeat(np.arange(A.m, dtype=np.int64), np.diff(A.row_ptr))
+    order = np.argsort(A.col_idx.astype(np.int64) * A.m + rows, kind="stable")
+    cp = np.zeros(A.n + 1, np.int64)
+    np.add.at(cp, A.col_idx.astype(np.int64) + 1, 1)
+    np.cumsum(cp, out=cp)
+    return cp.astype(np.int32), rows[order].astype(np.int32), A.vals[order].copy()
+
+
 def csr_to_ell(A: CSR, width: Optional[int] = None, pad_value: float = -1.0):
     """(width, col_ids, vals), row-major m x width, padding marked with col_id = -1 (value -1 as in the paper's task text)."""
     L = np.diff(A.row_ptr)

@@ -50,6 +50,8 @@ def _L():
         lib.oracle_spmm_csr_rows.restype = i32
         lib.oracle_spmm_coo.argtypes = [i64, i64, i64, i64, p, p, p, p, p, f64, f64, i32, p, p]
         lib.oracle_spmm_coo.restype = i32
+        lib.oracle_spmm_csc.argtypes = [i64, i64, i64, i64, p, p, p, p, p, f64, f64, i32, p, p]
+        lib.oracle_spmm_csc.restype = i32
         lib.oracle_spmm_ell.argtypes = [i64, i64, i64, i64, p, p, p, p, f64, f64, i32, p, p]
         lib.oracle_spmm_ell.restype = i32
         lib.oracle_bf16_to_double.argtypes = [ctypes.c_uint16]
@@ -131,6 +133,22 @@ def spmm_coo(m, n, k, row_idx, col_idx, vals, B, Y0=None, alpha=1.0, beta=0.0, d
                               _DT[dtype], _p(Y), _p(S))
     if rc != 0:
         raise RuntimeError("oracle_spmm_coo failed")
+    return Y, S
+
+
+def spmm_csc(m, n, k, col_ptr, row_idx, vals, B, Y0=None, alpha=1.0, beta=0.0, dtype="f32"):
+    """CSC form (col_ptr of n + 1 entries, row_idx and vals in column-major order): (Y_ref, S_ref) of shape (m, k)."""
+    _check(dtype, vals, B, Y0)
+    col_ptr = np.ascontiguousarray(col_ptr, np.int32)
+    row_idx = np.ascontiguousarray(row_idx, np.int32)
+    assert col_ptr.shape[0] == n + 1 and B.size == n * k
+    if beta != 0.0 and Y0 is None:
+        raise ValueError("beta != 0 needs Y0")
+    Y, S = np.empty((m, k), np.float64), np.empty((m, k), np.float64)
+    rc = _L().oracle_spmm_csc(m, n, row_idx.shape[0], k, _p(col_ptr), _p(row_idx), _p(vals), _p(B), _p(Y0), float(alpha), float(beta),
+                              _DT[dtype], _p(Y), _p(S))
+    if rc != 0:
+        raise RuntimeError("oracle_spmm_csc failed")
     return Y, S
 
 

@@ -159,3 +159,25 @@ int oracle_spmm_ell(int64_t m, int64_t n, int64_t width, int64_t k, const int32_
     }
   return 0;
 }
+
+/* CSC form (paper, Appendix C, Table 6: tasks 10 / 11 "SpMV / SpMM CSC" -- values[nnz], row_indices[nnz],
+ * col_offsets[cols+1] = start of each column in values).  Column j contributes vals[p] * B[j, c] to row
+ * row_idx[p]; the sum over a row is taken in column order, which is the storage order. */
+int oracle_spmm_csc(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* col_ptr, const int32_t* row_idx,
+                    const void* vals, const void* B, const void* Y0, double alpha, double beta, int dtype,
+                    double* Y_ref, double* S_ref) {
+  (void)nnz;
+  if (dtype != ORACLE_F32 && dtype != ORACLE_BF16) return -1;
+  for (int64_t i = 0; i < m * k; ++i) { Y_ref[i] = 0.0; if (S_ref) S_ref[i] = 0.0; }
+  for (int64_t j = 0; j < n; ++j)
+    for (int64_t p = col_ptr[j]; p < col_ptr[j + 1]; ++p) {
+      const int64_t i = row_idx[p];
+      for (int64_t c = 0; c < k; ++c) {
+        const double t = load(vals, p, dtype) * load(B, j * k + c, dtype);
+        Y_ref[i * k + c] += t;
+        if (S_ref) S_ref[i * k + c] += fabs(t);
+      }
+    }
+  for (int64_t i = 0; i < m * k; ++i) Y_ref[i] = alpha * Y_ref[i] + (beta == 0.0 ? 0.0 : beta * load(Y0, i, dtype));
+  return 0;
+}

@@ -389,3 +389,35 @@ def test_coo_ell_hand_worked_fixture():
     assert W == 4 and list(ci[:4]) == [0, 3, -1, -1] and list(ci[4:8]) == [-1] * 4
     y, S = oracle.spmm_ell(m, n, W, 1, ci, va, x)
     assert list(y[:, 0]) == g["Ax"] and list(S[:, 0]) == g["S"]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_csc_oracle_vs_exact_dense(dtype):
+    rng = np.random.default_rng(41)
+    m, n, k = 8, 11, 3                              # rows != cols != k: a swapped index cannot pass
+    A = gen.random_csr(m, n, [2, 0, 5, 1, 3, 0, 4, 2], 6, allow_dup=False)
+    cp, ri, va = gen.csr_to_csc(A)
+    assert cp[-1] == A.nnz and np.all(np.diff(cp) >= 0)
+    B = rng.standard_normal(n * k).astype(np.float32)
+    Y0 = rng.standard_normal(m * k).astype(np.float32)
+    v_s, v_f = stored(va, dtype)
+    B_s, B_f = stored(B, dtype)
+    Y_s, Y_f = stored(Y0, dtype)
+    alpha, beta = -2.0, 0.5
+    Y, S = oracle.spmm_csc(m, n, k, cp, ri, v_s, B_s, Y_s, alpha, beta, dtype)
+    _, a_f = stored(A.vals, dtype)
+    D = dense_exact(A, a_f)
+    for i in range(m):
+        for c in range(k):
+            ex = Fraction(alpha) * sum(D[i][j] * frac(B_f[j * k + c]) for j in range(n)) + Fraction(beta) * frac(Y_f[i * k + c])
+            assert abs(Fraction(float(Y[i, c])) - ex) <= Fraction(float(S[i, c]) * 2.0 ** -48 + abs(float(ex)) * 2.0 ** -50)
+    # sorted unique columns: a row's entries come in the same order in both formats, so CSR and CSC agree bit for bit
+    a_s, _ = stored(A.vals, dtype)
+    Yr, Sr = oracle.spmm_csr(m, n, k, A.row_ptr, A.col_idx, a_s, B_s, Y_s, alpha, beta, dtype)
+    As = gen.random_csr(m, n, [2, 0, 5, 1, 3, 0, 4, 2], 6, allow_dup=False, sort_cols=True)
+    cp2, ri2, va2 = gen.csr_to_csc(As)
+    a2_s, _ = stored(As.vals, dtype)
+    v2_s, _ = stored(va2, dtype)
+    Y1, S1 = oracle.spmm_csr(m, n, k, As.row_ptr, As.col_idx, a2_s, B_s, Y_s, alpha, beta, dtype)
+    Y2, S2 = oracle.spmm_csc(m, n, k, cp2, ri2, v2_s, B_s, Y_s, alpha, beta, dtype)
+    assert np.array_equal(Y1, Y2) and np.array_equal(S1, S2)
