@@ -112,7 +112,7 @@ int b200sp_spmv(b200sp_plan* plan, const int32_t* col_idx, const void* vals, con
 int b200sp_spmm(b200sp_plan* plan, int64_t k, const int32_t* col_idx, const void* vals, const void* B, void* Y,
                 float alpha, float beta, int dtype, void* stream);
 
-/* ---- COO and ELL front ends -------------------------------------------------------------------
+/* ---- COO, CSC and ELL front ends -------------------------------------------------------------------
  * The other sparse formats of the paper's benchmark (Appendix C, Table 6): tasks 8 / 9 "SpMV / SpMM COO"
  * (values, row_indices, col_indices, each nnz long) and tasks 14 / 15 "SpMV / SpMM ELL" (values and
  * col_ids of size rows x max_nnz_per_row, padding positions marked with -1).  Same operations, scalars,
@@ -123,12 +123,23 @@ int b200sp_spmm(b200sp_plan* plan, int64_t k, const int32_t* col_idx, const void
  * order (synchronises the stream once), caches them, and then runs the CSR kernels; unsorted or
  * out-of-range row indices return B200SP_ERR_UNSUPPORTED.  b200sp_cache_clear drops the cached offsets.
  *
+ * CSC (tasks 10 / 11: values, row_indices, col_offsets of cols + 1 entries): the first call for a given
+ * (device, col_ptr, row_idx, m, n, nnz) copies the pattern to the host, builds the row-major order of the
+ * entries there (a stable counting sort by row, so a row's entries are added in ascending column order on every
+ * run), uploads it and caches it together with a scratch array of nnz values; it synchronises the stream.
+ * Every call then permutes vals into that order with one kernel and runs the CSR kernels.  Inconsistent
+ * col_ptr / row_idx return B200SP_ERR_BAD_CSR.  Calls that share a cached pattern must not overlap on the GPU.
+ *
  * ELL: row-major, row i occupies entries [i*width, (i+1)*width) of col_ids and vals; an entry is padding
  * when its col_id is negative (its value is ignored, whatever it holds).  m * width < 2^31.  No plan, no
  * cache, no synchronisation. */
 int spmv_coo(int64_t m, int64_t n, int64_t nnz, const int32_t* row_idx, const int32_t* col_idx, const void* vals,
              const void* x, void* y, float alpha, float beta, int dtype, void* stream);
 int spmm_coo(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_idx, const int32_t* col_idx, const void* vals,
+             const void* B, void* Y, float alpha, float beta, int dtype, void* stream);
+int spmv_csc(int64_t m, int64_t n, int64_t nnz, const int32_t* col_ptr, const int32_t* row_idx, const void* vals,
+             const void* x, void* y, float alpha, float beta, int dtype, void* stream);
+int spmm_csc(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* col_ptr, const int32_t* row_idx, const void* vals,
              const void* B, void* Y, float alpha, float beta, int dtype, void* stream);
 int spmv_ell(int64_t m, int64_t n, int64_t width, const int32_t* col_ids, const void* vals, const void* x, void* y,
              float alpha, float beta, int dtype, void* stream);

@@ -20,7 +20,7 @@ EXPORTS = (
     "spmv_csr", "spmm_csr", "b200sp_plan_create", "b200sp_plan_destroy", "b200sp_plan_info", "b200sp_spmv",
     "b200sp_spmm", "spmv_csr_host", "spmm_csr_host", "b200sp_validate_csr", "b200sp_cache_clear",
     "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_launch_count", "b200sp_set_option",
-    "b200sp_check", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell",
+    "b200sp_check", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell", "spmv_csc", "spmm_csc",
 )
 
 
@@ -71,7 +71,9 @@ def lib() -> ctypes.CDLL:
         L.spmm_coo.argtypes = L.spmm_csr.argtypes
         L.spmv_ell.argtypes = [i64, i64, i64, p, p, p, p, f32, f32, i32, p]
         L.spmm_ell.argtypes = [i64, i64, i64, i64, p, p, p, p, f32, f32, i32, p]
-        for name in ("spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell"):
+        L.spmv_csc.argtypes = L.spmv_csr.argtypes
+        L.spmm_csc.argtypes = L.spmm_csr.argtypes
+        for name in ("spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell", "spmv_csc", "spmm_csc"):
             getattr(L, name).restype = i32
         L.spmv_csr_noalloc.restype = i32
         L.b200sp_noalloc_max_items.restype = i64
@@ -151,6 +153,14 @@ def spmv_coo(m, n, nnz, row_idx, col_idx, vals, x, y, alpha, beta, dtype, stream
 
 def spmm_coo(m, n, nnz, k, row_idx, col_idx, vals, B, Y, alpha, beta, dtype, stream=None):
     _ck(lib().spmm_coo(m, n, nnz, k, _ptr(row_idx), _ptr(col_idx), _ptr(vals), _ptr(B), _ptr(Y), alpha, beta, _dt(dtype), _stream(stream)), "spmm_coo")
+
+
+def spmv_csc(m, n, nnz, col_ptr, row_idx, vals, x, y, alpha, beta, dtype, stream=None):
+    _ck(lib().spmv_csc(m, n, nnz, _ptr(col_ptr), _ptr(row_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype), _stream(stream)), "spmv_csc")
+
+
+def spmm_csc(m, n, nnz, k, col_ptr, row_idx, vals, B, Y, alpha, beta, dtype, stream=None):
+    _ck(lib().spmm_csc(m, n, nnz, k, _ptr(col_ptr), _ptr(row_idx), _ptr(vals), _ptr(B), _ptr(Y), alpha, beta, _dt(dtype), _stream(stream)), "spmm_csc")
 
 
 def spmv_ell(m, n, width, col_ids, vals, x, y, alpha, beta, dtype, stream=None):

@@ -974,6 +974,103 @@ int spmm_coo(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_id
   return spmm_csr(m, n, nnz, k, rp, col_idx, vals, B, Y, alpha, beta, dtype, stream);
 }
 
+// ---- CSC front end: a transpose plan (built on the host, stable in column order), then the CSR path ----
+struct CscEntry { int32_t* row_ptr = nullptr; int32_t* col = nullptr; int32_t* perm = nullptr; void* vals_t = nullptr; };
+static std::map<std::tuple<int, const void*, const void*, int64_t, int64_t, int64_t>, CscEntry> g_csc_cache;
+
+static void csc_free(CscEntry& e) {
+  for (void* q : {(void*)e.row_ptr, (void*)e.col, (void*)e.perm, e.vals_t}) if (q) cudaFree(q);
+  e = CscEntry();
+}
+
+static int csc_plan(CscEntry* out, int64_t m, int64_t n, int64_t nnz, const int32_t* col_ptr, const int32_t* row_idx, cudaStream_t stream) {
+  int d = 0;
+  CU(cudaGetDevice(&d));
+  const auto key = std::make_tuple(d, (const void*)col_ptr, (const void*)row_idx, m, n, nnz);
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    auto it = g_csc_cache.find(key);
+    if (it != g_csc_cache.end()) { *out = it->second; return B200SP_OK; }
+  }
+  // pattern to the host, stable counting sort by row (entries of a row end up in ascending column order), back to the device
+  std::vector<int32_t> h_cp((size_t)n + 1), h_ri((size_t)nnz), h_rp((size_t)m + 1, 0), h_col((size_t)nnz), h_perm((size_t)nnz);
+  CU(cudaMemcpyAsync(h_cp.data(), col_ptr, ((size_t)n + 1) * 4, cudaMemcpyDeviceToHost, stream));
+  if (nnz > 0) CU(cudaMemcpyAsync(h_ri.data(), row_idx, (size_t)nnz * 4, cudaMemcpyDeviceToHost, stream));
+  CU(cudaStreamSynchronize(stream));
+  if (h_cp[0] != 0 || h_cp[(size_t)n] != nnz) return B200SP_ERR_BAD_CSR;
+  for (int64_t p = 0; p < nnz; ++p) {
+    if (h_ri[(size_t)p] < 0 || h_ri[(size_t)p] >= m) return B200SP_ERR_BAD_CSR;
+    h_rp[(size_t)h_ri[(size_t)p] + 1]++;
+  }
+  for (int64_t i = 0; i < m; ++i) h_rp[(size_t)i + 1] += h_rp[(size_t)i];
+  {
+    std::vector<int32_t> next(h_rp.begin(), h_rp.end() - 1);
+    for (int64_t j = 0; j < n; ++j) {
+      if (h_cp[(size_t)j + 1] < h_cp[(size_t)j]) return B200SP_ERR_BAD_CSR;
+      for (int32_t p = h_cp[(size_t)j]; p < h_cp[(size_t)j + 1]; ++p) {
+        const int32_t q = next[(size_t)h_ri[(size_t)p]]++;
+        h_col[(size_t)q] = (int32_t)j;
+        h_perm[(size_t)q] = p;
+      }
+    }
+  }
+  CscEntry e;
+  auto fail = [&](cudaError_t err, const char* what) { csc_free(e); return cuda_fail(err, what); };
+  cudaError_t err;
+  if ((err = cudaMalloc(&e.row_ptr, ((size_t)m + 1) * 4)) != cudaSuccess) return fail(err, "cudaMalloc");
+  const size_t nz = nnz > 0 ? (size_t)nnz : 1;
+  if ((err = cudaMalloc(&e.col, nz * 4)) != cudaSuccess) return fail(err, "cudaMalloc");
+  if ((err = cudaMalloc(&e.perm, nz * 4)) != cudaSuccess) return fail(err, "cudaMalloc");
+  if ((err = cudaMalloc(&e.vals_t, nz * 4)) != cudaSuccess) return fail(err, "cudaMalloc");
+  if ((err = cudaMemcpyAsync(e.row_ptr, h_rp.data(), ((size_t)m + 1) * 4, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return fail(err, "cudaMemcpyAsync");
+  if (nnz > 0) {
+    if ((err = cudaMemcpyAsync(e.col, h_col.data(), (size_t)nnz * 4, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return fail(err, "cudaMemcpyAsync");
+    if ((err = cudaMemcpyAsync(e.perm, h_perm.data(), (size_t)nnz * 4, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return fail(err, "cudaMemcpyAsync");
+  }
+  if ((err = cudaStreamSynchronize(stream)) != cudaSuccess) return fail(err, "cudaStreamSynchronize");
+  std::lock_guard<std::mutex> lock(g_mutex);
+  auto ins = g_csc_cache.emplace(key, e);
+  if (!ins.second) { csc_free(e); e = ins.first->second; }
+  *out = e;
+  return B200SP_OK;
+}
+
+static int csc_call(bool is_mm, int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* col_ptr, const int32_t* row_idx, const void* vals,
+                    const void* in, void* out, float alpha, float beta, int dtype, void* stream_v) {
+  int rc = check_sizes(m, n, nnz);
+  if (rc != B200SP_OK) return rc;
+  if (dtype != B200SP_F32 && dtype != B200SP_BF16) return B200SP_ERR_INVALID_ARG;
+  if (k <= 0) return B200SP_ERR_INVALID_ARG;
+  if (!col_ptr || (nnz > 0 && (!row_idx || !vals))) return B200SP_ERR_INVALID_ARG;
+  if (m == 0) return B200SP_OK;
+  DeviceInfo* dev = nullptr;
+  rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  CscEntry e;
+  rc = csc_plan(&e, m, n, nnz, col_ptr, row_idx, stream);
+  if (rc != B200SP_OK) return rc;
+  if (nnz > 0) {
+    long long blocks = (nnz + 255) / 256;
+    if (blocks > (long long)dev->sms * 16) blocks = (long long)dev->sms * 16;
+    rc = dtype == B200SP_F32
+             ? launch(csc_permute_vals_kernel<float>, dim3((unsigned)blocks), dim3(256), stream, nullptr, 0, dev, (long long)nnz, (const int*)e.perm, (const float*)vals, (float*)e.vals_t)
+             : launch(csc_permute_vals_kernel<bf16_t>, dim3((unsigned)blocks), dim3(256), stream, nullptr, 0, dev, (long long)nnz, (const int*)e.perm, (const bf16_t*)vals, (bf16_t*)e.vals_t);
+    if (rc != B200SP_OK) return rc;
+  }
+  return is_mm ? spmm_csr(m, n, nnz, k, e.row_ptr, e.col, e.vals_t, in, out, alpha, beta, dtype, stream_v)
+               : spmv_csr(m, n, nnz, e.row_ptr, e.col, e.vals_t, in, out, alpha, beta, dtype, stream_v);
+}
+
+int spmv_csc(int64_t m, int64_t n, int64_t nnz, const int32_t* col_ptr, const int32_t* row_idx, const void* vals, const void* x, void* y,
+             float alpha, float beta, int dtype, void* stream) {
+  return csc_call(false, m, n, nnz, 1, col_ptr, row_idx, vals, x, y, alpha, beta, dtype, stream);
+}
+int spmm_csc(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* col_ptr, const int32_t* row_idx, const void* vals, const void* B,
+             void* Y, float alpha, float beta, int dtype, void* stream) {
+  return csc_call(true, m, n, nnz, k, col_ptr, row_idx, vals, B, Y, alpha, beta, dtype, stream);
+}
+
 // ---- ELL front end ----
 static int check_ell(int64_t m, int64_t n, int64_t width, const void* col_ids, const void* vals, const void* in, const void* out, int dtype) {
   if (m < 0 || n < 0 || width < 0 || n >= ((int64_t)1 << 31) || m >= ((int64_t)1 << 31) - 1) return B200SP_ERR_INVALID_ARG;
@@ -1152,6 +1249,8 @@ void b200sp_cache_clear(void) {
   g_cache.clear();
   for (auto& kv : g_coo_cache) cudaFree(kv.second.row_ptr);
   g_coo_cache.clear();
+  for (auto& kv : g_csc_cache) csc_free(kv.second);
+  g_csc_cache.clear();
 }
 
 const char* b200sp_status_string(int s) {

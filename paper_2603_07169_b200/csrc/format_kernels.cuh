@@ -29,6 +29,14 @@ __global__ void __launch_bounds__(256) coo_row_ptr_kernel(const int* __restrict_
   if (b) atomicOr(bad, 1);
 }
 
+// CSC front end, per call: values permuted into the row-major order that the transpose plan computed.
+template <typename T>
+__global__ void __launch_bounds__(256) csc_permute_vals_kernel(long long nnz, const int* __restrict__ perm, const T* __restrict__ vals,
+                                                               T* __restrict__ vals_t) {
+  for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < nnz; q += (long long)gridDim.x * blockDim.x)
+    vals_t[q] = vals[perm[q]];
+}
+
 // ELL SpMV: LPR adjacent lanes own one row and stride over its `width` slots, VECW slots per load.
 template <typename T, int LPR, int VECW, int THREADS>
 __global__ void __launch_bounds__(THREADS)

@@ -50,6 +50,45 @@ def test_coo_spmv_and_spmm(name, dtype):
     b200sp.b200sp_cache_clear()
 
 
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("name", ["power_law", "uniform16", "stencil", "short_ragged"])
+def test_csc_spmv_and_spmm(name, dtype):
+    A = matrices()[name]
+    rng = np.random.default_rng(3)
+    cp, ri, va = gen.csr_to_csc(A)
+    x = rng.standard_normal(A.n).astype(np.float32)
+    y0 = rng.standard_normal(A.m).astype(np.float32)
+    v_s, x_s, y0_s = store(va, dtype), store(x, dtype), store(y0, dtype)
+    d_cp, d_ri, d_v = to_dev(cp), to_dev(ri), to_dev(v_s)
+    for rep in range(2):                                  # second call uses the cached transpose plan
+        y = to_dev(y0_s).clone()
+        b200sp.spmv_csc(A.m, A.n, A.nnz, d_cp, d_ri, d_v, to_dev(x_s), y, 0.5, -1.0, dtype)
+        torch.cuda.synchronize()
+        y_ref, S = oracle.spmm_csc(A.m, A.n, 1, cp, ri, v_s, x_s, y0_s, 0.5, -1.0, dtype)
+        y0f = y0 if dtype == "f32" else gen.bf16_to_f32(y0_s)
+        assert_within(to_host(y, dtype), y_ref[:, 0], S[:, 0], dtype, 1.0, np.abs(y0f.astype(np.float64)), what="csc spmv " + name)
+    k = 16
+    B = rng.standard_normal(A.n * k).astype(np.float32)
+    B_s = store(B, dtype)
+    Y = empty_out(A.m * k, dtype)
+    b200sp.spmm_csc(A.m, A.n, A.nnz, k, d_cp, d_ri, d_v, to_dev(B_s), Y, 1.0, 0.0, dtype)
+    torch.cuda.synchronize()
+    Y_ref, S = oracle.spmm_csc(A.m, A.n, k, cp, ri, v_s, B_s, None, 1.0, 0.0, dtype)
+    assert_within(to_host(Y, dtype).reshape(A.m, k), Y_ref, S, dtype, what="csc spmm " + name)
+    b200sp.b200sp_cache_clear()
+
+
+def test_csc_inconsistent_pattern_is_refused():
+    A = matrices()["short_ragged"]
+    cp, ri, va = gen.csr_to_csc(A)
+    bad = ri.copy(); bad[5] = A.m
+    y = empty_out(A.m, "f32")
+    with pytest.raises(b200sp.B200spError) as e:
+        b200sp.spmv_csc(A.m, A.n, A.nnz, to_dev(cp), to_dev(bad), to_dev(va), to_dev(np.ones(A.n, np.float32)), y, 1.0, 0.0, "f32")
+    assert e.value.status == 6
+    b200sp.b200sp_cache_clear()
+
+
 def test_coo_unsorted_rows_are_refused():
     A = matrices()["short_ragged"]
     r, c, v = gen.csr_to_coo(A)
