@@ -179,6 +179,11 @@ int spmv_csr_host(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, con
                   const void* vals, const void* x, void* y, float alpha, float beta, int dtype, void* stream);
 int spmm_csr_host(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_ptr, const int32_t* col_idx,
                   const void* vals, const void* B, void* Y, float alpha, float beta, int dtype, void* stream);
+/* The matrix (row_ptr, col_idx, vals) is resident on the DEVICE, x and y are HOST buffers: copies x (and y when
+ * beta != 0) in, runs spmv_csr with its cached plan, copies y back and synchronises `stream`.  This is one step of
+ * an iterative method whose matrix stays on the GPU. */
+int spmv_csr_vec_host(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx, const void* vals,
+                      const void* x_host, void* y_host, float alpha, float beta, int dtype, void* stream);
 
 /* ---- checking and housekeeping ---------------------------------------------------------------
  * b200sp_validate_csr checks on the device that row_ptr[0] = 0, row_ptr[m] = nnz, row_ptr is

@@ -20,7 +20,7 @@ EXPORTS = (
     "spmv_csr", "spmm_csr", "b200sp_plan_create", "b200sp_plan_destroy", "b200sp_plan_info", "b200sp_spmv",
     "b200sp_spmm", "spmv_csr_host", "spmm_csr_host", "b200sp_validate_csr", "b200sp_cache_clear",
     "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_launch_count", "b200sp_set_option",
-    "b200sp_check", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell", "spmv_csc", "spmm_csc",
+    "b200sp_check", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell", "spmv_csc", "spmm_csc", "spmv_csr_vec_host",
 )
 
 
@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.spmv_csr.argtypes = [i64, i64, i64, p, p, p, p, p, f32, f32, i32, p]
         L.spmm_csr.argtypes = [i64, i64, i64, i64, p, p, p, p, p, f32, f32, i32, p]
         L.spmv_csr_host.argtypes = L.spmv_csr.argtypes
+        L.spmv_csr_vec_host.argtypes = L.spmv_csr.argtypes
+        L.spmv_csr_vec_host.restype = i32
         L.spmv_csr_noalloc.argtypes = L.spmv_csr.argtypes
         L.b200sp_spmv_naive.argtypes = L.spmv_csr.argtypes
         L.b200sp_spmv_naive.restype = i32
@@ -193,6 +195,12 @@ def b200sp_noalloc_max_items() -> int:
 def spmv_csr_host(m, n, nnz, row_ptr, col_idx, vals, x, y, alpha, beta, dtype, stream=None):
     _ck(lib().spmv_csr_host(m, n, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype),
                             _stream(stream)), "spmv_csr_host")
+
+
+def spmv_csr_vec_host(m, n, nnz, row_ptr, col_idx, vals, x_host, y_host, alpha, beta, dtype, stream=None):
+    """Device-resident matrix, host x and y (one step of an iterative method)."""
+    _ck(lib().spmv_csr_vec_host(m, n, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(x_host), _ptr(y_host), alpha, beta, _dt(dtype),
+                                _stream(stream)), "spmv_csr_vec_host")
 
 
 def spmm_csr_host(m, n, nnz, k, row_ptr, col_idx, vals, B, Y, alpha, beta, dtype, stream=None):

@@ -1210,6 +1210,33 @@ static int host_call(bool is_mm, int64_t m, int64_t n, int64_t nnz, int64_t k, c
   return done(B200SP_OK);
 }
 
+// Matrix resident on the device, vectors on the host (the shape of an iterative solver's step).
+int spmv_csr_vec_host(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx, const void* vals, const void* x_host,
+                      void* y_host, float alpha, float beta, int dtype, void* stream_v) {
+  int rc = check_sizes(m, n, nnz);
+  if (rc != B200SP_OK) return rc;
+  if (dtype != B200SP_F32 && dtype != B200SP_BF16) return B200SP_ERR_INVALID_ARG;
+  if (m > 0 && (!row_ptr || !y_host)) return B200SP_ERR_INVALID_ARG;
+  if (nnz > 0 && (!col_idx || !vals || !x_host)) return B200SP_ERR_INVALID_ARG;
+  if (m == 0) return B200SP_OK;
+  cudaStream_t stream = (cudaStream_t)stream_v;
+  const size_t e = dtype == B200SP_F32 ? 4 : 2;
+  const size_t bx = ((size_t)n * e + 255) & ~(size_t)255, by = (size_t)m * e;
+  char* base = nullptr;
+  CU(cudaMallocAsync((void**)&base, bx + by + 256, stream));
+  auto done = [&](int code) { cudaFreeAsync(base, stream); cudaStreamSynchronize(stream); return code; };
+  cudaError_t err = cudaSuccess;
+  if (n > 0) err = cudaMemcpyAsync(base, x_host, (size_t)n * e, cudaMemcpyHostToDevice, stream);
+  if (err == cudaSuccess && beta != 0.0f) err = cudaMemcpyAsync(base + bx, y_host, by, cudaMemcpyHostToDevice, stream);
+  if (err != cudaSuccess) return done(cuda_fail(err, "cudaMemcpyAsync"));
+  rc = spmv_csr(m, n, nnz, row_ptr, col_idx, vals, base, base + bx, alpha, beta, dtype, stream_v);
+  if (rc != B200SP_OK) return done(rc);
+  err = cudaMemcpyAsync(y_host, base + bx, by, cudaMemcpyDeviceToHost, stream);
+  if (err == cudaSuccess) err = cudaStreamSynchronize(stream);
+  if (err != cudaSuccess) return done(cuda_fail(err, "copy of y"));
+  return done(B200SP_OK);
+}
+
 int spmv_csr_host(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx, const void* vals, const void* x,
                   void* y, float alpha, float beta, int dtype, void* stream) {
   return host_call(false, m, n, nnz, 1, row_ptr, col_idx, vals, x, y, alpha, beta, dtype, stream);

@@ -293,3 +293,8 @@ def test_host_buffer_entry_point(dtype):
     b200sp.spmv_csr_host(A.m, A.n, A.nnz, A.row_ptr, A.col_idx, vals, x, y, w.alpha, w.beta, dtype)
     y_ref, S = oracle.spmv_csr(A.m, A.n, A.row_ptr, A.col_idx, vals, x, y0, w.alpha, w.beta, dtype)
     assert_within(y, y_ref, S, dtype)
+    # matrix on the device, vectors on the host
+    y2 = y0.copy()
+    b200sp.spmv_csr_vec_host(A.m, A.n, A.nnz, to_dev(A.row_ptr), to_dev(A.col_idx), to_dev(vals), x, y2, w.alpha, w.beta, dtype)
+    assert_within(y2, y_ref, S, dtype)
+    b200sp.b200sp_cache_clear()
