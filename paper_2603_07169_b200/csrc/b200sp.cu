@@ -211,7 +211,7 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   p->row_ptr = row_ptr;
   b200sp_plan_info_t& I = p->info;
   I.m = m; I.n = n; I.nnz = nnz;
-  const int items = g_opt.merge_items == 4096 ? 4096 : 2048;
+  const int items = g_opt.merge_items == 4096 ? 4096 : (g_opt.merge_items == 1024 ? 1024 : 2048);
   I.spmv_tile_items = items;
   I.spmv_tiles = (int32_t)((m + nnz + items - 1) / items);
   I.spmm_tile_nnz = kSpmmTileNnz;
@@ -462,6 +462,11 @@ int run_spmv_merge(b200sp_plan* p, const int32_t* col_idx, const T* vals, const 
     const int grid = tiles < ctas * dev->sms ? tiles : ctas * dev->sms;
     rc = launch_smem(kernel, dim3(grid), dim3(kThreads), smem, stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr,
                      col_idx, vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail, tiles, stages, dev->err_flag);
+  } else if (g_opt.merge_threads == 64) {
+    auto kernel = spmv_merge_tile_kernel<T, ITEMS, 64, SHORT>;
+    if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
+    rc = launch(kernel, dim3(tiles), dim3(64), stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx,
+                vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail);
   } else if (g_opt.merge_threads == 128) {
     auto kernel = spmv_merge_tile_kernel<T, ITEMS, 128, SHORT>;
     if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
@@ -545,6 +550,7 @@ int run_spmv(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, 
     if (rc != B200SP_OK) return rc;
     if (!p->cols_local) {
       if (I.spmv_tile_items == 4096) return run_spmv_merge<T, 4096>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+      if (I.spmv_tile_items == 1024) return run_spmv_merge<T, 1024>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
       return run_spmv_merge<T, 2048>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
     }
   }
@@ -552,6 +558,7 @@ int run_spmv(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, 
   if (I.spmv_kernel == 2) return run_spmv_uniform<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (I.spmv_kernel == 1) return run_spmv_row_direct<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (I.spmv_tile_items == 4096) return run_spmv_merge<T, 4096>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  if (I.spmv_tile_items == 1024) return run_spmv_merge<T, 1024>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (g_opt.merge_short == 8) return run_spmv_merge<T, 2048, 8>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (g_opt.merge_short == 16) return run_spmv_merge<T, 2048, 16>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (g_opt.merge_short == 64) return run_spmv_merge<T, 2048, 64>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
@@ -1319,12 +1326,12 @@ int b200sp_set_option(const char* name, int value) {
   if (!strcmp(name, "bstage_nnz")) { if (value < 1024) return B200SP_ERR_INVALID_ARG; g_opt.bstage_nnz = value; return B200SP_OK; }
   if (!strcmp(name, "spmm_bstage")) { g_opt.spmm_bstage = value ? 1 : 0; return B200SP_OK; }
   if (!strcmp(name, "spmm_sliced")) { g_opt.spmm_sliced = value ? 1 : 0; return B200SP_OK; }
-  if (!strcmp(name, "merge_threads")) { if (value != 128 && value != 256) return B200SP_ERR_INVALID_ARG; g_opt.merge_threads = value; return B200SP_OK; }
+  if (!strcmp(name, "merge_threads")) { if (value != 64 && value != 128 && value != 256) return B200SP_ERR_INVALID_ARG; g_opt.merge_threads = value; return B200SP_OK; }
   if (!strcmp(name, "sub_lanes")) { if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != 16 && value != 32) return B200SP_ERR_INVALID_ARG; g_opt.sub_lanes = value; return B200SP_OK; }
   if (!strcmp(name, "merge_short")) { if (value != 8 && value != 16 && value != 32 && value != 64) return B200SP_ERR_INVALID_ARG; g_opt.merge_short = value; return B200SP_OK; }
   if (!strcmp(name, "merge_carve")) { if (value < -1 || value > 100) return B200SP_ERR_INVALID_ARG; g_opt.merge_carve = value; return B200SP_OK; }
   if (!strcmp(name, "merge_staged")) { g_opt.merge_staged = value ? 1 : 0; return B200SP_OK; }
-  if (!strcmp(name, "merge_items")) { if (value != 2048 && value != 4096) return B200SP_ERR_INVALID_ARG; g_opt.merge_items = value; return B200SP_OK; }
+  if (!strcmp(name, "merge_items")) { if (value != 1024 && value != 2048 && value != 4096) return B200SP_ERR_INVALID_ARG; g_opt.merge_items = value; return B200SP_OK; }
   if (!strcmp(name, "merge_stages")) { if (value < 2 || value > kMergeMaxStages) return B200SP_ERR_INVALID_ARG; g_opt.merge_stages = value; return B200SP_OK; }
   if (!strcmp(name, "merge_ctas")) { if (value < 1 || value > 8) return B200SP_ERR_INVALID_ARG; g_opt.merge_ctas = value; return B200SP_OK; }
   if (!strcmp(name, "uni_unroll")) { if (value != 1 && value != 2 && value != 4) return B200SP_ERR_INVALID_ARG; g_opt.uni_unroll = value; return B200SP_OK; }
