@@ -1,0 +1,140 @@
+// Host side of libb200sp.so: the plan pass (row statistics, bins, splits, long-row list) and the plan cache.
+// One of the pieces of the single translation unit b200sp.cu; include/b200sp.h states the contract of every entry point.
+#pragma once
+#include "host_runtime.cuh"
+#include "plan_kernels.cuh"
+
+namespace {
+
+std::map<std::tuple<int, const void*, int64_t, int64_t, int64_t>, b200sp_plan*> g_cache;
+
+int plan_free(b200sp_plan* p) {
+  if (!p) return B200SP_OK;
+  int rc = B200SP_OK;
+  for (void* q : {(void*)p->split_row, (void*)p->carry, (void*)p->tail, (void*)p->spmm_split_row, (void*)p->long_rows})
+    if (q) { cudaError_t e = cudaFree(q); if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree"); }
+  delete p;
+  return rc;
+}
+
+int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, cudaStream_t stream) {
+  DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  b200sp_plan* p = new b200sp_plan();
+  CU(cudaGetDevice(&p->device));
+  p->row_ptr = row_ptr;
+  b200sp_plan_info_t& I = p->info;
+  I.m = m; I.n = n; I.nnz = nnz;
+  const int items = g_opt.merge_items == 4096 ? 4096 : (g_opt.merge_items == 1024 ? 1024 : 2048);
+  I.spmv_tile_items = items;
+  I.spmv_tiles = (int32_t)((m + nnz + items - 1) / items);
+  I.spmm_tile_nnz = kSpmmTileNnz;
+  I.spmm_tiles = (int32_t)((nnz + kSpmmTileNnz - 1) / kSpmmTileNnz);
+  I.spmv_kernel = g_opt.spmv_kernel >= 0 ? g_opt.spmv_kernel : 0;
+  if (m == 0) { *out = p; return B200SP_OK; }
+
+  PlanStats* d_stats = nullptr;
+  PlanStats h = {};
+  h.min_len = 0x7FFFFFFF;
+  auto fail = [&](int code) { if (d_stats) cudaFree(d_stats); plan_free(p); return code; };
+#define CUP(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail(cuda_fail(e_, #call)); } while (0)
+  CUP(cudaMalloc(&d_stats, sizeof(PlanStats)));
+  CUP(cudaMemcpyAsync(d_stats, &h, sizeof h, cudaMemcpyHostToDevice, stream));
+  {
+    const int blocks = (int)((m + 256 * 8 - 1) / (256 * 8));
+    const int grid = blocks < dev->sms * 8 ? (blocks > 0 ? blocks : 1) : dev->sms * 8;
+    plan_stats_kernel<<<grid, 256, 0, stream>>>(row_ptr, (int)m, d_stats);
+    g_launches++;
+  }
+  const size_t nt = (size_t)I.spmv_tiles, ns = (size_t)I.spmm_tiles;
+  CUP(cudaMalloc(&p->split_row, (nt + 1) * sizeof(int32_t)));
+  CUP(cudaMalloc(&p->carry, (nt + 1) * sizeof(float)));
+  CUP(cudaMalloc(&p->tail, (nt + 1) * sizeof(float)));
+  CUP(cudaMalloc(&p->spmm_split_row, (ns + 1) * sizeof(int32_t)));
+  I.scratch_bytes = (int64_t)((nt + 1) * 12 + (ns + 1) * 4);
+  plan_merge_split_kernel<<<(unsigned)((nt + 1 + 255) / 256), 256, 0, stream>>>(row_ptr, (int)m, (int)nnz, items, (int)nt, p->split_row);
+  plan_nnz_split_kernel<<<(unsigned)((ns + 1 + 255) / 256), 256, 0, stream>>>(row_ptr, (int)m, (int)nnz, kSpmmTileNnz, (int)ns, p->spmm_split_row);
+  g_launches += 2;
+  CUP(cudaGetLastError());
+  CUP(cudaMemcpyAsync(&h, d_stats, sizeof h, cudaMemcpyDeviceToHost, stream));
+  CUP(cudaStreamSynchronize(stream));
+  CUP(cudaFree(d_stats));
+  d_stats = nullptr;
+  if (!h.bad && h.bin_rows[4] > 0) {   // list of the rows in the last length bin (> kLongRow), sorted on the host
+    const int cap = (int)h.bin_rows[4];
+    int* d_count = nullptr;
+    CUP(cudaMalloc(&p->long_rows, (size_t)cap * sizeof(int32_t)));
+    CUP(cudaMalloc(&d_count, sizeof(int)));
+    cudaError_t e = cudaMemsetAsync(d_count, 0, sizeof(int), stream);
+    if (e == cudaSuccess) {
+      const int blocks = (int)((m + 255) / 256);
+      plan_long_rows_kernel<<<blocks < dev->sms * 8 ? blocks : dev->sms * 8, 256, 0, stream>>>(row_ptr, (int)m, kLongRow, cap, p->long_rows, d_count);
+      g_launches++;
+      e = cudaGetLastError();
+    }
+    std::vector<int32_t> tmp((size_t)cap);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(tmp.data(), p->long_rows, (size_t)cap * sizeof(int32_t), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e == cudaSuccess) { std::sort(tmp.begin(), tmp.end()); e = cudaMemcpyAsync(p->long_rows, tmp.data(), (size_t)cap * sizeof(int32_t), cudaMemcpyHostToDevice, stream); }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    cudaFree(d_count);
+    if (e != cudaSuccess) return fail(cuda_fail(e, "plan long-row list"));
+    p->num_long = cap;
+    I.scratch_bytes += (int64_t)cap * 4;
+  }
+#undef CUP
+  if (h.bad) { plan_free(p); return B200SP_ERR_BAD_CSR; }
+  I.min_row_len = h.min_len; I.max_row_len = h.max_len;
+  for (int j = 0; j < B200SP_NUM_BINS; ++j) { I.bin_rows[j] = (int64_t)h.bin_rows[j]; I.bin_nnz[j] = (int64_t)h.bin_nnz[j]; }
+  // Kernel choice from the row statistics: when every row is short and the mean is not far below the
+  // maximum, a thread per row wastes little and rows never need splitting -> row-direct kernel.
+  // Anything with long or very uneven rows goes to the merge-tile kernel.
+  const bool row_direct_ok = nnz > 0 && h.max_len <= kRowMaxLen && aligned16(row_ptr) &&
+                             (h.max_len <= 8 || nnz * 4 >= (int64_t)h.max_len * m);
+  // Rows all of one length 4, 8, ..., 128: sub-warp-per-row kernel with 128-bit loads and no shared memory.
+  const bool uniform_ok = nnz > 0 && h.min_len == h.max_len && h.max_len >= 4 && h.max_len <= 128 && (h.max_len & (h.max_len - 1)) == 0;
+  const bool row_direct_possible = nnz > 0 && h.max_len <= kRowMaxLen && aligned16(row_ptr);
+  int choice = uniform_ok ? 2 : (row_direct_ok ? 1 : 0);
+  // Small problems (launch-latency regime): one sub-warp per row, no scratch, maximum spread over the SMs -- unless the
+  // rows are uniform (the uniform-row kernel is as flat) or the row-direct kernel would still get a tile for every SM.
+  if (nnz > 0 && nnz <= kSmallNnz && h.max_len <= 4096 && !uniform_ok && !(row_direct_ok && m >= (int64_t)kRowThreads * dev->sms)) choice = 3;
+  if (g_opt.spmv_kernel == 3) choice = h.max_len <= 65536 ? 3 : 0;
+  if (g_opt.spmv_kernel == 0) choice = 0;
+  if (g_opt.spmv_kernel == 1) choice = row_direct_possible ? 1 : 0;
+  if (g_opt.spmv_kernel == 2) choice = uniform_ok ? 2 : (row_direct_ok ? 1 : 0);
+  I.spmv_kernel = choice;
+  *out = p;
+  return B200SP_OK;
+}
+
+int check_common(const b200sp_plan* p, const void* col_idx, const void* vals, const void* dense_in, const void* dense_out, int dtype) {
+  if (!p) return B200SP_ERR_INVALID_ARG;
+  if (dtype != B200SP_F32 && dtype != B200SP_BF16) return B200SP_ERR_INVALID_ARG;
+  const b200sp_plan_info_t& I = p->info;
+  if (I.nnz > 0 && (!col_idx || !vals || !dense_in)) return B200SP_ERR_INVALID_ARG;
+  if (I.m > 0 && !dense_out) return B200SP_ERR_INVALID_ARG;
+  if (!aligned16(col_idx) || !aligned16(vals) || !aligned16(dense_in) || !aligned16(dense_out)) return B200SP_ERR_INVALID_ARG;
+  return B200SP_OK;
+}
+
+int get_cached_plan(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, cudaStream_t stream) {
+  int dev = 0;
+  CU(cudaGetDevice(&dev));
+  const auto key = std::make_tuple(dev, (const void*)row_ptr, m, n, nnz);
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    auto it = g_cache.find(key);
+    if (it != g_cache.end()) { *out = it->second; return B200SP_OK; }
+  }
+  b200sp_plan* p = nullptr;
+  int rc = b200sp_plan_create(&p, m, n, nnz, row_ptr, stream);
+  if (rc != B200SP_OK) return rc;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  auto ins = g_cache.emplace(key, p);
+  if (!ins.second) { plan_free(p); p = ins.first->second; }
+  *out = p;
+  return B200SP_OK;
+}
+
+}  // namespace

@@ -1,0 +1,182 @@
+// Host side of libb200sp.so: constants, tuning switches, device queries, the launch helper and argument checks.
+// One of the pieces of the single translation unit b200sp.cu; include/b200sp.h states the contract of every entry point.
+#pragma once
+#include "../../include/b200sp.h"
+
+#include <algorithm>
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace b200sp;
+
+namespace {
+
+constexpr int kVersion = 100;  // 0.1.0
+
+// SpMV merge-tile configuration
+constexpr int kItems = 4096;
+constexpr int kThreads = 256;
+constexpr int kShortMax = 32;
+// SpMV row-direct kernel: eligibility and shared-memory budget (two CTAs per SM)
+constexpr int kRowThreads = 256;
+constexpr int kRowMaxLen = 64;
+constexpr int kSmemPerSm = 227 * 1024;   // usable shared memory per SM (each CTA also reserves 1 KB)
+// SpMM
+constexpr int kSpmmThreads = 256;
+constexpr int kSpmmTileNnz = 4096;
+constexpr int kSmallNnz = 1 << 20;   // at or below this many nonzeros SpMV uses the sub-warp-per-row kernel
+constexpr int kLongRow = 1024;   // rows longer than this get a CTA of their own in SpMM (last length bin of the plan)
+
+thread_local std::string g_last_error;
+std::atomic<int64_t> g_launches{0};
+std::mutex g_mutex;
+
+struct Options {
+  int spmv_kernel = -1;
+  int x_l2_window = 0;   // measured: no gain on the large workloads (x stays in L2 anyway), +1.4 us per launch on tiny ones
+  int row_stages = 2;   // shared-memory stages per CTA of the row-direct kernel (2..4)
+  int row_ctas = 3;     // CTAs per SM the row-direct kernel is sized for (1..4)
+  int row_unroll = 8;   // gathers in flight per thread (8 or 16)
+  int row_smem_kb = 220;  // shared memory per SM the row-direct kernel may use for its stages (the rest stays L1)
+  int row_threads = 256;  // threads per CTA of the row-direct kernel (128 or 256)
+  int uni_unroll = 2;     // groups of four nonzeros in flight per thread of the uniform-row kernel (1, 2 or 4)
+  int uni_ctas = 0;       // CTAs per SM for the uniform-row kernel (0 = as many as fit)
+  int merge_staged = 0;   // 1 = persistent staged merge kernel, 0 = one-tile-per-CTA merge kernel
+  int merge_items = 2048; // merge items per tile (2048 or 4096)
+  int merge_stages = 3;   // shared-memory stages per CTA of the staged merge kernel (2..4)
+  int merge_ctas = 2;     // CTAs per SM of the staged merge kernel
+  int merge_threads = 128; // threads per CTA of the one-tile-per-CTA merge kernel (128 or 256)
+  int bstage_threads = 1024; // threads per CTA of that kernel (256, 512 or 1024)
+  int bstage_nnz = 131072;   // nonzeros per CTA it aims for
+  int spmm_bstage = 1;     // 1 = hold the slice of B in shared memory when A has few columns (default), 0 = never
+  int spmm_sliced = 1;     // 1 = k-sliced SpMM kernel (default), 0 = one pass over all of k
+  int sub_lanes = 0;       // lanes per row of the sub-warp kernel (0 = from the mean row length)
+  int merge_short = 32;    // rows up to this many products are added by one thread (8, 16, 32, 64)
+  int merge_carve = 30;    // shared-memory carveout (percent) requested for it, -1 = leave to the driver
+} g_opt;
+
+struct DeviceInfo {
+  bool known = false;
+  int cc_major = 0, sms = 0, persist_max = 0, window_max = 0, l2_bytes = 0;
+  size_t persist_set = 0;
+  int* err_flag = nullptr;  // device int: set by a kernel whose bounded wait ran out
+};
+DeviceInfo g_dev[64];
+
+int cuda_fail(cudaError_t e, const char* what) {
+  char buf[512];
+  snprintf(buf, sizeof buf, "%s: %s", what, cudaGetErrorString(e));
+  g_last_error = buf;
+  (void)cudaGetLastError();
+  return B200SP_ERR_CUDA;
+}
+#define CU(call)                                                   \
+  do {                                                             \
+    cudaError_t e_ = (call);                                       \
+    if (e_ != cudaSuccess) return cuda_fail(e_, #call);            \
+  } while (0)
+
+int device_info(DeviceInfo** out) {
+  int dev = 0;
+  CU(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return B200SP_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceInfo& d = g_dev[dev];
+  if (!d.known) {
+    CU(cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+    CU(cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev));
+    CU(cudaDeviceGetAttribute(&d.persist_max, cudaDevAttrMaxPersistingL2CacheSize, dev));
+    CU(cudaDeviceGetAttribute(&d.window_max, cudaDevAttrMaxAccessPolicyWindowSize, dev));
+    CU(cudaDeviceGetAttribute(&d.l2_bytes, cudaDevAttrL2CacheSize, dev));
+    d.known = true;
+  }
+  *out = &d;
+  return d.cc_major == 10 ? B200SP_OK : B200SP_ERR_ARCH;
+}
+
+// The flag that kernels with bounded waits raise; allocated on first use (those kernels only).
+int ensure_err_flag(DeviceInfo* d) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!d->err_flag) {
+    CU(cudaMalloc(&d->err_flag, sizeof(int)));
+    CU(cudaMemset(d->err_flag, 0, sizeof(int)));
+  }
+  return B200SP_OK;
+}
+
+// Launch with an optional L2 access-policy window (persisting hits) over the gathered operand.
+template <typename... KArgs, typename... Args>
+int launch_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, const void* win_ptr,
+                size_t win_bytes, DeviceInfo* dev, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  cfg.attrs = attr;
+  cfg.numAttrs = 0;
+  if (win_ptr && win_bytes && g_opt.x_l2_window && dev->persist_max > 0 && dev->window_max > 0) {
+    size_t want = win_bytes < (size_t)dev->persist_max ? win_bytes : (size_t)dev->persist_max;
+    {
+      std::lock_guard<std::mutex> lock(g_mutex);
+      if (want > dev->persist_set) {
+        if (cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want) == cudaSuccess) dev->persist_set = want;
+        else (void)cudaGetLastError();
+      }
+    }
+    if (dev->persist_set > 0) {
+      const size_t wb = win_bytes < (size_t)dev->window_max ? win_bytes : (size_t)dev->window_max;
+      attr[0].id = cudaLaunchAttributeAccessPolicyWindow;
+      attr[0].val.accessPolicyWindow.base_ptr = const_cast<void*>(win_ptr);
+      attr[0].val.accessPolicyWindow.num_bytes = wb;
+      attr[0].val.accessPolicyWindow.hitRatio = wb <= dev->persist_set ? 1.0f : (float)((double)dev->persist_set / (double)wb);
+      attr[0].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+      attr[0].val.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
+      cfg.numAttrs = 1;
+    }
+  }
+  CU(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return B200SP_OK;
+}
+
+template <typename... KArgs, typename... Args>
+int launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream, const void* win_ptr, size_t win_bytes,
+           DeviceInfo* dev, Args... args) {
+  return launch_smem(kernel, grid, block, 0, stream, win_ptr, win_bytes, dev, args...);
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+int check_sizes(int64_t m, int64_t n, int64_t nnz) {
+  const int64_t lim = (int64_t)1 << 31;
+  if (m < 0 || n < 0 || nnz < 0 || m >= lim - 1 || n >= lim || nnz >= lim) return B200SP_ERR_INVALID_ARG;
+  if (nnz > 0 && (m == 0 || n == 0)) return B200SP_ERR_INVALID_ARG;
+  return B200SP_OK;
+}
+
+}  // namespace
+
+struct b200sp_plan {
+  int device = 0;
+  const int32_t* row_ptr = nullptr;
+  b200sp_plan_info_t info = {};
+  int32_t* split_row = nullptr;       // spmv tiles + 1
+  float* carry = nullptr;             // spmv tiles
+  float* tail = nullptr;              // spmv tiles
+  int32_t* spmm_split_row = nullptr;  // spmm tiles + 1
+  int32_t* long_rows = nullptr;       // rows longer than kLongRow, ascending
+  int num_long = 0;
+  const void* probed_col_idx = nullptr;   // col_idx the column-locality probe last ran on
+  bool cols_local = true;                 // its verdict: adjacent rows share most of their lines of x
+};

@@ -1,0 +1,130 @@
+// Host side of libb200sp.so: SpMM kernel selection and launches.
+// One of the pieces of the single translation unit b200sp.cu; include/b200sp.h states the contract of every entry point.
+#pragma once
+#include "host_spmv.cuh"
+#include "spmm_kernels.cuh"
+#include "spmm_bstage_kernels.cuh"
+
+namespace {
+
+template <typename T, int VEC, int LANES, int NCH>
+int launch_spmm(const b200sp_plan_info_t& I, const int32_t* row_ptr, int k, const int32_t* col_idx, const T* vals, const T* B, T* Y,
+                float alpha, float beta, cudaStream_t stream, DeviceInfo* dev) {
+  constexpr int GROUPS = kSpmmThreads / LANES;
+  const unsigned grid = (unsigned)((I.m + GROUPS - 1) / GROUPS);
+  return launch(spmm_row_group_kernel<T, VEC, LANES, NCH, kSpmmThreads>, dim3(grid), dim3(kSpmmThreads), stream, B,
+                (size_t)I.n * k * sizeof(T), dev, (int)I.m, k, row_ptr, col_idx, vals, B, Y, alpha, beta);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn tensor_map_encoder() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!tried) {
+    tried = true;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    else
+      (void)cudaGetLastError();
+  }
+  return fn;
+}
+
+// B slice in shared memory: used when A has few enough columns and every row of B is re-used often enough.
+template <typename T, int VEC, int LANES, int THREADS = 1024>
+int launch_spmm_bstage(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const T* B, T* Y, float alpha, float beta,
+                       cudaStream_t stream, DeviceInfo* dev, EncodeTiledFn encode) {
+  const b200sp_plan_info_t& I = p->info;
+  constexpr int KS = LANES * VEC, ROW_BYTES = LANES * 16;
+  const int box_rows = I.n < 256 ? (int)I.n : 256;
+  const int boxes = (int)((I.n + box_rows - 1) / box_rows);
+  const size_t smem = (size_t)boxes * box_rows * ROW_BYTES;
+  CUtensorMap map;
+  const cuuint64_t gdim[2] = {(cuuint64_t)k, (cuuint64_t)I.n};
+  const cuuint64_t gstride[1] = {(cuuint64_t)k * sizeof(T)};
+  const cuuint32_t box[2] = {(cuuint32_t)KS, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult cr = encode(&map, sizeof(T) == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<T*>(B), gdim,
+                             gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (cr != CUDA_SUCCESS) return B200SP_ERR_UNSUPPORTED;
+  auto kernel = spmm_bstage_kernel<T, VEC, LANES, THREADS>;
+  static bool configured[64] = {};
+  if (!configured[p->device]) {
+    CU(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerSm - 2048));
+    configured[p->device] = true;
+  }
+  const int slices = (k + KS - 1) / KS;
+  long long chunks = (I.nnz + g_opt.bstage_nnz - 1) / g_opt.bstage_nnz;   // a given number of nonzeros per CTA ...
+  const long long fill = (2LL * dev->sms + slices - 1) / slices;   // ... but at least two CTAs per SM over the grid
+  if (chunks < fill) chunks = fill;
+  if (chunks > I.m) chunks = I.m;
+  if (chunks < 1) chunks = 1;
+  const int rows_per_chunk = (int)((I.m + chunks - 1) / chunks);
+  const int row_chunks = (int)((I.m + rows_per_chunk - 1) / rows_per_chunk);
+  if ((long long)slices * row_chunks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+  int rc = ensure_err_flag(dev);
+  if (rc != B200SP_OK) return rc;
+  return launch_smem(kernel, dim3((unsigned)(slices * row_chunks)), dim3(THREADS), smem, stream, nullptr, 0, dev, map, (int)I.m, (int)I.n,
+                     k, row_chunks, rows_per_chunk, box_rows, p->row_ptr, col_idx, vals, Y, alpha, beta, dev->err_flag);
+}
+
+template <typename T, int VEC>
+int run_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const T* B, T* Y, float alpha, float beta,
+             cudaStream_t stream, DeviceInfo* dev) {
+  const b200sp_plan_info_t& I = p->info;
+  if (I.m == 0) return B200SP_OK;
+  if (alpha == 0.0f || I.nnz == 0) return run_scale<T>((long long)I.m * k, Y, beta, stream, dev);
+  if (k % VEC == 0 && g_opt.spmm_bstage && I.nnz >= 4 * I.n && ((size_t)k * sizeof(T)) % 16 == 0) {
+    // widest slice of B (128, 64 or 32 bytes per row) whose n rows fit in one SM's shared memory
+    const size_t budget = (size_t)kSmemPerSm - 4096;
+    const size_t n_pad = (size_t)((I.n + 255) / 256) * 256;
+    EncodeTiledFn encode = tensor_map_encoder();
+    if (encode && n_pad * 32 <= budget) {
+      int rc;
+      if (g_opt.bstage_threads == 256) {
+        if (n_pad * 128 <= budget) rc = launch_spmm_bstage<T, VEC, 8, 256>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+        else if (n_pad * 64 <= budget) rc = launch_spmm_bstage<T, VEC, 4, 256>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+        else rc = launch_spmm_bstage<T, VEC, 2, 256>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+      } else if (g_opt.bstage_threads == 512) {
+        if (n_pad * 128 <= budget) rc = launch_spmm_bstage<T, VEC, 8, 512>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+        else if (n_pad * 64 <= budget) rc = launch_spmm_bstage<T, VEC, 4, 512>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+        else rc = launch_spmm_bstage<T, VEC, 2, 512>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+      } else {
+        if (n_pad * 128 <= budget) rc = launch_spmm_bstage<T, VEC, 8>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+        else if (n_pad * 64 <= budget) rc = launch_spmm_bstage<T, VEC, 4>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+        else rc = launch_spmm_bstage<T, VEC, 2>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
+      }
+      if (rc != B200SP_ERR_UNSUPPORTED) return rc;   // unsupported shape for the tensor map: fall through to the sliced kernel
+    }
+  }
+  if (k % VEC == 0 && g_opt.spmm_sliced) {
+    constexpr int KS = 8 * VEC, GROUPS = kSpmmThreads / 8;
+    const int slices = (k + KS - 1) / KS;
+    const int row_blocks = (int)((I.m + GROUPS - 1) / GROUPS);
+    if ((long long)slices * row_blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+    int rc = launch(spmm_slice_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)(slices * row_blocks)), dim3(kSpmmThreads), stream,
+                    nullptr, 0, dev,
+                    (int)I.m, k, row_blocks, p->row_ptr, col_idx, vals, B, Y, alpha, beta, kLongRow);
+    if (rc != B200SP_OK || p->num_long == 0) return rc;
+    return launch(spmm_long_row_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)(slices * p->num_long)), dim3(kSpmmThreads), stream, nullptr, 0,
+                  dev, k, p->num_long, (const int*)p->long_rows, p->row_ptr, col_idx, vals, B, Y, alpha, beta);
+  }
+  if (k % VEC != 0) {  // ragged k: scalar lanes
+    if (k <= 8) return launch_spmm<T, 1, 8, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+    return launch_spmm<T, 1, 32, 2>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+  }
+  const int vecs = k / VEC;  // vector columns per row
+  if (vecs <= 4) return launch_spmm<T, VEC, 4, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+  if (vecs <= 8) return launch_spmm<T, VEC, 8, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+  if (vecs <= 16) return launch_spmm<T, VEC, 16, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+  if (vecs <= 32) return launch_spmm<T, VEC, 32, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+  return launch_spmm<T, VEC, 32, 2>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+}
+
+}  // namespace
