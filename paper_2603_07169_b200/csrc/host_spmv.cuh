@@ -282,46 +282,3 @@ int run_spmv(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, 
 }
 
 }  // namespace
-
-// ---- scratch for spmv_csr_noalloc: lives in the library image, one copy per GPU that loads it ----
-constexpr int kNoAllocMaxTiles = 65536;   // merge tiles of kItems items: m + nnz <= 65536 * 4096 = 268,435,456
-struct NoAllocScratch {
-  int32_t split_row[kNoAllocMaxTiles + 4];
-  float carry[kNoAllocMaxTiles];
-  float tail[kNoAllocMaxTiles];
-};
-static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
-// In host code the name above is only a handle; the device address comes from cudaGetSymbolAddress,
-// looked up once per device with that device current.
-static NoAllocScratch* g_noalloc_ptr[64] = {};
-
-static int noalloc_scratch(NoAllocScratch** out) {
-  int dev = 0;
-  CU(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return B200SP_ERR_UNSUPPORTED;
-  std::lock_guard<std::mutex> lock(g_mutex);
-  if (!g_noalloc_ptr[dev]) {
-    void* ptr = nullptr;
-    CU(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
-    g_noalloc_ptr[dev] = static_cast<NoAllocScratch*>(ptr);
-  }
-  *out = g_noalloc_ptr[dev];
-  return B200SP_OK;
-}
-
-template <typename T>
-static int run_spmv_noalloc(int64_t m, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx, const T* vals, const T* x, T* y,
-                            float alpha, float beta, cudaStream_t stream, DeviceInfo* dev, NoAllocScratch* sc) {
-  if (alpha == 0.0f || nnz == 0) return run_scale<T>(m, y, beta, stream, dev);
-  const int tiles = (int)((m + nnz + kItems - 1) / kItems);
-  int rc = launch(plan_merge_split_kernel, dim3((tiles + 1 + 255) / 256), dim3(256), stream, nullptr, 0, dev, row_ptr, (int)m, (int)nnz,
-                  kItems, tiles, (int*)sc->split_row);
-  if (rc != B200SP_OK) return rc;
-  rc = launch(spmv_merge_tile_kernel<T, kItems, kThreads, kShortMax>, dim3(tiles), dim3(kThreads), stream, nullptr, 0, dev, (int)m,
-              (int)nnz, row_ptr, col_idx, vals, x, y, alpha, beta, (const int*)sc->split_row, sc->carry, sc->tail);
-  if (rc != B200SP_OK) return rc;
-  if (tiles > 1)
-    rc = launch(spmv_carry_fixup_kernel<T, kItems>, dim3((tiles + 127) / 128), dim3(128), stream, nullptr, 0, dev, tiles, row_ptr,
-                (const int*)sc->split_row, (const float*)sc->carry, (const float*)sc->tail, y, alpha, beta);
-  return rc;
-}
