@@ -163,7 +163,7 @@ __device__ __forceinline__ void ld_a4(const int* col_idx, const bf16_t* vals, in
 // VEC columns of the slice in FP32 registers with four independent 16-byte reads of B in flight.
 // Rows longer than long_thresh are left to spmm_long_row_kernel.
 template <typename T, int VEC, int THREADS>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 2048 / THREADS)
 spmm_slice_kernel(int m, int k, int row_blocks, const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
                   const T* __restrict__ vals, const T* __restrict__ B, T* __restrict__ Y, float alpha, float beta, int long_thresh) {
   constexpr int LANES = 8, GROUPS = THREADS / LANES, KS = LANES * VEC;
