@@ -42,7 +42,7 @@ NCU_TRAFFIC_BYTES = {
     ("c3", "f32"): 305_818_112,     # profiles/spmv_merge_tile_c3_f32.md
     ("c4", "bf16"): 690_968_832,    # profiles/spmv_row_tile_c4_bf16.md
     ("c1", "f32"): 3_163_648,       # profiles/spmv_row_tile_c1_f32.md
-    ("c5k64", "f32"): 1_136_199_368,  # profiles/spmm_slice_c5k64_f32.md
+    ("c5k64", "f32"): 1_274_698_040,  # profiles/spmm_slice_c5k64_f32.md
 }
 
 
