@@ -227,6 +227,9 @@ int64_t b200sp_launch_count(void);
  *   "sub_lanes"      lanes per row of the sub-warp kernel (1..32, power of two), 0 = from the mean row length
  *   "spmm_bstage"    1 = SpMM keeps a slice of B in shared memory when A has few columns (default), 0 = never
  *   "spmm_sliced"    1 = SpMM walks k in 128-byte slices so that a slice of B stays in L2 (default), 0 = one pass
+ *   "merge_scan"     1 = merge kernel that reduces rows with an in-register segmented scan, 0 = products parked in
+ *                    shared memory and added per row (default)
+ *   "merge_stride"   with merge_scan: walk the tiles with this stride (made coprime to their number), 0 = in order
  *   "merge_staged"   1 = persistent staged merge kernel, 0 = one tile per CTA (default)
  *   "merge_threads"  threads per CTA of the one-tile-per-CTA merge kernel, 128 or 256
  *   "merge_carve"    shared-memory carveout in percent requested for it (-1 = driver default)

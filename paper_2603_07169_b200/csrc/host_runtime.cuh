@@ -59,6 +59,8 @@ struct Options {
   int spmm_bstage = 1;     // 1 = hold the slice of B in shared memory when A has few columns (default), 0 = never
   int spmm_sliced = 1;     // 1 = k-sliced SpMM kernel (default), 0 = one pass over all of k
   int sub_lanes = 0;       // lanes per row of the sub-warp kernel (0 = from the mean row length)
+  int merge_stride = 0;    // tile order of the scan merge kernel: stride through the tiles (0 / 1 = plain order)
+  int merge_scan = 0;      // 1 = merge kernel with the in-register segmented scan, 0 = products through shared memory (default: as fast on power-law rows, faster on short rows)
   int merge_short = 32;    // rows up to this many products are added by one thread (8, 16, 32, 64)
   int merge_carve = 30;    // shared-memory carveout (percent) requested for it, -1 = leave to the driver
 } g_opt;

@@ -6,6 +6,7 @@
 #include "spmv_row_kernels.cuh"
 #include "spmv_uniform_kernels.cuh"
 #include "spmv_merge_stage_kernels.cuh"
+#include "spmv_merge_scan_kernels.cuh"
 
 namespace {
 
@@ -178,6 +179,17 @@ int run_spmv_merge(b200sp_plan* p, const int32_t* col_idx, const T* vals, const 
     const int grid = tiles < ctas * dev->sms ? tiles : ctas * dev->sms;
     rc = launch_smem(kernel, dim3(grid), dim3(kThreads), smem, stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr,
                      col_idx, vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail, tiles, stages, dev->err_flag);
+  } else if (g_opt.merge_scan && ITEMS <= 2048) {
+    constexpr int SCAN_ITEMS = ITEMS <= 2048 ? ITEMS : 2048;
+    auto kernel = spmv_merge_scan_kernel<T, SCAN_ITEMS, 128>;
+    if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
+    int stride = 1;   // tile order: a stride coprime to the tile count (1 = plain order)
+    if (g_opt.merge_stride > 1 && tiles > 2 * g_opt.merge_stride) {
+      stride = g_opt.merge_stride;
+      while (gcd_int(stride, tiles) != 1) ++stride;
+    }
+    rc = launch(kernel, dim3(tiles), dim3(128), stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx,
+                vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail, stride);
   } else if (g_opt.merge_threads == 64) {
     auto kernel = spmv_merge_tile_kernel<T, ITEMS, 64, SHORT>;
     if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));

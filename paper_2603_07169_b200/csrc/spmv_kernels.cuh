@@ -28,7 +28,8 @@ spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const in
   constexpr int MAX_LONG = ITEMS / (SHORT_MAX + 1) + 2;
   constexpr int WARPS = THREADS / 32;
   __shared__ float prod[PROD_N + PROD_N / 32 + 1];
-  __shared__ int long_rows[MAX_LONG];
+  __shared__ int long_rows[MAX_LONG];       // row of each long segment; -row-1 when the row began in an earlier tile
+  __shared__ int2 long_span[MAX_LONG];      // its products: local [first, last)
   __shared__ int n_long;
 
   const int tid = threadIdx.x;
@@ -40,6 +41,7 @@ spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const in
   const int p0 = (int)(d0 - r0), p1 = (int)(d1 - r1);
   const int a0 = p0 & ~(G - 1);
   if (tid == 0) n_long = 0;
+  const int carry_start = r1 < m ? __ldg(row_ptr + r1) : 0;   // start of the unfinished last row, needed in phase 3: requested early
 
   // ---- phase 1: products of nonzeros [p0, p1) in flat order
   const int nq = (p1 - a0 + G - 1) / G;
@@ -95,7 +97,9 @@ spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const in
       if (rs < p0) tail[t] = acc;            // row began in an earlier tile: completed by the fix-up kernel
       else epilogue_store(y, r, acc, alpha, beta);
     } else {
-      long_rows[atomicAdd(&n_long, 1)] = r;  // order of the list does not affect any value
+      const int slot = atomicAdd(&n_long, 1);  // order of the list does not affect any value
+      long_rows[slot] = rs < p0 ? -r - 1 : r;
+      long_span[slot] = make_int2(s - a0, re - a0);
     }
   }
   __syncthreads();
@@ -105,20 +109,19 @@ spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const in
   const int nl = n_long;
   for (int i = warp; i < nl; i += WARPS) {
     const int r = long_rows[i];
-    const int rs = row_ptr[r], re = row_ptr[r + 1];
-    const int s = max(rs, p0);
+    const int2 span = long_span[i];
     float acc = 0.0f;
-    for (int q = s - a0 + lane; q < re - a0; q += 32) acc += prod[pad_index(q)];
+    for (int q = span.x + lane; q < span.y; q += 32) acc += prod[pad_index(q)];
     acc = warp_sum(acc);
     if (lane == 0) {
-      if (rs < p0) tail[t] = acc;
+      if (r < 0) tail[t] = acc;
       else epilogue_store(y, r, acc, alpha, beta);
     }
   }
   if (warp == WARPS - 1) {
     float acc = 0.0f;
     if (r1 < m) {
-      const int s = max(row_ptr[r1], p0);
+      const int s = max(carry_start, p0);
       for (int q = s - a0 + lane; q < p1 - a0; q += 32) acc += prod[pad_index(q)];
       acc = warp_sum(acc);
     }

@@ -144,10 +144,14 @@ def test_workloads_full_size(name):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
-@pytest.mark.parametrize("staged,items,stages", [(0, 2048, 3), (0, 4096, 3), (1, 2048, 2), (1, 2048, 4), (1, 4096, 3)])
+@pytest.mark.parametrize("staged,items,stages", [(0, 2048, 3), (0, 4096, 3), (1, 2048, 2), (1, 2048, 4), (1, 4096, 3), (2, 2048, 3), (2, 1024, 3)])
 def test_merge_kernel_variants(staged, items, stages, dtype):
-    """Both merge kernels (one tile per CTA; persistent with staged copies) at both tile sizes."""
+    """The merge kernels (one tile per CTA; persistent with staged copies; staged = 2: in-register segmented scan with a
+    strided tile order) at their tile sizes."""
     b200sp.b200sp_set_option("spmv_kernel", 0)
+    b200sp.b200sp_set_option("merge_scan", 1 if staged == 2 else 0)
+    b200sp.b200sp_set_option("merge_stride", 101 if staged == 2 else 0)
+    staged = 0 if staged == 2 else staged
     b200sp.b200sp_set_option("merge_staged", staged)
     b200sp.b200sp_set_option("merge_items", items)
     b200sp.b200sp_set_option("merge_stages", stages)
@@ -161,7 +165,7 @@ def test_merge_kernel_variants(staged, items, stages, dtype):
             assert_within(y, y_ref, S, dtype, what="%s staged=%d items=%d" % (name, staged, items))
         b200sp.b200sp_check()
     finally:
-        for k, v in (("spmv_kernel", -1), ("merge_staged", 1), ("merge_items", 2048), ("merge_stages", 3)):
+        for k, v in (("spmv_kernel", -1), ("merge_staged", 0), ("merge_items", 2048), ("merge_stages", 3), ("merge_scan", 0), ("merge_stride", 0)):
             b200sp.b200sp_set_option(k, v)
 
 
