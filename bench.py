@@ -157,11 +157,11 @@ def measure(w, dtype, steps, warmup, dev, l2_bytes, barrier=None, min_copies=2, 
     sets = [DeviceSet(w, dtype, dev) for _ in range(R)]
     stream = torch.cuda.current_stream()
 
-    def call(s):
+    def call(s, st=stream):                  # st: the launching stream (a capture stream when recorded into a CUDA graph)
         if w.k:
-            b200sp.spmm_csr(A.m, A.n, A.nnz, w.k, s.rp, s.ci, s.va, s.inp, s.out, w.alpha, w.beta, dtype, stream)
+            b200sp.spmm_csr(A.m, A.n, A.nnz, w.k, s.rp, s.ci, s.va, s.inp, s.out, w.alpha, w.beta, dtype, st)
         else:
-            b200sp.spmv_csr(A.m, A.n, A.nnz, s.rp, s.ci, s.va, s.inp, s.out, w.alpha, w.beta, dtype, stream)
+            b200sp.spmv_csr(A.m, A.n, A.nnz, s.rp, s.ci, s.va, s.inp, s.out, w.alpha, w.beta, dtype, st)
 
     t_plan0 = time.perf_counter()
     call(sets[0])                       # first call builds and caches the plan for this row_ptr
@@ -197,9 +197,19 @@ def measure(w, dtype, steps, warmup, dev, l2_bytes, barrier=None, min_copies=2, 
         b.synchronize()
         iso.append(a.elapsed_time(b))
     iso.sort()
+    # warm: the same operand set back to back (whatever fits stays in L2; not comparable with the HBM roofline)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    call(sets[0])
+    a.record(stream)
+    for i in range(min(steps, 50)):
+        call(sets[0])
+    b.record(stream)
+    b.synchronize()
+    warm_ms = a.elapsed_time(b) / min(steps, 50)
     ms_step = ms / steps
     flops = 2.0 * A.nnz * max(w.k, 1)
-    res = {"ms_total": ms, "ms_per_step": ms_step, "ms_per_step_isolated_median": iso[len(iso) // 2], "gbs": abytes / ms_step * 1e-6,
+    res = {"ms_total": ms, "ms_per_step": ms_step, "ms_per_step_isolated_median": iso[len(iso) // 2], "ms_per_step_warm": warm_ms,
+           "gbs": abytes / ms_step * 1e-6,
            "gflops": flops / ms_step * 1e-6, "algorithmic_bytes": abytes, "copies": R, "launches": launches,
            "plan_ms_first_call": plan_ms, "t0": t0, "t1": t1, "nnz": A.nnz, "m": A.m}
     res["cusparse_ms"] = None
@@ -255,6 +265,44 @@ def measure_format(kind, w, dtype, steps, dev, l2_bytes):
     ms = a.elapsed_time(b) / steps
     b200sp.b200sp_cache_clear()
     return {"ms_per_step": round(ms, 5), "gbs": round(abytes / ms * 1e-6, 1), "algorithmic_bytes": abytes, "copies": R}
+
+
+def latency_floor(call, sets, dev, nbytes):
+    """Per-call device time of 100 calls replayed from a CUDA graph, beside an empty kernel and a copy of the same bytes."""
+    import torch
+    import paper_2603_07169_b200 as b200sp
+
+    def graph_us(fn, calls=100, replays=5):
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                for i in range(calls):
+                    fn(i)
+        torch.cuda.current_stream().wait_stream(side)
+        g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(replays):
+            g.replay()
+        b.record()
+        b.synchronize()
+        return a.elapsed_time(b) / (replays * calls) * 1e3
+
+    out = {}
+    try:
+        tab = torch.zeros(1024, dtype=torch.float32, device=dev)
+        sink = torch.zeros(1, dtype=torch.float32, device=dev)
+        src = torch.zeros(nbytes // 8, dtype=torch.float32, device=dev)
+        dst = torch.empty_like(src)
+        out["graph_replay_us_per_call"] = round(graph_us(lambda i: call(sets[i % len(sets)], torch.cuda.current_stream())), 3)
+        out["empty_kernel_us"] = round(graph_us(lambda i: b200sp.b200sp_probe_gather(tab, 1024, 0, sink, torch.cuda.current_stream())), 3)
+        out["copy_same_bytes_us"] = round(graph_us(lambda i: dst.copy_(src)), 3)
+    except Exception as ex:  # pragma: no cover
+        out["latency_floor_error"] = repr(ex)
+    return out
 
 
 def aggregate_over_ranks(ms_local: float, bytes_per_step: int, steps: int, world: int, dist=None, device="cpu"):
@@ -641,10 +689,13 @@ def main():
                 r = measure(ww, dt, min(steps, 50), 5, dev, l2, cusparse=cusp)
                 extras["%s_%s" % (name, dt)] = {
                     "ms_per_step": round(r["ms_per_step"], 5), "ms_isolated_median": round(r["ms_per_step_isolated_median"], 5),
+                    "ms_warm_l2": round(r["ms_per_step_warm"], 5),
                     "gbs": round(r["gbs"], 1), "frac_of_hbm": round(r["gbs"] / peak, 4), "gflops": round(r["gflops"], 1),
                     "algorithmic_bytes": r["algorithmic_bytes"], "nnz": r["nnz"], "copies": r["copies"],
                     "plan_ms_first_call": round(r["plan_ms_first_call"], 3),
                     "cusparse_ms": round(r["cusparse_ms"], 5) if isinstance(r["cusparse_ms"], float) else r["cusparse_ms"]}
+                if name == "c1":   # launch-latency regime: per-call device time from a CUDA graph, and the floors on the same box
+                    extras["c1_f32"].update(latency_floor(r["_call"], r["_sets"], dev, r["algorithmic_bytes"]))
                 if not ww.k:   # SpMV: time at the measured L1-miss gather rate for this x
                     extras["%s_%s" % (name, dt)]["gather_bound_ms"] = round(ww.A.nnz / probe_gather_rate(ww.A.n, dev) * 1e3, 5)
                 del r
@@ -696,6 +747,7 @@ def main():
                   % (head["copies"], head["copies"] * head["algorithmic_bytes"] / 1e6, l2 / 1e6),
             "plan": "cached per row_ptr; first call incl. plan %.3f ms (excluded)" % head["plan_ms_first_call"],
             "ms_per_step_isolated_median": head["ms_per_step_isolated_median"],
+            "ms_per_step_warm_l2": head["ms_per_step_warm"],
             "parallelism": "replicas only (single-GPU path)" if world > 1 else "1 GPU"}
         achieved = head["algorithmic_bytes"] / (head["ms_total"] / steps) * 1e-6
         line = {"metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup,
