@@ -111,3 +111,32 @@ def test_host_buffer_entry_point(dtype):
     b200sp.spmm_csr_host(A.m, A.n, A.nnz, w.k, A.row_ptr, A.col_idx, vals, B, Y, 1.0, 0.0, dtype)
     Y_ref, S = oracle.spmm_csr(A.m, A.n, w.k, A.row_ptr, A.col_idx, vals, B, None, 1.0, 0.0, dtype)
     assert_within(Y.reshape(A.m, w.k), Y_ref, S, dtype)
+
+
+def test_output_larger_than_2_31_elements():
+    """m * k > 2^31: the row-times-k offsets must be 64-bit.  BF16 storage, few columns (the kernel that holds a slice of B in
+    shared memory) and the k-sliced kernel; only sampled rows are copied back and compared."""
+    import torch
+    from gpu_util import to_dev
+    m, n, k = 600_000, 2048, 4096
+    rng = np.random.default_rng(77)
+    lens = rng.integers(4, 17, m)
+    A = gen.random_csr(m, n, lens, seed=9, sort_cols=True)
+    B = gen.to_bf16(rng.standard_normal(n * k).astype(np.float32))
+    vals = gen.to_bf16(A.vals)
+    d_rp, d_ci, d_va, d_B = to_dev(A.row_ptr), to_dev(A.col_idx), to_dev(vals), to_dev(B)
+    rows = np.unique(np.concatenate([[0, m - 1, 524_288, 524_289], rng.integers(0, m, 300)])).astype(np.int64)
+    Y_ref, S = oracle.spmm_csr(m, n, k, A.row_ptr, A.col_idx, vals, B, None, 1.0, 0.0, "bf16", rows=rows, nthreads=oracle.max_threads())
+    for bstage in (1, 0):
+        b200sp.b200sp_set_option("spmm_bstage", bstage)
+        try:
+            d_Y = torch.full((m * k,), 0x7FC0, dtype=torch.int16, device="cuda:0")      # NaN patterns: every entry must be overwritten
+            b200sp.spmm_csr(m, n, A.nnz, k, d_rp, d_ci, d_va, d_B, d_Y, 1.0, 0.0, "bf16")
+            torch.cuda.synchronize()
+            Y = d_Y.view(m, k)[torch.from_numpy(rows).to("cuda:0")].cpu().numpy().view(np.uint16)
+            assert_within(Y, Y_ref, S, "bf16", what="m*k > 2^31, bstage=%d" % bstage)
+            del d_Y
+        finally:
+            b200sp.b200sp_set_option("spmm_bstage", 1)
+            b200sp.b200sp_cache_clear()
+    b200sp.b200sp_check()
