@@ -221,29 +221,37 @@ int b200sp_probe_gather(const float* table, int64_t table_elems, int64_t gathers
 /* Number of kernels this library has launched from this process so far (all entry points). */
 int64_t b200sp_launch_count(void);
 
-/* Tuning switches for A/B measurements; unknown names return B200SP_ERR_INVALID_ARG.
- *   "spmv_kernel"   -1 = choose from the plan statistics (default), 0 = merge-tile, 1 = row-direct,
- *                    2 = uniform-row, 3 = sub-warp per row; a kernel the matrix is not eligible for falls back
- *   "sub_lanes"      lanes per row of the sub-warp kernel (1..32, power of two), 0 = from the mean row length
+/* Tuning switches for A/B measurements (the defaults are what the measurements in the repository selected);
+ * unknown names or values out of range return B200SP_ERR_INVALID_ARG.
+ *  kernel choice
+ *   "spmv_kernel"    -1 = choose from the plan statistics (default), 0 = merge-tile, 1 = row-direct, 2 = uniform-row,
+ *                    3 = sub-warp per row; a kernel the matrix is not eligible for falls back to an eligible one
  *   "spmm_bstage"    1 = SpMM keeps a slice of B in shared memory when A has few columns (default), 0 = never
- *   "spmm_sliced"    1 = SpMM walks k in 128-byte slices so that a slice of B stays in L2 (default), 0 = one pass
- *   "merge_scan"     1 = merge kernel that reduces rows with an in-register segmented scan, 0 = products parked in
- *                    shared memory and added per row (default)
+ *   "spmm_sliced"    1 = SpMM walks k in 128-byte slices so that a slice of B can stay in L2 (default), 0 = one pass
+ *  merge-tile SpMV kernel
+ *   "merge_items"    merge items per tile: 1024, 2048 (default) or 4096
+ *   "merge_threads"  threads per CTA: 64, 128 (default) or 256
+ *   "merge_carve"    shared-memory carveout in percent requested for it, default 30 (-1 = leave to the driver)
+ *   "merge_short"    rows of up to this many products are added by one thread: 8, 16, 32 (default) or 64
+ *   "merge_scan"     1 = reduce rows with an in-register segmented scan, 0 = products through shared memory (default)
  *   "merge_stride"   with merge_scan: walk the tiles with this stride (made coprime to their number), 0 = in order
- *   "merge_staged"   1 = persistent staged merge kernel, 0 = one tile per CTA (default)
- *   "merge_threads"  threads per CTA of the one-tile-per-CTA merge kernel, 128 or 256
- *   "merge_carve"    shared-memory carveout in percent requested for it (-1 = driver default)
- *   "merge_items"    merge items per tile, 2048 or 4096 (applies to plans created afterwards)
- *   "merge_stages"   shared-memory stages per CTA of the staged merge kernel, 2..4
- *   "merge_ctas"     CTAs per SM of the staged merge kernel
- *   "uni_unroll"     groups of four nonzeros in flight per thread of the uniform-row kernel: 1, 2 or 4
- *   "uni_ctas"       CTAs per SM for the uniform-row kernel, 0 = as many as fit
+ *   "merge_staged"   1 = persistent variant with bulk-copy stages, 0 = one tile per CTA (default)
+ *   "merge_stages", "merge_ctas"   stages per CTA (2..4) and CTAs per SM of the staged variant
+ *  row-direct SpMV kernel
+ *   "row_stages"     shared-memory stages per CTA, 2 (default) .. 4
+ *   "row_ctas"       CTAs per SM the tiles are sized for, default 3
+ *   "row_smem_kb"    shared memory per SM it may use for stages, default 220 (what is left stays L1)
+ *   "row_threads"    threads per CTA, 128 or 256 (default)
+ *   "row_unroll"     gathers in flight per thread, 8 (default) or 16
+ *  other kernels
+ *   "uni_unroll"     groups of four nonzeros in flight per thread of the uniform-row kernel: 1, 2 (default) or 4
+ *   "uni_ctas"       CTAs per SM for the uniform-row kernel, 0 = as many as fit (default)
+ *   "sub_lanes"      lanes per row of the sub-warp kernel (1..32, power of two), 0 = from the mean row length (default)
+ *   "bstage_threads" threads per CTA of the SpMM kernel with B in shared memory: 256, 512 or 1024 (default)
+ *   "bstage_nnz"     nonzeros of A per CTA that kernel aims for, default 131072
  *   "x_l2_window"    1 = pin x in L2 with a per-launch access-policy window, 0 = off (default: measured to give
  *                    nothing on large problems, where x stays in L2 anyway, and to cost 1.4 us per launch on tiny ones)
- *   "row_stages"     shared-memory stages per CTA of the row-direct kernel, 2..4
- *   "row_ctas"       CTAs per SM the row-direct kernel sizes its tiles for, 1..4
- *   "row_unroll"     gathers in flight per thread in the row-direct kernel: 4, 8 or 16
- * "spmv_kernel" applies to plans created afterwards, the others to the next call. */
+ * "spmv_kernel" and "merge_items" apply to plans created afterwards, the others to the next call. */
 int b200sp_set_option(const char* name, int value);
 
 #ifdef __cplusplus
