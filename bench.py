@@ -756,6 +756,7 @@ def main():
                 "gpu_launches": int(head["launches"]),
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                              "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dtype)), "peak_kind": "of " + peak_kind,
+                             "frac_of_nominal_7700": achieved / 7700.0,
                              "note": "algorithmic bytes per step over event time per step (the step is the SpMV kernel; plan cached)",
                              "secondary": None if gather_rate is None else {
                                  "bound": "L1-miss gather (one L2 request per random x read)", "gathers_per_s": gather_rate,
