@@ -677,7 +677,7 @@ def main():
     if not args.no_extras and rank == 0:
         del head["_sets"], head["_call"]
         torch.cuda.empty_cache()
-        todo = [("c2", "bf16"), ("c3", "f32"), ("c4", "bf16"), ("c1", "f32"), ("c5k64", "f32"), ("c5k64", "bf16"),
+        todo = [("c2", "bf16"), ("c3", "f32"), ("c3p", "f32"), ("c4", "bf16"), ("c1", "f32"), ("c5k64", "f32"), ("c5k64", "bf16"),
                 ("c5k256", "f32"), ("c5k256", "bf16")]
         cache = {args.workload: w}
         for name, dt in todo:

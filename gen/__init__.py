@@ -51,6 +51,8 @@ def _L():
         lib.gen_uniform_rows.argtypes = [i64, i64, i32, u64, p, p, p]
         lib.gen_rmat.argtypes = [i32, i64, f64, f64, f64, u64, p, p, p]
         lib.gen_rmat.restype = i64
+        lib.gen_rmat_relabel.argtypes = [i32, i64, f64, f64, f64, u64, p, p, p]
+        lib.gen_rmat_relabel.restype = i64
         lib.gen_stencil27_nnz.argtypes = [i64]
         lib.gen_stencil27_nnz.restype = i64
         lib.gen_stencil27.argtypes = [i64, f32, f32, f32, u64, p, p, p]
@@ -137,12 +139,14 @@ def uniform_rows(m: int, n: int, per_row: int, seed: int) -> CSR:
     return CSR(m, n, rp, ci, va, "uniform%d_%d" % (per_row, m))
 
 
-def rmat(scale: int, e_gen: int, seed: int, a: float = 0.57, b: float = 0.19, c: float = 0.19) -> CSR:
-    """R-MAT graph on 2^scale vertices from e_gen generated edges (sorted, duplicates dropped), values (0, 1]."""
+def rmat(scale: int, e_gen: int, seed: int, a: float = 0.57, b: float = 0.19, c: float = 0.19, relabel: bool = False) -> CSR:
+    """R-MAT graph on 2^scale vertices from e_gen generated edges (sorted, duplicates dropped), values (0, 1].
+    ``relabel`` renames every vertex by one pseudo-random bijection (same edges, same degrees, no index locality)."""
     m = 1 << scale
     rp, ci, va = np.empty(m + 1, np.int32), np.empty(e_gen, np.int32), np.empty(e_gen, np.float32)
-    nnz = _L().gen_rmat(scale, e_gen, a, b, c, seed, _ptr(rp), _ptr(ci), _ptr(va))
-    return CSR(m, m, rp, ci[:nnz].copy(), va[:nnz].copy(), "rmat_%d" % scale)
+    fn = _L().gen_rmat_relabel if relabel else _L().gen_rmat
+    nnz = fn(scale, e_gen, a, b, c, seed, _ptr(rp), _ptr(ci), _ptr(va))
+    return CSR(m, m, rp, ci[:nnz].copy(), va[:nnz].copy(), "rmat_%d%s" % (scale, "_relabel" if relabel else ""))
 
 
 def stencil27(N: int, seed: int, diag: float = 26.0, off: float = -1.0, sigma: float = 0.01) -> CSR:
@@ -254,6 +258,7 @@ def workload(name: str, scale_down: int = 0) -> Workload:
     c1  2D 5-point Laplacian 256^2, x U[-1,1), alpha 1, beta 0                       (FP32)
     c2  m = n = 2^20, exactly 16 nnz/row, vals N(0,1), x and y0 U[-1,1), alpha 1.5, beta 0.5 (FP32, BF16)
     c3  R-MAT scale 22, 34.14 M generated edges, vals and x U(0,1], alpha 1, beta 0    (FP32)
+    c3p the edges of c3 with every vertex renamed by one pseudo-random bijection (secondary measurement) (FP32)
     c4  27-point stencil 160^3, diag 26, off -1 + N(0, 0.01^2), x N(0,1)               (BF16)
     c5k64 / c5k256  m = n = 2^19, 32 nnz/row, vals N(0,1), B N(0,1) n x k              (FP32, BF16)
     """
@@ -272,6 +277,11 @@ def workload(name: str, scale_down: int = 0) -> Workload:
         e_gen = 34_140_000 >> (2 * s)
         A = rmat(scale, e_gen, 1003)
         return Workload("c3", A, x=uniform_open_low(A.n, 1003, 10), dtypes=("f32",))
+    if name == "c3p":
+        scale = 22 - 2 * s
+        e_gen = 34_140_000 >> (2 * s)
+        A = rmat(scale, e_gen, 1003, relabel=True)
+        return Workload("c3p", A, x=uniform_open_low(A.n, 1003, 10), dtypes=("f32",))
     if name == "c4":
         N = 160 >> s
         A = stencil27(N, 1004)

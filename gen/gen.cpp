@@ -112,8 +112,35 @@ void gen_uniform_rows(int64_t m, int64_t n, int32_t per_row, uint64_t seed,
 // (a, b, c, 1-a-b-c) per level; no noise, no relabelling, self loops kept; sorted by (row, col),
 // duplicates dropped.  Returns nnz after dedup; the caller passes buffers of e_gen entries.
 // Values uniform (0,1].
+// A bijection of [0, 2^scale): two rounds of xor-shift and an odd multiply-add, each invertible mod 2^scale.
+static inline uint32_t relabel_vertex(uint32_t v, int32_t scale, uint64_t seed) {
+  const uint32_t mask = scale >= 32 ? 0xFFFFFFFFu : ((1u << scale) - 1u);
+  const int32_t sh = scale / 2 > 0 ? scale / 2 : 1;
+  const uint32_t m1 = ((uint32_t)rnd(seed, 300, 0) | 1u), m2 = ((uint32_t)rnd(seed, 300, 1) | 1u);
+  const uint32_t c1 = (uint32_t)(rnd(seed, 300, 2)), c2 = (uint32_t)(rnd(seed, 300, 3));
+  v ^= v >> sh; v = (v * m1 + c1) & mask;
+  v ^= v >> sh; v = (v * m2 + c2) & mask;
+  v ^= v >> sh;
+  return v;
+}
+
+static int64_t gen_rmat_impl(int32_t scale, int64_t e_gen, double a, double b, double c, uint64_t seed, bool relabel,
+                             int32_t* row_ptr, int32_t* col_idx, float* vals);
+
 int64_t gen_rmat(int32_t scale, int64_t e_gen, double a, double b, double c, uint64_t seed,
                  int32_t* row_ptr, int32_t* col_idx, float* vals) {
+  return gen_rmat_impl(scale, e_gen, a, b, c, seed, false, row_ptr, col_idx, vals);
+}
+
+// Same edges with every vertex renamed by one pseudo-random bijection (rows and columns alike): the
+// degree distribution stays, the hot rows and columns no longer sit together at the low indices.
+int64_t gen_rmat_relabel(int32_t scale, int64_t e_gen, double a, double b, double c, uint64_t seed,
+                         int32_t* row_ptr, int32_t* col_idx, float* vals) {
+  return gen_rmat_impl(scale, e_gen, a, b, c, seed, true, row_ptr, col_idx, vals);
+}
+
+static int64_t gen_rmat_impl(int32_t scale, int64_t e_gen, double a, double b, double c, uint64_t seed, bool relabel,
+                             int32_t* row_ptr, int32_t* col_idx, float* vals) {
   std::vector<uint64_t> keys((size_t)e_gen);
   const uint32_t ta = (uint32_t)std::llround(a * 4294967296.0);
   const uint32_t tb = (uint32_t)std::llround((a + b) * 4294967296.0);
@@ -130,6 +157,7 @@ int64_t gen_rmat(int32_t scale, int64_t e_gen, double a, double b, double c, uin
       row = (row << 1) | rb;
       col = (col << 1) | cb;
     }
+    if (relabel) { row = relabel_vertex(row, scale, seed); col = relabel_vertex(col, scale, seed); }
     keys[(size_t)e] = ((uint64_t)row << 32) | col;
   }
 #ifdef _OPENMP

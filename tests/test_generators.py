@@ -57,6 +57,20 @@ def test_rmat_small_is_power_law():
     assert 0.9 < A.nnz / (34_140_000 >> 6) <= 1.0
 
 
+def test_rmat_relabel_keeps_degrees_and_moves_hubs():
+    A = gen.rmat(14, 140_000, 7)
+    B = gen.rmat(14, 140_000, 7, relabel=True)
+    check_csr(B)
+    assert sorted_unique_rows(B)
+    assert A.nnz == B.nnz      # a bijection on vertex names merges no two distinct edges
+    assert np.array_equal(np.sort(np.diff(A.row_ptr)), np.sort(np.diff(B.row_ptr)))
+    assert np.array_equal(np.sort(np.bincount(A.col_idx, minlength=A.n)), np.sort(np.bincount(B.col_idx, minlength=B.n)))
+    assert np.diff(B.row_ptr).argmax() != 0
+    # hot columns are no longer packed at the low indices
+    half = lambda M: (M.col_idx < M.n // 2).mean()
+    assert half(A) > 0.7 and 0.35 < half(B) < 0.65
+
+
 def test_stencil27():
     A = gen.stencil27(20, 1004)
     check_csr(A)

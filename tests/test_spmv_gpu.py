@@ -125,7 +125,7 @@ def test_integer_data_is_exact_fp32():
 
 
 # ---------------------------------------------------------------- the measured workloads
-@pytest.mark.parametrize("name,scale", [("c1", 0), ("c2", 2), ("c3", 2), ("c4", 2)])
+@pytest.mark.parametrize("name,scale", [("c1", 0), ("c2", 2), ("c3", 2), ("c3p", 2), ("c4", 2)])
 def test_workloads_scaled(name, scale, kernel_choice):
     w = gen.workload(name, scale_down=scale)
     for dtype in w.dtypes:
