@@ -42,6 +42,8 @@ spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const in
   const int a0 = p0 & ~(G - 1);
   if (tid == 0) n_long = 0;
   const int carry_start = r1 < m ? __ldg(row_ptr + r1) : 0;   // start of the unfinished last row, needed in phase 3: requested early
+  // the row bounds of phase 2 come straight from global memory: start them towards L2 now
+  for (int r = r0 + tid * 32; r <= r1; r += THREADS * 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(row_ptr + r));
 
   // ---- phase 1: products of nonzeros [p0, p1) in flat order
   const int nq = (p1 - a0 + G - 1) / G;
