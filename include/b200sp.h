@@ -34,6 +34,10 @@
  *    size, unknown dtype, k <= 0, misaligned pointer) return B200SP_ERR_INVALID_ARG and launch
  *    nothing; a device that is not compute capability 10.x returns B200SP_ERR_ARCH; a failing CUDA
  *    call returns B200SP_ERR_CUDA and its message is kept for b200sp_last_cuda_error().
+ *  - Device memory the library needs (plan scratch, the staging buffers of the "host" entry
+ *    points) comes from a stream-ordered memory pool of its own, one per device, created at first
+ *    use.  The pool keeps up to 1 GiB of freed memory for the next call (option "pool_keep_mb",
+ *    read when the pool is created); b200sp_cache_clear hands all unused pool memory back.
  *  - There is no CPU fallback: without a B200 the compute entry points fail.
  */
 #ifndef B200SP_H_
@@ -100,8 +104,9 @@ int spmm_csr(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_pt
  * When the row statistics select the row-direct SpMV kernel, the first b200sp_spmv / spmv_csr call with a given
  * col_idx additionally samples how local the columns are (one small kernel and one synchronisation of the stream)
  * and falls back to the merge-tile kernel for matrices with scattered columns.
- * It allocates a few bytes per tile of device memory (released by b200sp_plan_destroy) and
- * synchronises `stream` once.  A plan may be used from one stream at a time. */
+ * It takes one block of a few bytes per tile from the library's pool, in the order of `stream`, and
+ * synchronises `stream` once.  A plan may be used from one stream at a time.  b200sp_plan_destroy
+ * synchronises the plan's device before it returns the block. */
 int b200sp_plan_create(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, void* stream);
 int b200sp_plan_destroy(b200sp_plan* plan);
 int b200sp_plan_info(const b200sp_plan* plan, b200sp_plan_info_t* out); /* `out` is a host pointer */
@@ -172,7 +177,7 @@ int64_t b200sp_noalloc_max_items(void);   /* largest m + nnz that spmv_csr_noall
 
 /* ---- host-buffer calls -----------------------------------------------------------------------
  * Same operations with every array in HOST memory (pinned memory makes the copies asynchronous and
- * faster, pageable memory works).  Each call allocates device buffers from the stream-ordered pool,
+ * faster, pageable memory works).  Each call takes device buffers from the library's stream-ordered pool,
  * copies the inputs in, plans (cached per pattern shape is impossible here, so the plan is rebuilt),
  * runs the kernels, copies y / Y back and synchronises `stream` before returning. */
 int spmv_csr_host(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx,
@@ -191,7 +196,7 @@ int spmv_csr_vec_host(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr,
  * B200SP_ERR_BAD_CSR if any check fails. */
 int b200sp_validate_csr(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx, void* stream);
 
-void b200sp_cache_clear(void);                 /* destroys every plan cached by the one-shot calls */
+void b200sp_cache_clear(void);                 /* destroys every plan cached by the one-shot calls and trims the library's memory pools */
 const char* b200sp_status_string(int status);  /* static string, never NULL */
 const char* b200sp_last_cuda_error(void);      /* message of this thread's last failing CUDA call, "" if none */
 int b200sp_version(void);                      /* major * 10000 + minor * 100 + patch */
@@ -251,6 +256,9 @@ int64_t b200sp_launch_count(void);
  *   "bstage_nnz"     nonzeros of A per CTA that kernel aims for, default 131072
  *   "x_l2_window"    1 = pin x in L2 with a per-launch access-policy window, 0 = off (default: measured to give
  *                    nothing on large problems, where x stays in L2 anyway, and to cost 1.4 us per launch on tiny ones)
+ *  memory
+ *   "pool_keep_mb"   MiB of freed memory the library's pool keeps across synchronisation points, default 1024
+ *                    (read when a device's pool is created, i.e. before the first call that allocates on it)
  * "spmv_kernel" and "merge_items" apply to plans created afterwards, the others to the next call. */
 int b200sp_set_option(const char* name, int value);
 

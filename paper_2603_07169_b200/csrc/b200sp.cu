@@ -282,10 +282,11 @@ static int host_call(bool is_mm, int64_t m, int64_t n, int64_t nnz, int64_t k, c
   auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
   const size_t total = up(b_rp) + up(b_ci) + up(b_va) + up(b_in) + up(b_out) + 256;
   char* base = nullptr;
-  CU(cudaMallocAsync((void**)&base, total, stream));
+  rc = pool_alloc(dev, (void**)&base, total, stream);
+  if (rc != B200SP_OK) return rc;
   char* d_rp = base; char* d_ci = d_rp + up(b_rp); char* d_va = d_ci + up(b_ci); char* d_in = d_va + up(b_va); char* d_out = d_in + up(b_in);
   b200sp_plan* p = nullptr;
-  auto done = [&](int code) { if (p) plan_free(p); cudaFreeAsync(base, stream); cudaStreamSynchronize(stream); return code; };
+  auto done = [&](int code) { if (p) plan_free(p, true, stream); cudaFreeAsync(base, stream); cudaStreamSynchronize(stream); return code; };
 #define CUH(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return done(cuda_fail(e_, #call)); } while (0)
   CUH(cudaMemcpyAsync(d_rp, row_ptr, b_rp, cudaMemcpyHostToDevice, stream));
   if (nnz > 0) {
@@ -317,8 +318,12 @@ int spmv_csr_vec_host(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr,
   cudaStream_t stream = (cudaStream_t)stream_v;
   const size_t e = dtype == B200SP_F32 ? 4 : 2;
   const size_t bx = ((size_t)n * e + 255) & ~(size_t)255, by = (size_t)m * e;
+  DeviceInfo* dev = nullptr;
+  rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
   char* base = nullptr;
-  CU(cudaMallocAsync((void**)&base, bx + by + 256, stream));
+  rc = pool_alloc(dev, (void**)&base, bx + by + 256, stream);
+  if (rc != B200SP_OK) return rc;
   auto done = [&](int code) { cudaFreeAsync(base, stream); cudaStreamSynchronize(stream); return code; };
   cudaError_t err = cudaSuccess;
   if (n > 0) err = cudaMemcpyAsync(base, x_host, (size_t)n * e, cudaMemcpyHostToDevice, stream);
@@ -373,6 +378,8 @@ void b200sp_cache_clear(void) {
   g_coo_cache.clear();
   for (auto& kv : g_csc_cache) csc_free(kv.second);
   g_csc_cache.clear();
+  for (DeviceInfo& d : g_dev)
+    if (d.pool) cudaMemPoolTrimTo(d.pool, 0);
 }
 
 const char* b200sp_status_string(int s) {
@@ -413,6 +420,7 @@ int b200sp_set_option(const char* name, int value) {
   if (!strcmp(name, "bstage_threads")) { if (value != 256 && value != 512 && value != 1024) return B200SP_ERR_INVALID_ARG; g_opt.bstage_threads = value; return B200SP_OK; }
   if (!strcmp(name, "bstage_nnz")) { if (value < 1024) return B200SP_ERR_INVALID_ARG; g_opt.bstage_nnz = value; return B200SP_OK; }
   if (!strcmp(name, "spmm_bstage")) { g_opt.spmm_bstage = value ? 1 : 0; return B200SP_OK; }
+  if (!strcmp(name, "pool_keep_mb")) { if (value < 0) return B200SP_ERR_INVALID_ARG; g_opt.pool_keep_mb = value; return B200SP_OK; }
   if (!strcmp(name, "spmm_sliced")) { g_opt.spmm_sliced = value ? 1 : 0; return B200SP_OK; }
   if (!strcmp(name, "merge_threads")) { if (value != 64 && value != 128 && value != 256) return B200SP_ERR_INVALID_ARG; g_opt.merge_threads = value; return B200SP_OK; }
   if (!strcmp(name, "sub_lanes")) { if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != 16 && value != 32) return B200SP_ERR_INVALID_ARG; g_opt.sub_lanes = value; return B200SP_OK; }

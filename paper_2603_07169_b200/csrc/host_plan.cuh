@@ -8,11 +8,25 @@ namespace {
 
 std::map<std::tuple<int, const void*, int64_t, int64_t, int64_t>, b200sp_plan*> g_cache;
 
-int plan_free(b200sp_plan* p) {
+// Frees a plan.  With stream_ordered the block goes back to the pool in the order of `stream` (the caller
+// knows that every kernel that used the plan ran there); otherwise the device is synchronised first.
+int plan_free(b200sp_plan* p, bool stream_ordered = false, cudaStream_t stream = nullptr) {
   if (!p) return B200SP_OK;
   int rc = B200SP_OK;
-  for (void* q : {(void*)p->split_row, (void*)p->carry, (void*)p->tail, (void*)p->spmm_split_row, (void*)p->long_rows})
-    if (q) { cudaError_t e = cudaFree(q); if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree"); }
+  if (p->block) {
+    cudaError_t e = cudaSuccess;
+    if (stream_ordered) {
+      e = cudaFreeAsync(p->block, stream);
+    } else {
+      int cur = 0;
+      e = cudaGetDevice(&cur);
+      if (e == cudaSuccess && cur != p->device) e = cudaSetDevice(p->device);
+      if (e == cudaSuccess) e = cudaDeviceSynchronize();
+      if (e == cudaSuccess) e = cudaFree(p->block);
+      if (cur != p->device) cudaSetDevice(cur);
+    }
+    if (e != cudaSuccess) rc = cuda_fail(e, "freeing a plan");
+  }
   delete p;
   return rc;
 }
@@ -34,12 +48,28 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   I.spmv_kernel = g_opt.spmv_kernel >= 0 ? g_opt.spmv_kernel : 0;
   if (m == 0) { *out = p; return B200SP_OK; }
 
-  PlanStats* d_stats = nullptr;
+  // one block from the pool: statistics, counter, split points, carries, tails, SpMM split points, long-row list
+  const size_t nt = (size_t)I.spmv_tiles, ns = (size_t)I.spmm_tiles;
+  const size_t long_cap = (size_t)(nnz / (kLongRow + 1)) + 1;     // rows longer than kLongRow: at most this many
+  auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+  const size_t o_stats = 0, o_count = o_stats + up(sizeof(PlanStats)), o_split = o_count + 256, o_carry = o_split + up((nt + 1) * 4),
+               o_tail = o_carry + up((nt + 1) * 4), o_msplit = o_tail + up((nt + 1) * 4), o_long = o_msplit + up((ns + 1) * 4),
+               total = o_long + up(long_cap * 4);
   PlanStats h = {};
   h.min_len = 0x7FFFFFFF;
-  auto fail = [&](int code) { if (d_stats) cudaFree(d_stats); plan_free(p); return code; };
+  auto fail = [&](int code) { plan_free(p, true, stream); cudaStreamSynchronize(stream); return code; };
 #define CUP(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail(cuda_fail(e_, #call)); } while (0)
-  CUP(cudaMalloc(&d_stats, sizeof(PlanStats)));
+  rc = pool_alloc(dev, &p->block, total, stream);
+  if (rc != B200SP_OK) { delete p; return rc; }
+  char* base = (char*)p->block;
+  PlanStats* d_stats = (PlanStats*)(base + o_stats);
+  int* d_count = (int*)(base + o_count);
+  p->split_row = (int32_t*)(base + o_split);
+  p->carry = (float*)(base + o_carry);
+  p->tail = (float*)(base + o_tail);
+  p->spmm_split_row = (int32_t*)(base + o_msplit);
+  p->long_rows = (int32_t*)(base + o_long);
+  I.scratch_bytes = (int64_t)total;
   CUP(cudaMemcpyAsync(d_stats, &h, sizeof h, cudaMemcpyHostToDevice, stream));
   {
     const int blocks = (int)((m + 256 * 8 - 1) / (256 * 8));
@@ -47,44 +77,30 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
     plan_stats_kernel<<<grid, 256, 0, stream>>>(row_ptr, (int)m, d_stats);
     g_launches++;
   }
-  const size_t nt = (size_t)I.spmv_tiles, ns = (size_t)I.spmm_tiles;
-  CUP(cudaMalloc(&p->split_row, (nt + 1) * sizeof(int32_t)));
-  CUP(cudaMalloc(&p->carry, (nt + 1) * sizeof(float)));
-  CUP(cudaMalloc(&p->tail, (nt + 1) * sizeof(float)));
-  CUP(cudaMalloc(&p->spmm_split_row, (ns + 1) * sizeof(int32_t)));
-  I.scratch_bytes = (int64_t)((nt + 1) * 12 + (ns + 1) * 4);
   plan_merge_split_kernel<<<(unsigned)((nt + 1 + 255) / 256), 256, 0, stream>>>(row_ptr, (int)m, (int)nnz, items, (int)nt, p->split_row);
   plan_nnz_split_kernel<<<(unsigned)((ns + 1 + 255) / 256), 256, 0, stream>>>(row_ptr, (int)m, (int)nnz, kSpmmTileNnz, (int)ns, p->spmm_split_row);
   g_launches += 2;
   CUP(cudaGetLastError());
   CUP(cudaMemcpyAsync(&h, d_stats, sizeof h, cudaMemcpyDeviceToHost, stream));
   CUP(cudaStreamSynchronize(stream));
-  CUP(cudaFree(d_stats));
-  d_stats = nullptr;
   if (!h.bad && h.bin_rows[4] > 0) {   // list of the rows in the last length bin (> kLongRow), sorted on the host
     const int cap = (int)h.bin_rows[4];
-    int* d_count = nullptr;
-    CUP(cudaMalloc(&p->long_rows, (size_t)cap * sizeof(int32_t)));
-    CUP(cudaMalloc(&d_count, sizeof(int)));
-    cudaError_t e = cudaMemsetAsync(d_count, 0, sizeof(int), stream);
-    if (e == cudaSuccess) {
-      const int blocks = (int)((m + 255) / 256);
-      plan_long_rows_kernel<<<blocks < dev->sms * 8 ? blocks : dev->sms * 8, 256, 0, stream>>>(row_ptr, (int)m, kLongRow, cap, p->long_rows, d_count);
-      g_launches++;
-      e = cudaGetLastError();
-    }
+    if ((size_t)cap > long_cap) return fail(B200SP_ERR_BAD_CSR);   // cannot happen for a monotone row_ptr
+    CUP(cudaMemsetAsync(d_count, 0, sizeof(int), stream));
+    const int blocks = (int)((m + 255) / 256);
+    plan_long_rows_kernel<<<blocks < dev->sms * 8 ? blocks : dev->sms * 8, 256, 0, stream>>>(row_ptr, (int)m, kLongRow, cap, p->long_rows, d_count);
+    g_launches++;
+    CUP(cudaGetLastError());
     std::vector<int32_t> tmp((size_t)cap);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(tmp.data(), p->long_rows, (size_t)cap * sizeof(int32_t), cudaMemcpyDeviceToHost, stream);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
-    if (e == cudaSuccess) { std::sort(tmp.begin(), tmp.end()); e = cudaMemcpyAsync(p->long_rows, tmp.data(), (size_t)cap * sizeof(int32_t), cudaMemcpyHostToDevice, stream); }
-    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
-    cudaFree(d_count);
-    if (e != cudaSuccess) return fail(cuda_fail(e, "plan long-row list"));
+    CUP(cudaMemcpyAsync(tmp.data(), p->long_rows, (size_t)cap * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    CUP(cudaStreamSynchronize(stream));
+    std::sort(tmp.begin(), tmp.end());
+    CUP(cudaMemcpyAsync(p->long_rows, tmp.data(), (size_t)cap * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+    CUP(cudaStreamSynchronize(stream));
     p->num_long = cap;
-    I.scratch_bytes += (int64_t)cap * 4;
   }
 #undef CUP
-  if (h.bad) { plan_free(p); return B200SP_ERR_BAD_CSR; }
+  if (h.bad) { plan_free(p, true, stream); cudaStreamSynchronize(stream); return B200SP_ERR_BAD_CSR; }
   I.min_row_len = h.min_len; I.max_row_len = h.max_len;
   for (int j = 0; j < B200SP_NUM_BINS; ++j) { I.bin_rows[j] = (int64_t)h.bin_rows[j]; I.bin_nnz[j] = (int64_t)h.bin_nnz[j]; }
   // Kernel choice from the row statistics: when every row is short and the mean is not far below the

@@ -62,6 +62,7 @@ struct Options {
   int merge_stride = 0;    // tile order of the scan merge kernel: stride through the tiles (0 / 1 = plain order)
   int merge_scan = 0;      // 1 = merge kernel with the in-register segmented scan, 0 = products through shared memory (default: as fast on power-law rows, faster on short rows)
   int merge_short = 32;    // rows up to this many products are added by one thread (8, 16, 32, 64)
+  int pool_keep_mb = 1024; // freed memory the library's pool keeps across synchronisation points, MiB (read when the pool is created)
   int merge_carve = 30;    // shared-memory carveout (percent) requested for it, -1 = leave to the driver
 } g_opt;
 
@@ -70,6 +71,7 @@ struct DeviceInfo {
   int cc_major = 0, sms = 0, persist_max = 0, window_max = 0, l2_bytes = 0;
   size_t persist_set = 0;
   int* err_flag = nullptr;  // device int: set by a kernel whose bounded wait ran out
+  cudaMemPool_t pool = nullptr;  // the library's own stream-ordered pool: plan scratch and the host entry points' staging buffers
 };
 DeviceInfo g_dev[64];
 
@@ -102,6 +104,40 @@ int device_info(DeviceInfo** out) {
   }
   *out = &d;
   return d.cc_major == 10 ? B200SP_OK : B200SP_ERR_ARCH;
+}
+
+// The library's own memory pool on this device.  It keeps up to "pool_keep_mb" of freed memory across
+// synchronisation points (the default pool of a device hands everything back at each of them, which makes
+// every allocation of the next call map fresh memory); b200sp_cache_clear trims it to nothing.
+int device_pool(DeviceInfo* d, cudaMemPool_t* out) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!d->pool) {
+    int dev = 0;
+    CU(cudaGetDevice(&dev));
+    cudaMemPoolProps props = {};
+    props.allocType = cudaMemAllocationTypePinned;
+    props.handleTypes = cudaMemHandleTypeNone;
+    props.location.type = cudaMemLocationTypeDevice;
+    props.location.id = dev;
+    cudaMemPool_t pool = nullptr;
+    CU(cudaMemPoolCreate(&pool, &props));
+    uint64_t keep = (uint64_t)(g_opt.pool_keep_mb < 0 ? 0 : g_opt.pool_keep_mb) << 20;
+    cudaError_t e = cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+    if (e != cudaSuccess) { cudaMemPoolDestroy(pool); return cuda_fail(e, "cudaMemPoolSetAttribute"); }
+    d->pool = pool;
+  }
+  *out = d->pool;
+  return B200SP_OK;
+}
+
+int pool_alloc(DeviceInfo* d, void** ptr, size_t bytes, cudaStream_t stream) {
+  cudaMemPool_t pool = nullptr;
+  int rc = device_pool(d, &pool);
+  if (rc != B200SP_OK) return rc;
+  cudaError_t e = cudaMallocFromPoolAsync(ptr, bytes, pool, stream);
+  if (e == cudaErrorMemoryAllocation) { (void)cudaGetLastError(); g_last_error = "out of device memory"; return B200SP_ERR_ALLOC; }
+  if (e != cudaSuccess) return cuda_fail(e, "cudaMallocFromPoolAsync");
+  return B200SP_OK;
 }
 
 // The flag that kernels with bounded waits raise; allocated on first use (those kernels only).
@@ -173,6 +209,7 @@ struct b200sp_plan {
   int device = 0;
   const int32_t* row_ptr = nullptr;
   b200sp_plan_info_t info = {};
+  void* block = nullptr;              // one allocation from the library's pool that holds every array below
   int32_t* split_row = nullptr;       // spmv tiles + 1
   float* carry = nullptr;             // spmv tiles
   float* tail = nullptr;              // spmv tiles
