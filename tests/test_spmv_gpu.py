@@ -302,3 +302,30 @@ def test_host_buffer_entry_point(dtype):
     b200sp.spmv_csr_vec_host(A.m, A.n, A.nnz, to_dev(A.row_ptr), to_dev(A.col_idx), to_dev(vals), x, y2, w.alpha, w.beta, dtype)
     assert_within(y2, y_ref, S, dtype)
     b200sp.b200sp_cache_clear()
+
+
+def test_library_pool_reuses_and_returns_memory():
+    """Repeated host-buffer calls and plan builds draw from the library's own pool: device memory in use does not grow
+    from call to call, results stay identical, and b200sp_cache_clear hands the pool's unused memory back."""
+    import torch
+    w = gen.workload("c2", scale_down=1)        # 2^18 rows, 4.2 M nonzeros: 38 MB of staging per call
+    A = w.A
+    y0 = w.y0.copy()
+    b200sp.b200sp_cache_clear()
+    torch.cuda.synchronize()
+    free_start = torch.cuda.mem_get_info()[0]
+    ys, frees = [], []
+    for _ in range(6):
+        y = y0.copy()
+        b200sp.spmv_csr_host(A.m, A.n, A.nnz, A.row_ptr, A.col_idx, A.vals, w.x, y, w.alpha, w.beta, "f32")
+        p = b200sp.b200sp_plan_create(A.m, A.n, A.nnz, to_dev(A.row_ptr))
+        b200sp.b200sp_plan_destroy(p)
+        ys.append(y)
+        frees.append(torch.cuda.mem_get_info()[0])
+    assert all(np.array_equal(ys[0], y) for y in ys[1:])
+    assert max(frees[1:]) - min(frees[1:]) <= (8 << 20)          # steady after the first call
+    assert free_start - frees[-1] >= (16 << 20)                  # the pool is holding the staging memory ...
+    b200sp.b200sp_cache_clear()
+    torch.cuda.empty_cache()
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] >= free_start - (8 << 20)    # ... and gives it back on request
