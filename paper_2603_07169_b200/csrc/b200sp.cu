@@ -356,7 +356,8 @@ int b200sp_validate_csr(int64_t m, int64_t n, int64_t nnz, const int32_t* row_pt
   cudaStream_t stream = (cudaStream_t)stream_v;
   int* d_bad = nullptr;
   int h_bad = 0;
-  CU(cudaMalloc(&d_bad, sizeof(int)));
+  rc = pool_alloc(dev, (void**)&d_bad, 256, stream);
+  if (rc != B200SP_OK) return rc;
   cudaError_t e = cudaMemsetAsync(d_bad, 0, sizeof(int), stream);
   if (e == cudaSuccess) {
     validate_csr_kernel<<<dev->sms * 8, 256, 0, stream>>>(row_ptr, col_idx, (int)m, (int)n, (int)nnz, d_bad);
@@ -364,8 +365,8 @@ int b200sp_validate_csr(int64_t m, int64_t n, int64_t nnz, const int32_t* row_pt
     e = cudaGetLastError();
   }
   if (e == cudaSuccess) e = cudaMemcpyAsync(&h_bad, d_bad, sizeof(int), cudaMemcpyDeviceToHost, stream);
+  cudaFreeAsync(d_bad, stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
-  cudaFree(d_bad);
   if (e != cudaSuccess) return cuda_fail(e, "b200sp_validate_csr");
   return h_bad ? B200SP_ERR_BAD_CSR : B200SP_OK;
 }

@@ -64,6 +64,7 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   char* base = (char*)p->block;
   PlanStats* d_stats = (PlanStats*)(base + o_stats);
   int* d_count = (int*)(base + o_count);
+  p->probe_out = (unsigned long long*)(base + o_count + 16);
   p->split_row = (int32_t*)(base + o_split);
   p->carry = (float*)(base + o_carry);
   p->tail = (float*)(base + o_tail);

@@ -215,6 +215,7 @@ struct b200sp_plan {
   float* tail = nullptr;              // spmv tiles
   int32_t* spmm_split_row = nullptr;  // spmm tiles + 1
   int32_t* long_rows = nullptr;       // rows longer than kLongRow, ascending
+  unsigned long long* probe_out = nullptr;  // two counters for the column-locality probe
   int num_long = 0;
   const void* probed_col_idx = nullptr;   // col_idx the column-locality probe last ran on
   bool cols_local = true;                 // its verdict: adjacent rows share most of their lines of x

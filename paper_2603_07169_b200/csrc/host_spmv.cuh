@@ -248,9 +248,9 @@ int run_spmv_subwarp(b200sp_plan* p, const int32_t* col_idx, const T* vals, cons
 int probe_col_locality(b200sp_plan* p, const int32_t* col_idx, cudaStream_t stream) {
   if (p->probed_col_idx == (const void*)col_idx) return B200SP_OK;
   const b200sp_plan_info_t& I = p->info;
-  unsigned long long* d_out = nullptr;
+  unsigned long long* d_out = p->probe_out;
   unsigned long long h[2] = {0, 0};
-  CU(cudaMalloc(&d_out, sizeof h));
+  if (!d_out) return B200SP_ERR_INVALID_ARG;
   cudaError_t e = cudaMemsetAsync(d_out, 0, sizeof h, stream);
   const int samples = I.m - 1 < 8192 ? (int)(I.m - 1) : 8192;
   if (e == cudaSuccess && samples > 0) {
@@ -260,7 +260,6 @@ int probe_col_locality(b200sp_plan* p, const int32_t* col_idx, cudaStream_t stre
   }
   if (e == cudaSuccess) e = cudaMemcpyAsync(h, d_out, sizeof h, cudaMemcpyDeviceToHost, stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
-  cudaFree(d_out);
   if (e != cudaSuccess) return cuda_fail(e, "column-locality probe");
   p->cols_local = h[1] == 0 || 2 * h[0] >= h[1];   // at least half of the sampled entries re-use a line of the row above
   p->probed_col_idx = col_idx;
