@@ -261,6 +261,7 @@ def workload(name: str, scale_down: int = 0) -> Workload:
     c3p the edges of c3 with every vertex renamed by one pseudo-random bijection (secondary measurement) (FP32)
     c4  27-point stencil 160^3, diag 26, off -1 + N(0, 0.01^2), x N(0,1)               (BF16)
     c5k64 / c5k256  m = n = 2^19, 32 nnz/row, vals N(0,1), B N(0,1) n x k              (FP32, BF16)
+    paper12_E / paper13_E  the paper's own SpMV / SpMM inputs: 2^E rows x 2048 columns at density 0.01 (K = 4096)
     """
     s = scale_down
     if name == "c1":
@@ -291,6 +292,13 @@ def workload(name: str, scale_down: int = 0) -> Workload:
         m = (1 << 19) >> (2 * s)
         A = uniform_rows(m, m, 32, 1005)
         return Workload(name, A, B=normal(m * k, 1005, 10), k=k, dtypes=("f32", "bf16"))
+    if name.startswith("paper12_") or name.startswith("paper13_"):
+        # the paper's own inputs (Table 6, tasks 12 / 13): rows = 2^e, 2048 columns, density 0.01, K = 4096 for SpMM
+        rows = 1 << int(name.split("_")[1])
+        k = 4096 if name.startswith("paper13_") else 0
+        A = paper_uniform(rows, 2048, 0.01, seed=rows + k)
+        return Workload(name, A, x=uniform(2048, -1.0, 1.0, 7, 1), B=(normal(2048 * k, 7, 2) if k else None), k=k,
+                        dtypes=("f32", "bf16"))
     raise ValueError("unknown workload %r" % name)
 
 

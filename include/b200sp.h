@@ -254,6 +254,8 @@ int64_t b200sp_launch_count(void);
  *   "sub_lanes"      lanes per row of the sub-warp kernel (1..32, power of two), 0 = from the mean row length (default)
  *   "bstage_threads" threads per CTA of the SpMM kernel with B in shared memory: 256, 512 or 1024 (default)
  *   "bstage_nnz"     nonzeros of A per CTA that kernel aims for, default 131072
+ *   "bstage_stage_a" 1 = its warps first copy their rows' (col, val) pairs into shared-memory buffers of their own (default),
+ *                    0 = the pairs are read from global memory inside the row loop
  *   "x_l2_window"    1 = pin x in L2 with a per-launch access-policy window, 0 = off (default: measured to give
  *                    nothing on large problems, where x stays in L2 anyway, and to cost 1.4 us per launch on tiny ones)
  *  memory

@@ -422,6 +422,7 @@ int b200sp_set_option(const char* name, int value) {
   if (!strcmp(name, "bstage_nnz")) { if (value < 1024) return B200SP_ERR_INVALID_ARG; g_opt.bstage_nnz = value; return B200SP_OK; }
   if (!strcmp(name, "spmm_bstage")) { g_opt.spmm_bstage = value ? 1 : 0; return B200SP_OK; }
   if (!strcmp(name, "pool_keep_mb")) { if (value < 0) return B200SP_ERR_INVALID_ARG; g_opt.pool_keep_mb = value; return B200SP_OK; }
+  if (!strcmp(name, "bstage_stage_a")) { g_opt.bstage_stage_a = value ? 1 : 0; return B200SP_OK; }
   if (!strcmp(name, "spmm_sliced")) { g_opt.spmm_sliced = value ? 1 : 0; return B200SP_OK; }
   if (!strcmp(name, "merge_threads")) { if (value != 64 && value != 128 && value != 256) return B200SP_ERR_INVALID_ARG; g_opt.merge_threads = value; return B200SP_OK; }
   if (!strcmp(name, "sub_lanes")) { if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != 16 && value != 32) return B200SP_ERR_INVALID_ARG; g_opt.sub_lanes = value; return B200SP_OK; }

@@ -56,6 +56,7 @@ struct Options {
   int merge_threads = 128; // threads per CTA of the one-tile-per-CTA merge kernel (128 or 256)
   int bstage_threads = 1024; // threads per CTA of that kernel (256, 512 or 1024)
   int bstage_nnz = 131072;   // nonzeros per CTA it aims for
+  int bstage_stage_a = 1;  // 1 = that kernel's warps copy their rows' (col, val) pairs into shared-memory buffers of their own (default), 0 = read them from global memory
   int spmm_bstage = 1;     // 1 = hold the slice of B in shared memory when A has few columns (default), 0 = never
   int spmm_sliced = 1;     // 1 = k-sliced SpMM kernel (default), 0 = one pass over all of k
   int sub_lanes = 0;       // lanes per row of the sub-warp kernel (0 = from the mean row length)

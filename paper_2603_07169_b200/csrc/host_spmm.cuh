@@ -43,7 +43,16 @@ int launch_spmm_bstage(b200sp_plan* p, int k, const int32_t* col_idx, const T* v
   constexpr int KS = LANES * VEC, ROW_BYTES = LANES * 16;
   const int box_rows = I.n < 256 ? (int)I.n : 256;
   const int boxes = (int)((I.n + box_rows - 1) / box_rows);
-  const size_t smem = (size_t)boxes * box_rows * ROW_BYTES;
+  const size_t bslice = (((size_t)boxes * box_rows * ROW_BYTES) + 127) & ~(size_t)127;
+  // what the slice of B leaves of the SM's shared memory is split among the warps as staging buffers for their (col, val) pairs
+  const size_t limit = (size_t)kSmemPerSm - 2048;
+  int capw = 0;
+  if (g_opt.bstage_stage_a && bslice < limit) {
+    const size_t per_warp = (limit - bslice) / (THREADS / 32);
+    const long long entries = (long long)(per_warp / (4 + sizeof(T))) & ~7LL;
+    if (entries >= 72) capw = (int)(entries > 4096 ? 4096 : entries) - 4;
+  }
+  const size_t smem = bslice + (capw > 0 ? (size_t)(THREADS / 32) * (capw + 4) * (4 + sizeof(T)) : 0);
   CUtensorMap map;
   const cuuint64_t gdim[2] = {(cuuint64_t)k, (cuuint64_t)I.n};
   const cuuint64_t gstride[1] = {(cuuint64_t)k * sizeof(T)};
@@ -71,7 +80,7 @@ int launch_spmm_bstage(b200sp_plan* p, int k, const int32_t* col_idx, const T* v
   int rc = ensure_err_flag(dev);
   if (rc != B200SP_OK) return rc;
   return launch_smem(kernel, dim3((unsigned)(slices * row_chunks)), dim3(THREADS), smem, stream, nullptr, 0, dev, map, (int)I.m, (int)I.n,
-                     k, row_chunks, rows_per_chunk, box_rows, p->row_ptr, col_idx, vals, Y, alpha, beta, dev->err_flag);
+                     k, row_chunks, rows_per_chunk, box_rows, (int)bslice, capw, p->row_ptr, col_idx, vals, Y, alpha, beta, dev->err_flag);
 }
 
 template <typename T, int VEC>

@@ -8,6 +8,13 @@
 // groups of LANES lanes walk their rows of A and read B from shared memory (about an order of magnitude
 // more gathers per clock than the L1-miss path), keeping VEC columns per lane in FP32 registers.  B is read
 // from L2 / HBM once per (slice, row chunk) instead of once per nonzero.
+//
+// The (col, val) pairs of A go through shared memory too: a warp's 32 / LANES groups own consecutive rows,
+// whose nonzeros are contiguous, so the warp first copies that range with coalesced loads into a buffer of
+// its own (capw entries, carved from the shared memory the slice of B leaves) and the groups then read their
+// pairs from there.  Read directly, the same pairs cost one L1 wavefront per group and request -- 40 % of the
+// L1 data pipe this kernel is bound by.  No CTA-wide barrier is involved: warps stay independent.  A set of
+// rows that does not fit the buffer (or capw = 0) is read from global memory as before.
 #pragma once
 #include <cuda.h>
 
@@ -25,12 +32,28 @@ template <typename T> struct RawFromSmem;
 template <> struct RawFromSmem<float> { typedef float4 type; };
 template <> struct RawFromSmem<bf16_t> { typedef uint4 type; };
 
+// four consecutive (col, val) pairs from a shared-memory buffer (index a multiple of 4)
+__device__ __forceinline__ void lds_a4(const int* col_s, const float* val_s, int q, int (&c)[4], float (&v)[4]) {
+  const int4 cc = *(const int4*)(col_s + q);
+  const float4 vv = *(const float4*)(val_s + q);
+  c[0] = cc.x; c[1] = cc.y; c[2] = cc.z; c[3] = cc.w; v[0] = vv.x; v[1] = vv.y; v[2] = vv.z; v[3] = vv.w;
+}
+__device__ __forceinline__ void lds_a4(const int* col_s, const bf16_t* val_s, int q, int (&c)[4], float (&v)[4]) {
+  const int4 cc = *(const int4*)(col_s + q);
+  const uint2 vv = *(const uint2*)(val_s + q);
+  c[0] = cc.x; c[1] = cc.y; c[2] = cc.z; c[3] = cc.w;
+  v[0] = __uint_as_float(vv.x << 16); v[1] = __uint_as_float(vv.x & 0xFFFF0000u);
+  v[2] = __uint_as_float(vv.y << 16); v[3] = __uint_as_float(vv.y & 0xFFFF0000u);
+}
+
+// Dynamic shared memory: [ slice of B: bslice_bytes | per warp: (capw + 4) ints, (capw + 4) values ]; capw + 4 is a multiple of 8.
 template <typename T, int VEC, int LANES, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 spmm_bstage_kernel(const __grid_constant__ CUtensorMap tmapB, int m, int n, int k, int row_chunks, int rows_per_chunk, int box_rows,
-                   const int* __restrict__ row_ptr, const int* __restrict__ col_idx, const T* __restrict__ vals, T* __restrict__ Y,
-                   float alpha, float beta, int* __restrict__ err) {
-  constexpr int GROUPS = THREADS / LANES, KS = LANES * VEC, ROW_BYTES = LANES * 16;
+                   int bslice_bytes, int capw, const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
+                   const T* __restrict__ vals, T* __restrict__ Y, float alpha, float beta, int* __restrict__ err) {
+  constexpr int KS = LANES * VEC, ROW_BYTES = LANES * 16, GPW = 32 / LANES, WARPS = THREADS / 32;
+  constexpr unsigned FULL = 0xFFFFFFFFu;
   typedef typename RawVec<T, VEC>::type raw_t;
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ __align__(8) unsigned long long bar;
@@ -51,36 +74,76 @@ spmm_bstage_kernel(const __grid_constant__ CUtensorMap tmapB, int m, int n, int 
     (void)mbar_wait_bounded(smem_addr(&bar), 0);   // bounded second chance for the copies in flight
     return;
   }
-  const int g = tid / LANES, l = tid % LANES;
+  const int warp = tid >> 5, lane = tid & 31;
+  const int gl = lane / LANES, l = lane % LANES;     // group inside the warp, lane inside the group
   const int col0 = col_base + l * VEC;
   const bool active = col0 < k;
   const unsigned char* Bs = smem + l * 16;
+  const int entries = capw + 4;
+  int* wcol = (int*)(smem + bslice_bytes + (size_t)warp * entries * (4 + sizeof(T)));
+  T* wval = (T*)(wcol + entries);
   const int r_begin = chunk * rows_per_chunk;
   const int r_end = min(m, r_begin + rows_per_chunk);
-  for (int row = r_begin + g; row < r_end; row += GROUPS) {
-    const int rs = __ldg(row_ptr + row), re = __ldg(row_ptr + row + 1);
+  for (int rb = r_begin + warp * GPW; rb < r_end; rb += WARPS * GPW) {   // GPW consecutive rows per warp and step
+    int bound = 0;
+    if (lane <= GPW) bound = __ldg(row_ptr + min(rb + lane, r_end));     // rows past the chunk's end come out empty
+    const int a = __shfl_sync(FULL, bound, 0), b_end = __shfl_sync(FULL, bound, GPW);
+    const int rs = __shfl_sync(FULL, bound, gl), re = __shfl_sync(FULL, bound, gl + 1);
+    const int row = rb + gl;
     float acc[VEC];
 #pragma unroll
     for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
-    int p = rs;
-    for (; p < re && (p & 3); ++p) {
-      const raw_t b = *(const raw_t*)(Bs + (size_t)__ldg(col_idx + p) * ROW_BYTES);
-      RawVec<T, VEC>::fma(b, to_f32(__ldg(vals + p)), acc);
-    }
-    for (; p + 4 <= re; p += 4) {
-      int c[4]; float v[4];
-      ld_a4(col_idx, vals, p, c, v);
-      raw_t b[4];
+    if (capw > 0 && b_end - a <= capw) {
+      // ---- the warp's nonzeros [a, b_end) into its buffer; entry p sits at p - (a & ~3), so p & 3 is kept
+      const int a4 = a & ~3;
+      __syncwarp();                      // the previous step's readers are done with the buffer
+#pragma unroll 4
+      for (int p = a + lane; p < b_end; p += 32) {
+        wcol[p - a4] = __ldg(col_idx + p);
+        wval[p - a4] = __ldg(vals + p);
+      }
+      __syncwarp();
+      int q = rs - a4;
+      const int qe = re - a4;
+      for (; q < qe && (q & 3); ++q) {
+        const raw_t b = *(const raw_t*)(Bs + (size_t)wcol[q] * ROW_BYTES);
+        RawVec<T, VEC>::fma(b, to_f32(wval[q]), acc);
+      }
+      for (; q + 4 <= qe; q += 4) {
+        int c[4]; float v[4];
+        lds_a4(wcol, wval, q, c, v);   // (one pair per lane plus shuffles round the group was measured slower: 2.26 against 1.86 ms)
+        raw_t b[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) b[u] = *(const raw_t*)(Bs + (size_t)c[u] * ROW_BYTES);
+        for (int u = 0; u < 4; ++u) b[u] = *(const raw_t*)(Bs + (size_t)c[u] * ROW_BYTES);
 #pragma unroll
-      for (int u = 0; u < 4; ++u) RawVec<T, VEC>::fma(b[u], v[u], acc);
+        for (int u = 0; u < 4; ++u) RawVec<T, VEC>::fma(b[u], v[u], acc);
+      }
+      for (; q < qe; ++q) {
+        const raw_t b = *(const raw_t*)(Bs + (size_t)wcol[q] * ROW_BYTES);
+        RawVec<T, VEC>::fma(b, to_f32(wval[q]), acc);
+      }
+    } else {
+      // ---- too many nonzeros for the buffer: pairs straight from global memory
+      int p = rs;
+      for (; p < re && (p & 3); ++p) {
+        const raw_t b = *(const raw_t*)(Bs + (size_t)__ldg(col_idx + p) * ROW_BYTES);
+        RawVec<T, VEC>::fma(b, to_f32(__ldg(vals + p)), acc);
+      }
+      for (; p + 4 <= re; p += 4) {
+        int c[4]; float v[4];
+        ld_a4(col_idx, vals, p, c, v);
+        raw_t b[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) b[u] = *(const raw_t*)(Bs + (size_t)c[u] * ROW_BYTES);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) RawVec<T, VEC>::fma(b[u], v[u], acc);
+      }
+      for (; p < re; ++p) {
+        const raw_t b = *(const raw_t*)(Bs + (size_t)__ldg(col_idx + p) * ROW_BYTES);
+        RawVec<T, VEC>::fma(b, to_f32(__ldg(vals + p)), acc);
+      }
     }
-    for (; p < re; ++p) {
-      const raw_t b = *(const raw_t*)(Bs + (size_t)__ldg(col_idx + p) * ROW_BYTES);
-      RawVec<T, VEC>::fma(b, to_f32(__ldg(vals + p)), acc);
-    }
-    if (active) {
+    if (active && row < r_end) {
       T* yp = Y + (long long)row * k + col0;
       float out[VEC];
       if (beta != 0.0f) {
