@@ -24,14 +24,17 @@ spmv_uniform_vec_kernel(long long quads, const int* __restrict__ col_idx, const 
   for (; g < quads; g += stride * UNROLL) {
     int4 c[UNROLL];
     float v[UNROLL][4];
+    float yold[UNROLL];
     bool ok[UNROLL];
 #pragma unroll
     for (int u = 0; u < UNROLL; ++u) {
       const long long q = g + (long long)u * stride;
       ok[u] = q < quads;
+      yold[u] = 0.0f;
       if (ok[u]) {
         c[u] = ld_stream_i4(col_idx + q * 4);
         ld_stream_vals4(vals + q * 4, v[u]);
+        if (beta != 0.0f && (q & (LPR - 1)) == 0) yold[u] = to_f32(y[q / LPR]);   // asked for now: its latency overlaps the gathers
       }
     }
     float part[UNROLL];
@@ -50,7 +53,11 @@ spmv_uniform_vec_kernel(long long quads, const int* __restrict__ col_idx, const 
       float s = part[u];
 #pragma unroll
       for (int o = 1; o < LPR; o <<= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-      if (ok[u] && (q & (LPR - 1)) == 0) epilogue_store(y, q / LPR, s, alpha, beta);
+      if (ok[u] && (q & (LPR - 1)) == 0) {
+        float r = alpha * s;
+        if (beta != 0.0f) r += beta * yold[u];
+        store_elem(y + q / LPR, r);
+      }
     }
   }
 }
