@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes (read + write) per launch of the dominant kernel from an ncu capture, keyed by
 # (workload, dtype); None where no capture has been made.  Sources: the summaries under profiles/.
 NCU_TRAFFIC_BYTES = {
-    ("c2", "f32"): 147_020_288,     # profiles/spmv_uniform_vec_c2_f32.md
+    ("c2", "f32"): 148_018_944,     # profiles/spmv_uniform_vec_c2_f32.md
     ("c2", "bf16"): 109_364_736,    # profiles/spmv_uniform_vec_c2_bf16.md
     ("c3", "f32"): 305_818_112,     # profiles/spmv_merge_tile_c3_f32.md
     ("c4", "bf16"): 690_968_832,    # profiles/spmv_row_tile_c4_bf16.md

@@ -434,7 +434,7 @@ int b200sp_set_option(const char* name, int value) {
   if (!strcmp(name, "merge_items")) { if (value != 1024 && value != 2048 && value != 4096) return B200SP_ERR_INVALID_ARG; g_opt.merge_items = value; return B200SP_OK; }
   if (!strcmp(name, "merge_stages")) { if (value < 2 || value > kMergeMaxStages) return B200SP_ERR_INVALID_ARG; g_opt.merge_stages = value; return B200SP_OK; }
   if (!strcmp(name, "merge_ctas")) { if (value < 1 || value > 8) return B200SP_ERR_INVALID_ARG; g_opt.merge_ctas = value; return B200SP_OK; }
-  if (!strcmp(name, "uni_unroll")) { if (value != 1 && value != 2 && value != 4) return B200SP_ERR_INVALID_ARG; g_opt.uni_unroll = value; return B200SP_OK; }
+  if (!strcmp(name, "uni_unroll")) { if (value != 0 && value != 1 && value != 2 && value != 4) return B200SP_ERR_INVALID_ARG; g_opt.uni_unroll = value; return B200SP_OK; }
   if (!strcmp(name, "uni_ctas")) { if (value < 0 || value > 32) return B200SP_ERR_INVALID_ARG; g_opt.uni_ctas = value; return B200SP_OK; }
   if (!strcmp(name, "spmv_kernel")) { if (value < -1 || value > 3) return B200SP_ERR_INVALID_ARG; g_opt.spmv_kernel = value; return B200SP_OK; }
   if (!strcmp(name, "x_l2_window")) { g_opt.x_l2_window = value ? 1 : 0; return B200SP_OK; }
