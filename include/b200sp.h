@@ -236,7 +236,7 @@ int64_t b200sp_launch_count(void);
  *  merge-tile SpMV kernel
  *   "merge_items"    merge items per tile: 1024, 2048 (default) or 4096
  *   "merge_threads"  threads per CTA: 64, 128 (default) or 256
- *   "merge_carve"    shared-memory carveout in percent requested for it, default 30 (-1 = leave to the driver)
+ *   "merge_carve"    shared-memory carveout in percent requested for it, default 45 (-1 = leave to the driver)
  *   "merge_short"    rows of up to this many products are added by one thread: 8, 16, 32 (default) or 64
  *   "merge_scan"     1 = reduce rows with an in-register segmented scan, 0 = products through shared memory (default)
  *   "merge_stride"   with merge_scan: walk the tiles with this stride (made coprime to their number), 0 = in order

@@ -64,7 +64,7 @@ struct Options {
   int merge_scan = 0;      // 1 = merge kernel with the in-register segmented scan, 0 = products through shared memory (default: as fast on power-law rows, faster on short rows)
   int merge_short = 32;    // rows up to this many products are added by one thread (8, 16, 32, 64)
   int pool_keep_mb = 1024; // freed memory the library's pool keeps across synchronisation points, MiB (read when the pool is created)
-  int merge_carve = 30;    // shared-memory carveout (percent) requested for it, -1 = leave to the driver
+  int merge_carve = 45;    // shared-memory carveout (percent) requested for it, -1 = leave to the driver
 } g_opt;
 
 struct DeviceInfo {
