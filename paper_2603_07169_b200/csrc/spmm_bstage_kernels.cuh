@@ -107,7 +107,7 @@ spmm_bstage_kernel(const __grid_constant__ CUtensorMap tmapB, int m, int n, int 
       const int qe = re - a4;
       for (; q < qe && (q & 3); ++q) {
         const raw_t b = *(const raw_t*)(Bs + (size_t)wcol[q] * ROW_BYTES);
-        RawVec<T, VEC>::fma(b, to_f32(wval[q]), acc);
+        RawVec<T, VEC>::fma_mixed(b, to_f32(wval[q]), acc);
       }
       for (; q + 4 <= qe; q += 4) {
         int c[4]; float v[4];
@@ -116,18 +116,18 @@ spmm_bstage_kernel(const __grid_constant__ CUtensorMap tmapB, int m, int n, int 
 #pragma unroll
         for (int u = 0; u < 4; ++u) b[u] = *(const raw_t*)(Bs + (size_t)c[u] * ROW_BYTES);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) RawVec<T, VEC>::fma(b[u], v[u], acc);
+        for (int u = 0; u < 4; ++u) RawVec<T, VEC>::fma_mixed(b[u], v[u], acc);
       }
       for (; q < qe; ++q) {
         const raw_t b = *(const raw_t*)(Bs + (size_t)wcol[q] * ROW_BYTES);
-        RawVec<T, VEC>::fma(b, to_f32(wval[q]), acc);
+        RawVec<T, VEC>::fma_mixed(b, to_f32(wval[q]), acc);
       }
     } else {
       // ---- too many nonzeros for the buffer: pairs straight from global memory
       int p = rs;
       for (; p < re && (p & 3); ++p) {
         const raw_t b = *(const raw_t*)(Bs + (size_t)__ldg(col_idx + p) * ROW_BYTES);
-        RawVec<T, VEC>::fma(b, to_f32(__ldg(vals + p)), acc);
+        RawVec<T, VEC>::fma_mixed(b, to_f32(__ldg(vals + p)), acc);
       }
       for (; p + 4 <= re; p += 4) {
         int c[4]; float v[4];
@@ -136,11 +136,11 @@ spmm_bstage_kernel(const __grid_constant__ CUtensorMap tmapB, int m, int n, int 
 #pragma unroll
         for (int u = 0; u < 4; ++u) b[u] = *(const raw_t*)(Bs + (size_t)c[u] * ROW_BYTES);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) RawVec<T, VEC>::fma(b[u], v[u], acc);
+        for (int u = 0; u < 4; ++u) RawVec<T, VEC>::fma_mixed(b[u], v[u], acc);
       }
       for (; p < re; ++p) {
         const raw_t b = *(const raw_t*)(Bs + (size_t)__ldg(col_idx + p) * ROW_BYTES);
-        RawVec<T, VEC>::fma(b, to_f32(__ldg(vals + p)), acc);
+        RawVec<T, VEC>::fma_mixed(b, to_f32(__ldg(vals + p)), acc);
       }
     }
     if (active && row < r_end) {
