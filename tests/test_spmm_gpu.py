@@ -51,6 +51,18 @@ def test_long_rows_and_both_kernels(sliced, dtype):
         b200sp.b200sp_set_option("spmm_sliced", 1)
 
 
+@pytest.mark.parametrize("k", [64, 256])
+def test_longest_sequential_rows_positive_data(k):
+    """Rows of exactly 1024 nonzeros are the longest that one lane group adds in sequence; with all-positive data nothing
+    cancels, so this is the case that comes closest to the FP32 bound (chain bound 1024 * 2^-24 * S; measured 0.2-0.25 of 1e-5 * S)."""
+    rng = np.random.default_rng(5)
+    A = gen.random_csr(400, 4000, np.full(400, 1024), seed=1024)
+    A.vals[:] = rng.random(A.nnz).astype(np.float32) + 0.01
+    B = rng.random(4000 * k).astype(np.float32) + 0.01
+    Y, Y_ref, S = run_spmm(A, B, k, None, 1.0, 0.0, "f32")
+    assert assert_within(Y, Y_ref, S, "f32", what="1024-term rows, positive data") < 0.5
+
+
 @pytest.mark.parametrize("dtype", DTYPES)
 @pytest.mark.parametrize("n,k", [(2048, 4096), (2048, 40), (1500, 72), (300, 264), (5000, 64), (100, 8)])
 def test_b_slice_in_shared_memory(n, k, dtype):
