@@ -28,6 +28,10 @@
  *    hundred bytes and synchronises the stream once).
  *  - beta == 0: y / Y is write-only (its old contents, NaN included, are ignored).  alpha == 0 or
  *    nnz == 0: y = beta * y without reading A.  m == 0: nothing is done.  x / B must not alias y / Y.
+ *  - The compute kernels are launched with programmatic stream serialisation (option "pdl"): a kernel waits for the
+ *    stream's earlier work (griddepcontrol.wait) before its first memory access, then lets the next kernel of the
+ *    stream be scheduled behind it.  Ordinary launches that follow see ordinary stream order.  A caller that launches
+ *    its own next kernel with the same attribute must call cudaGridDependencySynchronize() in it before reading y / Y.
  *  - Results are deterministic: the same inputs give bit-identical outputs on every call (no
  *    floating-point atomics; rows cut by a tile boundary are completed in a fixed order).
  *  - Errors: host-detectable problems (negative or too large sizes, NULL pointer with non-zero
@@ -258,6 +262,10 @@ int64_t b200sp_launch_count(void);
  *                    0 = the pairs are read from global memory inside the row loop
  *   "x_l2_window"    1 = pin x in L2 with a per-launch access-policy window, 0 = off (default: measured to give
  *                    nothing on large problems, where x stays in L2 anyway, and to cost 1.4 us per launch on tiny ones)
+ *  launch
+ *   "pdl"            1 = the SpMV and SpMM kernels are launched with programmatic stream serialisation (default): each begins
+ *                    with griddepcontrol.wait, so it may be scheduled while the stream's previous kernel drains and touches no
+ *                    memory before that kernel has completed; 0 = plain stream order
  *  memory
  *   "pool_keep_mb"   MiB of freed memory the library's pool keeps across synchronisation points, default 1024
  *                    (read when a device's pool is created, i.e. before the first call that allocates on it)

@@ -421,6 +421,7 @@ int b200sp_set_option(const char* name, int value) {
   if (!strcmp(name, "bstage_threads")) { if (value != 256 && value != 512 && value != 1024) return B200SP_ERR_INVALID_ARG; g_opt.bstage_threads = value; return B200SP_OK; }
   if (!strcmp(name, "bstage_nnz")) { if (value < 1024) return B200SP_ERR_INVALID_ARG; g_opt.bstage_nnz = value; return B200SP_OK; }
   if (!strcmp(name, "spmm_bstage")) { g_opt.spmm_bstage = value ? 1 : 0; return B200SP_OK; }
+  if (!strcmp(name, "pdl")) { g_opt.pdl = value ? 1 : 0; return B200SP_OK; }
   if (!strcmp(name, "pool_keep_mb")) { if (value < 0) return B200SP_ERR_INVALID_ARG; g_opt.pool_keep_mb = value; return B200SP_OK; }
   if (!strcmp(name, "bstage_stage_a")) { g_opt.bstage_stage_a = value ? 1 : 0; return B200SP_OK; }
   if (!strcmp(name, "spmm_sliced")) { g_opt.spmm_sliced = value ? 1 : 0; return B200SP_OK; }

@@ -56,6 +56,14 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// For kernels launched with programmatic stream serialisation: wait until every earlier kernel of the stream has
+// completed and its writes are visible, then allow the next such kernel to be scheduled behind this one.  Without
+// that launch attribute both instructions do nothing.
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;");
+}
+
 // y = alpha * acc + beta * y0 with the BLAS rule that beta == 0 never reads y0.
 template <typename T>
 __device__ __forceinline__ void epilogue_store(T* y, long long i, float acc, float alpha, float beta) {

@@ -63,6 +63,7 @@ struct Options {
   int merge_stride = 0;    // tile order of the scan merge kernel: stride through the tiles (0 / 1 = plain order)
   int merge_scan = 0;      // 1 = merge kernel with the in-register segmented scan, 0 = products through shared memory (default: as fast on power-law rows, faster on short rows)
   int merge_short = 32;    // rows up to this many products are added by one thread (8, 16, 32, 64)
+  int pdl = 1;             // 1 = launch the kernels that begin with griddepcontrol.wait with programmatic stream serialisation
   int pool_keep_mb = 1024; // freed memory the library's pool keeps across synchronisation points, MiB (read when the pool is created)
   int merge_carve = 45;    // shared-memory carveout (percent) requested for it, -1 = leave to the driver
 } g_opt;
@@ -151,6 +152,8 @@ int ensure_err_flag(DeviceInfo* d) {
   return B200SP_OK;
 }
 
+thread_local bool tl_pdl_kernel = false;   // set by a launcher whose kernel begins with griddepcontrol.wait; consumed by the next launch
+
 // Launch with an optional L2 access-policy window (persisting hits) over the gathered operand.
 template <typename... KArgs, typename... Args>
 int launch_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, const void* win_ptr,
@@ -160,7 +163,7 @@ int launch_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cu
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   cfg.attrs = attr;
   cfg.numAttrs = 0;
   if (win_ptr && win_bytes && g_opt.x_l2_window && dev->persist_max > 0 && dev->window_max > 0) {
@@ -183,6 +186,14 @@ int launch_smem(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cu
       cfg.numAttrs = 1;
     }
   }
+  if (tl_pdl_kernel && g_opt.pdl) {
+    // programmatic dependent launch: the kernel starts with griddepcontrol.wait, so it may be scheduled while the
+    // previous kernel of the stream drains; nothing of it touches memory before that kernel has completed
+    attr[cfg.numAttrs].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[cfg.numAttrs].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs++;
+  }
+  tl_pdl_kernel = false;
   CU(cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...));
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return B200SP_OK;

@@ -79,6 +79,7 @@ int launch_spmm_bstage(b200sp_plan* p, int k, const int32_t* col_idx, const T* v
   if ((long long)slices * row_chunks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
   int rc = ensure_err_flag(dev);
   if (rc != B200SP_OK) return rc;
+  tl_pdl_kernel = true;
   return launch_smem(kernel, dim3((unsigned)(slices * row_chunks)), dim3(THREADS), smem, stream, nullptr, 0, dev, map, (int)I.m, (int)I.n,
                      k, row_chunks, rows_per_chunk, box_rows, (int)bslice, capw, p->row_ptr, col_idx, vals, Y, alpha, beta, dev->err_flag);
 }
@@ -117,10 +118,12 @@ int run_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const
     const int slices = (k + KS - 1) / KS;
     const int row_blocks = (int)((I.m + GROUPS - 1) / GROUPS);
     if ((long long)slices * row_blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+    tl_pdl_kernel = true;
     int rc = launch(spmm_slice_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)(slices * row_blocks)), dim3(kSpmmThreads), stream,
                     nullptr, 0, dev,
                     (int)I.m, k, row_blocks, p->row_ptr, col_idx, vals, B, Y, alpha, beta, kLongRow);
     if (rc != B200SP_OK || p->num_long == 0) return rc;
+    tl_pdl_kernel = true;
     return launch(spmm_long_row_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)(slices * p->num_long)), dim3(kSpmmThreads), stream, nullptr, 0,
                   dev, k, p->num_long, (const int*)p->long_rows, p->row_ptr, col_idx, vals, B, Y, alpha, beta);
   }

@@ -51,6 +51,7 @@ int launch_row_direct(b200sp_plan* p, const int32_t* col_idx, const T* vals, con
   const int grid = tiles < ctas * dev->sms ? tiles : ctas * dev->sms;
   const int rc_flag = ensure_err_flag(dev);
   if (rc_flag != B200SP_OK) return rc_flag;
+  tl_pdl_kernel = true;
   return launch_smem(kernel, dim3(grid), dim3(THREADS), smem, stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz,
                      p->row_ptr, col_idx, vals, x, y, alpha, beta, R, cap, tiles, stages, rot_lanes, dev->err_flag, 0);
 }
@@ -86,6 +87,7 @@ int launch_row_direct_ell(int64_t m, int width, const int32_t* col_ids, const T*
   const int grid = tiles < ctas * dev->sms ? tiles : ctas * dev->sms;
   const int rc_flag = ensure_err_flag(dev);
   if (rc_flag != B200SP_OK) return rc_flag;
+  tl_pdl_kernel = true;
   return launch_smem(kernel, dim3(grid), dim3(THREADS), smem, stream, nullptr, 0, dev, (int)m, (int)(m * width), (const int*)nullptr, col_ids,
                      vals, x, y, alpha, beta, R, cap, tiles, stages, 0, dev->err_flag, width);
 }
@@ -130,6 +132,7 @@ int launch_uniform(b200sp_plan* p, const int32_t* col_idx, const T* vals, const 
   long long blocks = (quads + (long long)THREADS * UNROLL - 1) / ((long long)THREADS * UNROLL);
   const long long cap = (long long)dev->sms * ctas;
   if (blocks > cap) blocks = cap;
+  tl_pdl_kernel = true;
   return launch(kernel, dim3((unsigned)blocks), dim3(THREADS), stream, x, (size_t)I.n * sizeof(T), dev, quads, col_idx, vals, x, y, alpha, beta);
 }
 
@@ -194,23 +197,28 @@ int run_spmv_merge(b200sp_plan* p, const int32_t* col_idx, const T* vals, const 
   } else if (g_opt.merge_threads == 64) {
     auto kernel = spmv_merge_tile_kernel<T, ITEMS, 64, SHORT>;
     if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
+    tl_pdl_kernel = true;
     rc = launch(kernel, dim3(tiles), dim3(64), stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx,
                 vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail);
   } else if (g_opt.merge_threads == 128) {
     auto kernel = spmv_merge_tile_kernel<T, ITEMS, 128, SHORT>;
     if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
+    tl_pdl_kernel = true;
     rc = launch(kernel, dim3(tiles), dim3(128), stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx,
                 vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail);
   } else {
     auto kernel = spmv_merge_tile_kernel<T, ITEMS, kThreads, kShortMax>;
     if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
+    tl_pdl_kernel = true;
     rc = launch(kernel, dim3(tiles), dim3(kThreads), stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx,
                 vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail);
   }
   if (rc != B200SP_OK) return rc;
-  if (tiles > 1)
+  if (tiles > 1) {
+    tl_pdl_kernel = true;
     rc = launch(spmv_carry_fixup_kernel<T, ITEMS>, dim3((tiles + 127) / 128), dim3(128), stream, nullptr, 0, dev, tiles,
                 p->row_ptr, (const int*)p->split_row, (const float*)p->carry, (const float*)p->tail, y, alpha, beta);
+  }
   return rc;
 }
 
@@ -222,6 +230,7 @@ int launch_subwarp(b200sp_plan* p, const int32_t* col_idx, const T* vals, const 
   const long long groups_per_cta = THREADS / LPR;
   const long long blocks = (I.m + groups_per_cta - 1) / groups_per_cta;
   if (blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+  tl_pdl_kernel = true;
   return launch(spmv_subwarp_kernel<T, LPR, THREADS>, dim3((unsigned)blocks), dim3(THREADS), stream, x, (size_t)I.n * sizeof(T), dev,
                 (int)I.m, p->row_ptr, col_idx, vals, x, y, alpha, beta);
 }

@@ -62,6 +62,7 @@ spmm_bstage_kernel(const __grid_constant__ CUtensorMap tmapB, int m, int n, int 
   const int col_base = slice * KS;
   if (tid == 0) { mbar_init(smem_addr(&bar), 1); mbar_init_fence(); }
   __syncthreads();
+  grid_dependency_wait();   // nothing above touches global memory
   if (tid == 0) {
     const int boxes = (n + box_rows - 1) / box_rows;
     mbar_arrive_expect_tx(smem_addr(&bar), (unsigned)boxes * (unsigned)box_rows * ROW_BYTES);   // rows past n are zero-filled and still counted

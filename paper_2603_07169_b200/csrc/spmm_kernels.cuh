@@ -184,6 +184,7 @@ spmm_slice_kernel(int m, int k, int row_blocks, const int* __restrict__ row_ptr,
                   const T* __restrict__ vals, const T* __restrict__ B, T* __restrict__ Y, float alpha, float beta, int long_thresh) {
   constexpr int LANES = 8, GROUPS = THREADS / LANES, KS = LANES * VEC;
   typedef typename RawVec<T, VEC>::type raw_t;
+  grid_dependency_wait();
   const int slice = blockIdx.x / row_blocks, rb = blockIdx.x - slice * row_blocks;
   const int g = threadIdx.x / LANES, l8 = threadIdx.x % LANES;
   const long long row = (long long)rb * GROUPS + g;
@@ -237,6 +238,7 @@ spmm_long_row_kernel(int k, int num_long, const int* __restrict__ long_rows, con
                      float alpha, float beta) {
   constexpr int LANES = 8, GROUPS = THREADS / LANES, KS = LANES * VEC;
   __shared__ float part[GROUPS][KS];
+  grid_dependency_wait();
   const int slice = blockIdx.x / num_long;
   const long long row = long_rows[blockIdx.x - slice * num_long];
   const int g = threadIdx.x / LANES, l8 = threadIdx.x % LANES;

@@ -32,6 +32,7 @@ spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const in
   __shared__ int2 long_span[MAX_LONG];      // its products: local [first, last)
   __shared__ int n_long;
 
+  grid_dependency_wait();
   const int tid = threadIdx.x;
   const int t = blockIdx.x;
   const long long total = (long long)m + nnz;
@@ -138,6 +139,7 @@ template <typename T, int ITEMS>
 __global__ void __launch_bounds__(128)
 spmv_carry_fixup_kernel(int tiles, const int* __restrict__ row_ptr, const int* __restrict__ split_row,
                         const float* __restrict__ carry, const float* __restrict__ tail, T* __restrict__ y, float alpha, float beta) {
+  grid_dependency_wait();
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t < 1 || t >= tiles) return;
   const int r0 = split_row[t];

@@ -71,6 +71,7 @@ spmv_row_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const int*
     mbar_init_fence();
   }
   __syncthreads();
+  grid_dependency_wait();   // nothing above touches global memory
 
   // ---- producer (thread 0): stage i % stages <- tile blockIdx.x + i * gridDim.x
   int nb0 = 0, nb1 = 0;  // nonzero range of the next tile to issue (prefetched one step ahead)

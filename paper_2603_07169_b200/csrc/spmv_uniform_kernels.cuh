@@ -18,6 +18,7 @@ template <typename T, int LPR, int UNROLL, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 spmv_uniform_vec_kernel(long long quads, const int* __restrict__ col_idx, const T* __restrict__ vals,
                         const T* __restrict__ x, T* __restrict__ y, float alpha, float beta) {
+  grid_dependency_wait();
   const long long stride = (long long)gridDim.x * THREADS;
   long long g = (long long)blockIdx.x * THREADS + threadIdx.x;
   // every lane of a warp runs the same number of iterations: quads is a multiple of LPR and warps start on multiples of 32
@@ -98,6 +99,7 @@ template <typename T, int LPR, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 spmv_subwarp_kernel(int m, const int* __restrict__ row_ptr, const int* __restrict__ col_idx, const T* __restrict__ vals,
                     const T* __restrict__ x, T* __restrict__ y, float alpha, float beta) {
+  grid_dependency_wait();
   const long long gid = (long long)blockIdx.x * THREADS + threadIdx.x;
   const long long row = gid / LPR;
   const int sub = (int)(gid % LPR);
