@@ -329,3 +329,34 @@ def test_library_pool_reuses_and_returns_memory():
     torch.cuda.empty_cache()
     torch.cuda.synchronize()
     assert torch.cuda.mem_get_info()[0] >= free_start - (8 << 20)    # ... and gives it back on request
+
+
+@pytest.mark.parametrize("name,scale,dtype", [("c2", 2, "f32"), ("c2", 2, "bf16"), ("c3", 2, "f32"), ("c4", 2, "bf16"), ("c1", 0, "f32")])
+def test_dependent_calls_back_to_back(name, scale, dtype):
+    """Each call's input is the previous call's output, with no host synchronisation in between: the kernels are scheduled
+    behind one another (programmatic stream serialisation) and must still see the previous result complete.  The chain has
+    to be bit-identical to the same chain under plain stream order, and its first link has to match the oracle."""
+    w = gen.workload(name, scale_down=scale)
+    A = w.A
+    assert A.m == A.n
+    vals = store(A.vals, dtype)
+    d_rp, d_ci, d_va = to_dev(A.row_ptr), to_dev(A.col_idx), to_dev(vals)
+    x0 = store((w.x / 64.0).astype(np.float32), dtype)
+
+    def chain(pdl, links):
+        b200sp.b200sp_set_option("pdl", pdl)
+        try:
+            bufs = [to_dev(x0), empty_out(A.m, dtype)]
+            for i in range(links):
+                b200sp.spmv_csr(A.m, A.n, A.nnz, d_rp, d_ci, d_va, bufs[i % 2], bufs[(i + 1) % 2], 0.125, 0.0, dtype)
+            torch.cuda.synchronize()
+            return to_host(bufs[links % 2], dtype).copy()
+        finally:
+            b200sp.b200sp_set_option("pdl", 1)
+            b200sp.b200sp_cache_clear()
+
+    y1 = chain(1, 1)
+    y_ref, S = oracle.spmv_csr(A.m, A.n, A.row_ptr, A.col_idx, vals, x0, None, 0.125, 0.0, dtype)
+    assert_within(y1, y_ref, S, dtype, what="first link %s %s" % (name, dtype))
+    for links in (2, 7):
+        assert np.array_equal(chain(1, links), chain(0, links)), "chain of %d differs between launch modes" % links
