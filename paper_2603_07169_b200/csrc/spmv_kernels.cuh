@@ -27,7 +27,8 @@ spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const in
   constexpr int PROD_N = ITEMS + 2 * G;     // products of one tile, counted from the aligned start
   constexpr int MAX_LONG = ITEMS / (SHORT_MAX + 1) + 2;
   constexpr int WARPS = THREADS / 32;
-  __shared__ float prod[PROD_N + PROD_N / 32 + 1];
+  constexpr int PROD_SIZE = PROD_N + PROD_N / 32 + 1 + 8;
+  __shared__ float prod[PROD_SIZE];         // products from the front; the tile's row bounds (as ints) from the back: rows + nonzeros <= ITEMS, so they never meet
   __shared__ int long_rows[MAX_LONG];       // row of each long segment; -row-1 when the row began in an earlier tile
   __shared__ int2 long_span[MAX_LONG];      // its products: local [first, last)
   __shared__ int n_long;
@@ -43,8 +44,11 @@ spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const in
   const int a0 = p0 & ~(G - 1);
   if (tid == 0) n_long = 0;
   const int carry_start = r1 < m ? __ldg(row_ptr + r1) : 0;   // start of the unfinished last row, needed in phase 3: requested early
-  // the row bounds of phase 2 come straight from global memory: start them towards L2 now
-  for (int r = r0 + tid * 32; r <= r1; r += THREADS * 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(row_ptr + r));
+  // row_ptr[r0 .. r1] into the unused tail of prod (entry j at PROD_SIZE - 1 - j): phase 2 then needs no global load,
+  // which is what rows without nonzeros would otherwise spend their time waiting for
+  int* const bound_s = reinterpret_cast<int*>(prod) + (PROD_SIZE - 1);
+#pragma unroll 4
+  for (int j = tid; j <= r1 - r0; j += THREADS) bound_s[-j] = __ldg(row_ptr + r0 + j);
 
   // ---- phase 1: products of nonzeros [p0, p1) in flat order
   const int nq = (p1 - a0 + G - 1) / G;
@@ -91,7 +95,7 @@ spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const in
 
   // ---- phase 2: rows whose end lies in this tile, one thread per row
   for (int r = r0 + tid; r < r1; r += THREADS) {
-    const int rs = row_ptr[r], re = row_ptr[r + 1];
+    const int rs = bound_s[r0 - r], re = bound_s[r0 - r - 1];
     const int s = max(rs, p0);
     const int len = re - s;
     if (len <= SHORT_MAX) {
