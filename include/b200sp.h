@@ -253,7 +253,7 @@ int64_t b200sp_launch_count(void);
  *   "row_threads"    threads per CTA, 128 or 256 (default)
  *   "row_unroll"     gathers in flight per thread, 8 (default) or 16
  *  other kernels
- *   "uni_unroll"     groups of four nonzeros in flight per thread of the uniform-row kernel: 1, 2 or 4; 0 (default) = 1 for FP32, 2 for BF16
+ *   "uni_unroll"     groups of four nonzeros in flight per thread of the uniform-row kernel: 1, 2 or 4; 0 (default) = 1
  *   "uni_ctas"       CTAs per SM for the uniform-row kernel, 0 = as many as fit (default)
  *   "sub_lanes"      lanes per row of the sub-warp kernel (1..32, power of two), 0 = from the mean row length (default)
  *   "bstage_threads" threads per CTA of the SpMM kernel with B in shared memory: 256, 512 or 1024 (default)

@@ -47,7 +47,7 @@ struct Options {
   int row_unroll = 8;   // gathers in flight per thread (8 or 16)
   int row_smem_kb = 220;  // shared memory per SM the row-direct kernel may use for its stages (the rest stays L1)
   int row_threads = 256;  // threads per CTA of the row-direct kernel (128 or 256)
-  int uni_unroll = 0;     // groups of four nonzeros in flight per thread of the uniform-row kernel (1, 2 or 4); 0 = 1 for FP32 (32 registers, full occupancy), 2 for BF16
+  int uni_unroll = 0;     // groups of four nonzeros in flight per thread of the uniform-row kernel (1, 2 or 4); 0 = 1 (32 registers, full occupancy)
   int uni_ctas = 0;       // CTAs per SM for the uniform-row kernel (0 = as many as fit)
   int merge_staged = 0;   // 1 = persistent staged merge kernel, 0 = one-tile-per-CTA merge kernel
   int merge_items = 2048; // merge items per tile (2048 or 4096)

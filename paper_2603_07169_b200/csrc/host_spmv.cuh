@@ -139,7 +139,7 @@ int launch_uniform(b200sp_plan* p, const int32_t* col_idx, const T* vals, const 
 template <typename T, int LPR>
 int run_spmv_uniform_u(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
                        cudaStream_t stream, DeviceInfo* dev) {
-  const int unroll = g_opt.uni_unroll ? g_opt.uni_unroll : (sizeof(T) == 4 ? 1 : 2);   // measured on c2: FP32 67.9 / 69.7 us with 1 / 2, BF16 71.3 / 69.9 us
+  const int unroll = g_opt.uni_unroll ? g_opt.uni_unroll : 1;   // one group: 32 registers, all 2048 threads of an SM resident (c2 FP32 65.5 us against 67 us with two groups, BF16 68.2 against 69.8 us)
   if (unroll == 1) return launch_uniform<T, LPR, 1>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (unroll == 4) return launch_uniform<T, LPR, 4>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   return launch_uniform<T, LPR, 2>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
