@@ -38,8 +38,8 @@ FALLBACK_HBM_GBS = 6650.0
 # (workload, dtype); None where no capture has been made.  Sources: the summaries under profiles/.
 NCU_TRAFFIC_BYTES = {
     ("c2", "f32"): 148_018_944,     # profiles/spmv_uniform_vec_c2_f32.md
-    ("c2", "bf16"): 108_761_600,    # profiles/spmv_uniform_vec_c2_bf16.md
-    ("c3", "f32"): 305_535_488,     # profiles/spmv_merge_tile_c3_f32.md
+    ("c2", "bf16"): 108_764_928,    # profiles/spmv_uniform_vec_c2_bf16.md
+    ("c3", "f32"): 305_641_216,     # profiles/spmv_merge_tile_c3_f32.md
     ("c4", "bf16"): 690_968_832,    # profiles/spmv_row_tile_c4_bf16.md
     ("c1", "f32"): 3_163_648,       # profiles/spmv_row_tile_c1_f32.md
     ("c5k64", "f32"): 1_274_698_040,  # profiles/spmm_slice_c5k64_f32.md
