@@ -42,6 +42,7 @@ template <typename T, int LPR, int VECW, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 spmv_ell_kernel(int m, int width, const int* __restrict__ col_ids, const T* __restrict__ vals, const T* __restrict__ x,
                 T* __restrict__ y, float alpha, float beta) {
+  grid_dependency_wait();
   const long long gid = (long long)blockIdx.x * THREADS + threadIdx.x;
   const long long row = gid / LPR;
   const int sub = (int)(gid % LPR);

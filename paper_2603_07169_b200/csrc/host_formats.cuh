@@ -151,6 +151,7 @@ static int launch_ell_spmv(int64_t m, int width, const int32_t* col_ids, const T
   constexpr int THREADS = 128;
   const long long blocks = (m * LPR + THREADS - 1) / THREADS;
   if (blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+  tl_pdl_kernel = true;
   return launch(spmv_ell_kernel<T, LPR, VECW, THREADS>, dim3((unsigned)blocks), dim3(THREADS), stream, nullptr, 0, dev, (int)m, width, col_ids,
                 vals, x, y, alpha, beta);
 }
