@@ -90,6 +90,7 @@ int run_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const
   const b200sp_plan_info_t& I = p->info;
   if (I.m == 0) return B200SP_OK;
   if (alpha == 0.0f || I.nnz == 0) return run_scale<T>((long long)I.m * k, Y, beta, stream, dev);
+  if (k == 1) return run_spmv<T>(p, col_idx, vals, B, Y, alpha, beta, stream, dev);   // one column: the SpMV kernels
   if (k % VEC == 0 && g_opt.spmm_bstage && I.nnz >= 4 * I.n && ((size_t)k * sizeof(T)) % 16 == 0) {
     // widest slice of B (128, 64 or 32 bytes per row) whose n rows fit in one SM's shared memory
     const size_t budget = (size_t)kSmemPerSm - 4096;
@@ -114,20 +115,31 @@ int run_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const
     }
   }
   if (k % VEC == 0 && g_opt.spmm_sliced) {
-    constexpr int KS = 8 * VEC, GROUPS = kSpmmThreads / 8;
+    // lanes per row: eight (a 128-byte slice) unless k is narrower than that
+    const int vecs_k = k / VEC;
+    const int lanes = vecs_k >= 8 ? 8 : (vecs_k > 2 ? 4 : vecs_k);
+    const int KS = lanes * VEC, GROUPS = kSpmmThreads / lanes;
     const int slices = (k + KS - 1) / KS;
     const int row_blocks = (int)((I.m + GROUPS - 1) / GROUPS);
     if ((long long)slices * row_blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+    int rc;
     tl_pdl_kernel = true;
-    int rc = launch(spmm_slice_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)(slices * row_blocks)), dim3(kSpmmThreads), stream,
-                    nullptr, 0, dev,
-                    (int)I.m, k, row_blocks, p->row_ptr, col_idx, vals, B, Y, alpha, beta, kLongRow);
+#define B200SP_SLICE_LAUNCH(L)                                                                                                      \
+    rc = launch(spmm_slice_kernel<T, VEC, kSpmmThreads, L>, dim3((unsigned)(slices * row_blocks)), dim3(kSpmmThreads), stream, nullptr, 0, \
+                dev, (int)I.m, k, row_blocks, p->row_ptr, col_idx, vals, B, Y, alpha, beta, kLongRow)
+    if (lanes == 8) B200SP_SLICE_LAUNCH(8);
+    else if (lanes == 4) B200SP_SLICE_LAUNCH(4);
+    else if (lanes == 2) B200SP_SLICE_LAUNCH(2);
+    else B200SP_SLICE_LAUNCH(1);
+#undef B200SP_SLICE_LAUNCH
     if (rc != B200SP_OK || p->num_long == 0) return rc;
     tl_pdl_kernel = true;
-    return launch(spmm_long_row_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)(slices * p->num_long)), dim3(kSpmmThreads), stream, nullptr, 0,
+    return launch(spmm_long_row_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)(((k + 8 * VEC - 1) / (8 * VEC)) * p->num_long)), dim3(kSpmmThreads), stream, nullptr, 0,
                   dev, k, p->num_long, (const int*)p->long_rows, p->row_ptr, col_idx, vals, B, Y, alpha, beta);
   }
   if (k % VEC != 0) {  // ragged k: scalar lanes
+    if (k <= 2) return launch_spmm<T, 1, 2, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+    if (k <= 4) return launch_spmm<T, 1, 4, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
     if (k <= 8) return launch_spmm<T, 1, 8, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
     return launch_spmm<T, 1, 32, 2>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
   }

@@ -171,18 +171,18 @@ __device__ __forceinline__ void ld_a4(const int* col_idx, const bf16_t* vals, in
   v[2] = __uint_as_float(vv.y << 16); v[3] = __uint_as_float(vv.y & 0xFFFF0000u);
 }
 
-// k-sliced kernel.  The dense dimension is cut into slices of 8 * VEC columns = 128 bytes per row of B,
-// one cache line.  blockIdx.x = slice * row_blocks + row block, so CTAs run slice by slice and the
+// k-sliced kernel.  The dense dimension is cut into slices of LANES * VEC columns: 128 bytes per row of B, one cache
+// line, with the usual eight lanes per row; fewer lanes (4, 2, 1) when k itself is narrower than that, so that no lane idles.  blockIdx.x = slice * row_blocks + row block, so CTAs run slice by slice and the
 // part of B that a slice touches (n lines) can stay in L2 while every row of A passes over it; the
 // price is re-reading col_idx / vals once per slice.  Eight lanes own one row of A; all eight read the
 // row's (col, val) pairs with the same 128-bit loads (a broadcast, served by L1), and each lane keeps its
 // VEC columns of the slice in FP32 registers with four independent 16-byte reads of B in flight.
 // Rows longer than long_thresh are left to spmm_long_row_kernel.
-template <typename T, int VEC, int THREADS>
+template <typename T, int VEC, int THREADS, int LANES>
 __global__ void __launch_bounds__(THREADS, 2048 / THREADS)
 spmm_slice_kernel(int m, int k, int row_blocks, const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
                   const T* __restrict__ vals, const T* __restrict__ B, T* __restrict__ Y, float alpha, float beta, int long_thresh) {
-  constexpr int LANES = 8, GROUPS = THREADS / LANES, KS = LANES * VEC;
+  constexpr int GROUPS = THREADS / LANES, KS = LANES * VEC;
   typedef typename RawVec<T, VEC>::type raw_t;
   grid_dependency_wait();
   const int slice = blockIdx.x / row_blocks, rb = blockIdx.x - slice * row_blocks;
