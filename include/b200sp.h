@@ -70,8 +70,8 @@ typedef enum {
 /* Opaque: row statistics, row bins, nnz-balanced tile splits and the scratch the kernels need. */
 typedef struct b200sp_plan b200sp_plan;
 
-/* Row-length bins of the plan pass: rows of length 0, 1-4, 5-32, 33-1024 and > 1024. */
-#define B200SP_NUM_BINS 5
+/* Row-length bins of the plan pass: rows of length 0, 1-4, 5-32, 33-128, 129-1024 and > 1024. */
+#define B200SP_NUM_BINS 6
 
 /* What the plan pass found (b200sp_plan_info).  All counts are exact integers. */
 typedef struct {
@@ -83,8 +83,7 @@ typedef struct {
                                          2 = uniform-row sub-warp kernel, 3 = sub-warp-per-row kernel (small problems) */
   int32_t spmv_tile_items;            /* merge items (rows + nonzeros) per merge tile */
   int32_t spmv_tiles;                 /* number of merge tiles */
-  int32_t spmm_tile_nnz;              /* nonzeros per SpMM work unit */
-  int32_t spmm_tiles;                 /* number of SpMM work units */
+  int32_t reserved;                   /* 0 */
   int64_t scratch_bytes;              /* device memory held by the plan */
 } b200sp_plan_info_t;
 
@@ -92,7 +91,12 @@ typedef struct {
  * Task 12 / task 13 of the paper's Table 6 with alpha and beta.  The first call for a given
  * (device, row_ptr, m, n, nnz) builds a plan (see b200sp_plan_create; synchronises the stream once)
  * and caches it inside the library; later calls with the same key reuse it, so the CONTENTS of
- * row_ptr must not change while the plan is cached (b200sp_cache_clear drops all cached plans).
+ * row_ptr must not change while the plan is cached.  The key is the ADDRESS: if the caller frees row_ptr
+ * and an allocator hands the same address out again for another matrix with the same m, n and nnz (a
+ * caching allocator does this readily), the stale plan would be used and the result would be wrong
+ * without any error.  Call b200sp_cache_drop(row_ptr) before releasing or rewriting a row_ptr array (or
+ * b200sp_cache_clear for everything), or use the plan API, which has no hidden state.  The cache holds
+ * at most 64 plans and drops the least recently used one beyond that (dropping synchronises the device).
  * Two calls that use the same cached plan must not overlap on the GPU (they share its scratch).
  * dtype is a b200sp_dtype. */
 int spmv_csr(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx,
@@ -104,7 +108,8 @@ int spmm_csr(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_pt
 /* ---- plan API --------------------------------------------------------------------------------
  * The plan pass depends on the sparsity pattern's row structure only (row_ptr): it computes the
  * row-length statistics and bins, chooses the kernels, and computes the nnz-balanced split points
- * (a merge-path search over rows + nonzeros for SpMV, over nonzeros for SpMM), all on the device.
+ * (a merge-path search over rows + nonzeros) and the lists of rows of 129-1024 and of more than 1024 nonzeros that
+ * SpMM treats separately, all on the device.
  * When the row statistics select the row-direct SpMV kernel, the first b200sp_spmv / spmv_csr call with a given
  * col_idx additionally samples how local the columns are (one small kernel and one synchronisation of the stream)
  * and falls back to the merge-tile kernel for matrices with scattered columns.
@@ -182,8 +187,9 @@ int64_t b200sp_noalloc_max_items(void);   /* largest m + nnz that spmv_csr_noall
 /* ---- host-buffer calls -----------------------------------------------------------------------
  * Same operations with every array in HOST memory (pinned memory makes the copies asynchronous and
  * faster, pageable memory works).  Each call takes device buffers from the library's stream-ordered pool,
- * copies the inputs in, plans (cached per pattern shape is impossible here, so the plan is rebuilt),
- * runs the kernels, copies y / Y back and synchronises `stream` before returning. */
+ * copies the inputs in, plans, runs the kernels, copies y / Y back and synchronises `stream` before returning.
+ * The plan is cached under the HOST address of row_ptr and (m, n, nnz) like the plans of the device entry points, with
+ * the same rule: the contents of row_ptr must not change while it is cached (b200sp_cache_drop(row_ptr) forgets it). */
 int spmv_csr_host(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx,
                   const void* vals, const void* x, void* y, float alpha, float beta, int dtype, void* stream);
 int spmm_csr_host(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_ptr, const int32_t* col_idx,
@@ -201,6 +207,10 @@ int spmv_csr_vec_host(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr,
 int b200sp_validate_csr(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx, void* stream);
 
 void b200sp_cache_clear(void);                 /* destroys every plan cached by the one-shot calls and trims the library's memory pools */
+/* Forgets what the one-shot entry points cached under this address on the current device: the plan keyed on a row_ptr
+ * (device address, or host address for the *_host calls), the row offsets keyed on a COO row_idx, the transpose plan
+ * keyed on a CSC col_ptr.  Synchronises the device if anything was dropped.  Unknown addresses are not an error. */
+int b200sp_cache_drop(const void* key_ptr);
 const char* b200sp_status_string(int status);  /* static string, never NULL */
 const char* b200sp_last_cuda_error(void);      /* message of this thread's last failing CUDA call, "" if none */
 int b200sp_version(void);                      /* major * 10000 + minor * 100 + patch */
@@ -220,57 +230,10 @@ int b200sp_spmv_naive(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr,
 int b200sp_spmm_naive(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_ptr, const int32_t* col_idx, const void* vals,
                       const void* B, void* Y, float alpha, float beta, int dtype, void* stream);
 
-/* Measurement aid (no counterpart in the paper): enqueues `gathers` independent 4-byte reads of
- * table[h(i) mod table_elems] (table_elems a power of two, h a hash computed in registers), eight in
- * flight per thread, on as many CTAs as fit.  Timed by the caller with events it gives the rate at
- * which the SMs take random reads that miss L1, i.e. the bound on gathering x from a vector much
- * larger than L1.  `table` (table_elems floats) and `sink` (one float) are device pointers. */
-int b200sp_probe_gather(const float* table, int64_t table_elems, int64_t gathers, float* sink, void* stream);
-
 /* Number of kernels this library has launched from this process so far (all entry points). */
 int64_t b200sp_launch_count(void);
 
-/* Tuning switches for A/B measurements (the defaults are what the measurements in the repository selected);
- * unknown names or values out of range return B200SP_ERR_INVALID_ARG.
- *  kernel choice
- *   "spmv_kernel"    -1 = choose from the plan statistics (default), 0 = merge-tile, 1 = row-direct, 2 = uniform-row,
- *                    3 = sub-warp per row; a kernel the matrix is not eligible for falls back to an eligible one
- *   "spmm_bstage"    1 = SpMM keeps a slice of B in shared memory when A has few columns (default), 0 = never
- *   "spmm_sliced"    1 = SpMM walks k in 128-byte slices so that a slice of B can stay in L2 (default), 0 = one pass
- *  merge-tile SpMV kernel
- *   "merge_items"    merge items per tile: 1024, 2048 (default) or 4096
- *   "merge_threads"  threads per CTA: 64, 128 (default) or 256
- *   "merge_carve"    shared-memory carveout in percent requested for it, default 45 (-1 = leave to the driver)
- *   "merge_short"    rows of up to this many products are added by one thread: 8, 16, 32 (default) or 64
- *   "merge_scan"     1 = reduce rows with an in-register segmented scan, 0 = products through shared memory (default)
- *   "merge_stride"   with merge_scan: walk the tiles with this stride (made coprime to their number), 0 = in order
- *   "merge_staged"   1 = persistent variant with bulk-copy stages, 0 = one tile per CTA (default)
- *   "merge_stages", "merge_ctas"   stages per CTA (2..4) and CTAs per SM of the staged variant
- *  row-direct SpMV kernel
- *   "row_stages"     shared-memory stages per CTA, 2 (default) .. 4
- *   "row_ctas"       CTAs per SM the tiles are sized for, default 3
- *   "row_smem_kb"    shared memory per SM it may use for stages, default 220 (what is left stays L1)
- *   "row_threads"    threads per CTA, 128 or 256 (default)
- *   "row_unroll"     gathers in flight per thread, 8 (default) or 16
- *  other kernels
- *   "uni_unroll"     groups of four nonzeros in flight per thread of the uniform-row kernel: 1, 2 or 4; 0 (default) = 1
- *   "uni_ctas"       CTAs per SM for the uniform-row kernel, 0 = as many as fit (default)
- *   "sub_lanes"      lanes per row of the sub-warp kernel (1..32, power of two), 0 = from the mean row length (default)
- *   "bstage_threads" threads per CTA of the SpMM kernel with B in shared memory: 256, 512 or 1024 (default)
- *   "bstage_nnz"     nonzeros of A per CTA that kernel aims for, default 131072
- *   "bstage_stage_a" 1 = its warps first copy their rows' (col, val) pairs into shared-memory buffers of their own (default),
- *                    0 = the pairs are read from global memory inside the row loop
- *   "x_l2_window"    1 = pin x in L2 with a per-launch access-policy window, 0 = off (default: measured to give
- *                    nothing on large problems, where x stays in L2 anyway, and to cost 1.4 us per launch on tiny ones)
- *  launch
- *   "pdl"            1 = the SpMV and SpMM kernels are launched with programmatic stream serialisation (default): each begins
- *                    with griddepcontrol.wait, so it may be scheduled while the stream's previous kernel drains and touches no
- *                    memory before that kernel has completed; 0 = plain stream order
- *  memory
- *   "pool_keep_mb"   MiB of freed memory the library's pool keeps across synchronisation points, default 1024
- *                    (read when a device's pool is created, i.e. before the first call that allocates on it)
- * "spmv_kernel" and "merge_items" apply to plans created afterwards, the others to the next call. */
-int b200sp_set_option(const char* name, int value);
+/* Tuning switches, test switches and measurement probes live in b200sp_tuning.h: they are not part of the contract above. */
 
 #ifdef __cplusplus
 }

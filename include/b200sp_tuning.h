@@ -1,0 +1,79 @@
+/*
+ * b200sp -- tuning switches, test switches and measurement probes of libb200sp.so.
+ *
+ * Nothing here is needed to use the operations declared in b200sp.h (paper: Appendix C, Table 6, tasks 8-15); the
+ * defaults are what the measurements kept with the library selected.  The switches exist so that each design choice
+ * can be measured against its alternative on the same build, and so that failure paths can be reached in tests
+ * without faulting a GPU.  Every accepted value of every switch is exercised against the CPU reference by the test
+ * suite.  The probes have no counterpart in the paper: they measure the hardware rates that bound the kernels
+ * (the paper's Appendix A sorts kernels by which such rate limits them).
+ */
+#ifndef B200SP_TUNING_H_
+#define B200SP_TUNING_H_
+
+#include "b200sp.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Sets a switch for the whole process; unknown names or values out of range return B200SP_ERR_INVALID_ARG.
+ *  kernel choice
+ *   "spmv_kernel"    -1 = choose from the plan statistics (default), 0 = merge-tile, 1 = row-direct, 2 = uniform-row,
+ *                    3 = sub-warp per row; a kernel the matrix is not eligible for falls back to an eligible one
+ *   "spmm_bstage"    1 = SpMM keeps a slice of B in shared memory when A has few columns (default), 0 = never
+ *   "spmm_sliced"    1 = SpMM walks k in 128-byte slices so that a slice of B can stay in L2 (default), 0 = one pass
+ *   "spmm_ranges"    SpMM with sorted columns: 0 = choose the number of column ranges per slice so that a range of B
+ *                    fits in L2 (default), 1 = never split, 2..8 = this many ranges
+ *  merge-tile SpMV kernel
+ *   "merge_items"    merge items per tile: 1024, 2048 (default) or 4096
+ *   "merge_threads"  threads per CTA: 64, 128 (default) or 256
+ *   "merge_carve"    shared-memory carveout in percent requested for it: 0, 25, 45 (default), 60, 75, 100 or -1 = leave to the driver
+ *   "merge_short"    rows of up to this many products are added by one thread: 8, 16, 32 (default) or 64
+ *   "merge_empty"    1 = when many rows have no nonzeros they are kept out of the merge list and their y is written by a
+ *                    pass of its own (default), 0 = every row is a merge item
+ *  row-direct SpMV kernel
+ *   "row_stages"     shared-memory stages per CTA, 2 (default) .. 4
+ *   "row_ctas"       CTAs per SM the tiles are sized for, 1..4, default 3
+ *   "row_smem_kb"    shared memory per SM it may use for stages: 48, 96, 160, 220 (default) or 227 (what is left stays L1)
+ *   "row_threads"    threads per CTA, 128 or 256 (default)
+ *   "row_unroll"     gathers in flight per thread, 8 (default) or 16
+ *  other kernels
+ *   "uni_unroll"     groups of four nonzeros in flight per thread of the uniform-row kernel: 1, 2 or 4; 0 (default) = 1
+ *   "uni_ctas"       CTAs per SM for the uniform-row kernel: 1, 2, 4, 8 or 0 = as many as fit (default)
+ *   "sub_lanes"      least number of lanes per row of the sub-warp kernel (1..32, power of two), 0 = from the mean row
+ *                    length (default); more lanes are used where a lane would otherwise add more than 128 products
+ *   "bstage_threads" threads per CTA of the SpMM kernel with B in shared memory: 256, 512 or 1024 (default)
+ *   "bstage_nnz"     nonzeros of A per CTA that kernel aims for: 16384, 65536, 131072 (default) or 524288
+ *   "bstage_stage_a" 1 = its warps first copy their rows' (col, val) pairs into shared-memory buffers of their own (default),
+ *                    0 = the pairs are read from global memory inside the row loop
+ *   "x_l2_window"    1 = pin the gathered operand (x, or B for SpMM) in L2 with a per-launch access-policy window, 0 = off
+ *                    (default; the measured effect is recorded with the benchmarks)
+ *  launch
+ *   "pdl"            1 = the SpMV and SpMM kernels are launched with programmatic stream serialisation (default): each begins
+ *                    with griddepcontrol.wait, so it may be scheduled while the stream's previous kernel drains and touches no
+ *                    memory before that kernel has completed; 0 = plain stream order
+ *  memory
+ *   "pool_keep_mb"   MiB of freed memory the library's pool keeps across synchronisation points, default 1024
+ *                    (read when a device's pool is created, i.e. before the first call that allocates on it)
+ *  test switches (they make a failure path run; none of them can fault or hang the device)
+ *   "spin_limit"       polls after which a kernel's bounded wait on a shared-memory barrier gives up, default 1048576
+ *   "debug_no_copies"  1 = the kernels that stage data through shared memory (row-direct SpMV, ELL row-direct SpMV, SpMM with
+ *                      B in shared memory) issue no copy and arm no barrier, so their waits run out after "spin_limit" polls
+ *                      with nothing in flight; the launch raises the flag that b200sp_check reports and its output is undefined
+ *   "fail_alloc_after" N > 0: the N-th allocation the library makes from its memory pool from now on fails with
+ *                      B200SP_ERR_ALLOC (the switch then clears itself); 0 = off (default)
+ * "spmv_kernel" and "merge_items" apply to plans created afterwards, the others to the next call. */
+int b200sp_set_option(const char* name, int value);
+
+/* Measurement aid (no counterpart in the paper): enqueues `gathers` independent 4-byte reads of
+ * table[h(i) mod table_elems] (table_elems a power of two, h a hash computed in registers), eight in
+ * flight per thread, on as many CTAs as fit.  Timed by the caller with events it gives the rate at
+ * which the SMs take random reads that miss L1, i.e. the bound on gathering x from a vector much
+ * larger than L1.  `table` (table_elems floats) and `sink` (one float) are device pointers. */
+int b200sp_probe_gather(const float* table, int64_t table_elems, int64_t gathers, float* sink, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* B200SP_TUNING_H_ */

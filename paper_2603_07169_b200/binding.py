@@ -20,16 +20,16 @@ EXPORTS = (
     "spmv_csr", "spmm_csr", "b200sp_plan_create", "b200sp_plan_destroy", "b200sp_plan_info", "b200sp_spmv",
     "b200sp_spmm", "spmv_csr_host", "spmm_csr_host", "b200sp_validate_csr", "b200sp_cache_clear",
     "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_launch_count", "b200sp_set_option",
-    "b200sp_check", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell", "spmv_csc", "spmm_csc", "spmv_csr_vec_host",
+    "b200sp_check", "b200sp_cache_drop", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell", "spmv_csc", "spmm_csc", "spmv_csr_vec_host",
 )
 
 
 class PlanInfo(ctypes.Structure):
     _fields_ = [("m", ctypes.c_int64), ("n", ctypes.c_int64), ("nnz", ctypes.c_int64),
                 ("min_row_len", ctypes.c_int32), ("max_row_len", ctypes.c_int32),
-                ("bin_rows", ctypes.c_int64 * 5), ("bin_nnz", ctypes.c_int64 * 5),
+                ("bin_rows", ctypes.c_int64 * 6), ("bin_nnz", ctypes.c_int64 * 6),
                 ("spmv_kernel", ctypes.c_int32), ("spmv_tile_items", ctypes.c_int32), ("spmv_tiles", ctypes.c_int32),
-                ("spmm_tile_nnz", ctypes.c_int32), ("spmm_tiles", ctypes.c_int32), ("scratch_bytes", ctypes.c_int64)]
+                ("reserved", ctypes.c_int32), ("scratch_bytes", ctypes.c_int64)]
 
     def as_dict(self):
         d = {}
@@ -44,7 +44,7 @@ class B200spError(RuntimeError):
         self.status = status
         msg = lib().b200sp_status_string(status).decode()
         detail = lib().b200sp_last_cuda_error().decode()
-        super().__init__("%s: %s (status %d)%s" % (where, msg, status, (": " + detail) if detail and status == 3 else ""))
+        super().__init__("%s: %s (status %d)%s" % (where, msg, status, (": " + detail) if detail and status in (3, 4) else ""))
 
 
 _lib = None
@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.b200sp_spmv.argtypes = [p, p, p, p, p, f32, f32, i32, p]
         L.b200sp_spmm.argtypes = [p, i64, p, p, p, p, f32, f32, i32, p]
         L.b200sp_validate_csr.argtypes = [i64, i64, i64, p, p, p]
+        L.b200sp_cache_drop.argtypes = [p]
+        L.b200sp_cache_drop.restype = i32
         L.b200sp_cache_clear.argtypes = []
         L.b200sp_cache_clear.restype = None
         L.b200sp_status_string.argtypes = [i32]
@@ -114,6 +116,52 @@ def _ptr(t) -> Optional[int]:
     return t.ctypes.data
 
 
+def _esize(dtype) -> int:
+    return 4 if _dt(dtype) == F32 else 2
+
+
+def _dev(t, elems: int, esize: int, what: str) -> Optional[int]:
+    """Address of a DEVICE operand.  The kernels dereference it on the GPU, and the library cannot tell a host address from
+    a device address or see how long an array is, so this is the only place where a wrong tensor can be stopped: it must be
+    a contiguous CUDA tensor on the current device with elements of `esize` bytes and at least `elems` of them.  Anything
+    else raises B200spError(INVALID_ARG) before the library is entered.  None stays NULL (the library checks NULL
+    against the sizes)."""
+    if t is None:
+        return None
+    import torch
+    ok = isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.device.index == torch.cuda.current_device() \
+        and t.element_size() == esize and (elems < 0 or t.numel() >= elems)
+    if not ok:
+        raise B200spError(1, "%s: expected a contiguous CUDA tensor on the current device with >= %d elements of %d bytes, got %s"
+                          % (what, elems, esize, _describe(t)))
+    return t.data_ptr()
+
+
+def _host(t, elems: int, esize: int, what: str) -> Optional[int]:
+    """Address of a HOST operand of the *_host entry points: a C-contiguous numpy array or a contiguous CPU tensor."""
+    if t is None:
+        return None
+    if hasattr(t, "is_cuda"):
+        ok = (not t.is_cuda) and t.is_contiguous() and t.element_size() == esize and (elems < 0 or t.numel() >= elems)
+        addr = t.data_ptr() if ok else None
+    else:
+        ok = hasattr(t, "ctypes") and t.flags["C_CONTIGUOUS"] and t.itemsize == esize and (elems < 0 or t.size >= elems)
+        addr = t.ctypes.data if ok else None
+    if not ok:
+        raise B200spError(1, "%s: expected a contiguous host array with >= %d elements of %d bytes, got %s"
+                          % (what, elems, esize, _describe(t)))
+    return addr
+
+
+def _describe(t) -> str:
+    try:
+        if hasattr(t, "is_cuda"):
+            return "torch tensor(device=%s, dtype=%s, numel=%d, contiguous=%s)" % (t.device, t.dtype, t.numel(), t.is_contiguous())
+        return "%s(dtype=%s, size=%d)" % (type(t).__name__, getattr(t, "dtype", "?"), getattr(t, "size", -1))
+    except Exception:  # pragma: no cover
+        return repr(type(t))
+
+
 def _stream(stream) -> Optional[int]:
     if stream is None:
         import torch
@@ -132,60 +180,88 @@ def _ck(status: int, where: str):
         raise B200spError(status, where)
 
 
+def _csr_args(m, n, nnz, k, row_ptr, col_idx, vals, dense_in, dense_out, dtype, what, conv=_dev):
+    e = _esize(dtype)
+    kk = max(k, 1)
+    return (conv(row_ptr, m + 1 if m > 0 else 0, 4, what + " row_ptr"), conv(col_idx, nnz, 4, what + " col_idx"), conv(vals, nnz, e, what + " vals"),
+            conv(dense_in, n * kk if nnz > 0 else 0, e, what + " x/B"), conv(dense_out, m * kk, e, what + " y/Y"))
+
+
 def spmv_csr(m, n, nnz, row_ptr, col_idx, vals, x, y, alpha, beta, dtype, stream=None):
-    _ck(lib().spmv_csr(m, n, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype),
-                       _stream(stream)), "spmv_csr")
+    a = _csr_args(m, n, nnz, 0, row_ptr, col_idx, vals, x, y, dtype, "spmv_csr")
+    _ck(lib().spmv_csr(m, n, nnz, a[0], a[1], a[2], a[3], a[4], alpha, beta, _dt(dtype), _stream(stream)), "spmv_csr")
 
 
 def spmm_csr(m, n, nnz, k, row_ptr, col_idx, vals, B, Y, alpha, beta, dtype, stream=None):
-    _ck(lib().spmm_csr(m, n, nnz, k, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(B), _ptr(Y), alpha, beta, _dt(dtype),
-                       _stream(stream)), "spmm_csr")
+    a = _csr_args(m, n, nnz, k, row_ptr, col_idx, vals, B, Y, dtype, "spmm_csr")
+    _ck(lib().spmm_csr(m, n, nnz, k, a[0], a[1], a[2], a[3], a[4], alpha, beta, _dt(dtype), _stream(stream)), "spmm_csr")
 
 
 def spmv_csr_noalloc(m, n, nnz, row_ptr, col_idx, vals, x, y, alpha, beta, dtype, stream=None):
     """SpMV for callers that may not allocate device memory: scratch comes from a fixed array inside the
     library (m + nnz <= b200sp_noalloc_max_items()); overlapping calls race on that array."""
-    _ck(lib().spmv_csr_noalloc(m, n, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype),
-                               _stream(stream)), "spmv_csr_noalloc")
+    if 0 <= m + nnz <= b200sp_noalloc_max_items():
+        a = _csr_args(m, n, nnz, 0, row_ptr, col_idx, vals, x, y, dtype, "spmv_csr_noalloc")
+    else:   # refused by the library on the sizes alone: nothing is dereferenced
+        a = [_ptr(t) for t in (row_ptr, col_idx, vals, x, y)]
+    _ck(lib().spmv_csr_noalloc(m, n, nnz, a[0], a[1], a[2], a[3], a[4], alpha, beta, _dt(dtype), _stream(stream)), "spmv_csr_noalloc")
 
 
 def spmv_coo(m, n, nnz, row_idx, col_idx, vals, x, y, alpha, beta, dtype, stream=None):
-    _ck(lib().spmv_coo(m, n, nnz, _ptr(row_idx), _ptr(col_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype), _stream(stream)), "spmv_coo")
+    e = _esize(dtype)
+    _ck(lib().spmv_coo(m, n, nnz, _dev(row_idx, nnz, 4, "spmv_coo row_idx"), _dev(col_idx, nnz, 4, "spmv_coo col_idx"),
+                       _dev(vals, nnz, e, "spmv_coo vals"), _dev(x, n if nnz > 0 else 0, e, "spmv_coo x"), _dev(y, m, e, "spmv_coo y"),
+                       alpha, beta, _dt(dtype), _stream(stream)), "spmv_coo")
 
 
 def spmm_coo(m, n, nnz, k, row_idx, col_idx, vals, B, Y, alpha, beta, dtype, stream=None):
-    _ck(lib().spmm_coo(m, n, nnz, k, _ptr(row_idx), _ptr(col_idx), _ptr(vals), _ptr(B), _ptr(Y), alpha, beta, _dt(dtype), _stream(stream)), "spmm_coo")
+    e = _esize(dtype)
+    _ck(lib().spmm_coo(m, n, nnz, k, _dev(row_idx, nnz, 4, "spmm_coo row_idx"), _dev(col_idx, nnz, 4, "spmm_coo col_idx"),
+                       _dev(vals, nnz, e, "spmm_coo vals"), _dev(B, n * k if nnz > 0 else 0, e, "spmm_coo B"), _dev(Y, m * k, e, "spmm_coo Y"),
+                       alpha, beta, _dt(dtype), _stream(stream)), "spmm_coo")
 
 
 def spmv_csc(m, n, nnz, col_ptr, row_idx, vals, x, y, alpha, beta, dtype, stream=None):
-    _ck(lib().spmv_csc(m, n, nnz, _ptr(col_ptr), _ptr(row_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype), _stream(stream)), "spmv_csc")
+    e = _esize(dtype)
+    _ck(lib().spmv_csc(m, n, nnz, _dev(col_ptr, n + 1, 4, "spmv_csc col_ptr"), _dev(row_idx, nnz, 4, "spmv_csc row_idx"),
+                       _dev(vals, nnz, e, "spmv_csc vals"), _dev(x, n if nnz > 0 else 0, e, "spmv_csc x"), _dev(y, m, e, "spmv_csc y"),
+                       alpha, beta, _dt(dtype), _stream(stream)), "spmv_csc")
 
 
 def spmm_csc(m, n, nnz, k, col_ptr, row_idx, vals, B, Y, alpha, beta, dtype, stream=None):
-    _ck(lib().spmm_csc(m, n, nnz, k, _ptr(col_ptr), _ptr(row_idx), _ptr(vals), _ptr(B), _ptr(Y), alpha, beta, _dt(dtype), _stream(stream)), "spmm_csc")
+    e = _esize(dtype)
+    _ck(lib().spmm_csc(m, n, nnz, k, _dev(col_ptr, n + 1, 4, "spmm_csc col_ptr"), _dev(row_idx, nnz, 4, "spmm_csc row_idx"),
+                       _dev(vals, nnz, e, "spmm_csc vals"), _dev(B, n * k if nnz > 0 else 0, e, "spmm_csc B"), _dev(Y, m * k, e, "spmm_csc Y"),
+                       alpha, beta, _dt(dtype), _stream(stream)), "spmm_csc")
 
 
 def spmv_ell(m, n, width, col_ids, vals, x, y, alpha, beta, dtype, stream=None):
-    _ck(lib().spmv_ell(m, n, width, _ptr(col_ids), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype), _stream(stream)), "spmv_ell")
+    e = _esize(dtype)
+    _ck(lib().spmv_ell(m, n, width, _dev(col_ids, m * width, 4, "spmv_ell col_ids"), _dev(vals, m * width, e, "spmv_ell vals"),
+                       _dev(x, n if m * width > 0 else 0, e, "spmv_ell x"), _dev(y, m, e, "spmv_ell y"), alpha, beta, _dt(dtype), _stream(stream)), "spmv_ell")
 
 
 def spmm_ell(m, n, width, k, col_ids, vals, B, Y, alpha, beta, dtype, stream=None):
-    _ck(lib().spmm_ell(m, n, width, k, _ptr(col_ids), _ptr(vals), _ptr(B), _ptr(Y), alpha, beta, _dt(dtype), _stream(stream)), "spmm_ell")
+    e = _esize(dtype)
+    _ck(lib().spmm_ell(m, n, width, k, _dev(col_ids, m * width, 4, "spmm_ell col_ids"), _dev(vals, m * width, e, "spmm_ell vals"),
+                       _dev(B, n * k if m * width > 0 else 0, e, "spmm_ell B"), _dev(Y, m * k, e, "spmm_ell Y"), alpha, beta, _dt(dtype),
+                       _stream(stream)), "spmm_ell")
 
 
 def b200sp_spmv_naive(m, n, nnz, row_ptr, col_idx, vals, x, y, alpha, beta, dtype, stream=None):
-    _ck(lib().b200sp_spmv_naive(m, n, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype),
-                                _stream(stream)), "b200sp_spmv_naive")
+    a = _csr_args(m, n, nnz, 0, row_ptr, col_idx, vals, x, y, dtype, "b200sp_spmv_naive")
+    _ck(lib().b200sp_spmv_naive(m, n, nnz, a[0], a[1], a[2], a[3], a[4], alpha, beta, _dt(dtype), _stream(stream)), "b200sp_spmv_naive")
 
 
 def b200sp_spmm_naive(m, n, nnz, k, row_ptr, col_idx, vals, B, Y, alpha, beta, dtype, stream=None):
-    _ck(lib().b200sp_spmm_naive(m, n, nnz, k, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(B), _ptr(Y), alpha, beta, _dt(dtype),
-                                _stream(stream)), "b200sp_spmm_naive")
+    a = _csr_args(m, n, nnz, k, row_ptr, col_idx, vals, B, Y, dtype, "b200sp_spmm_naive")
+    _ck(lib().b200sp_spmm_naive(m, n, nnz, k, a[0], a[1], a[2], a[3], a[4], alpha, beta, _dt(dtype), _stream(stream)), "b200sp_spmm_naive")
 
 
 def b200sp_probe_gather(table, table_elems, gathers, sink, stream=None):
-    """Enqueues the random-gather probe (see include/b200sp.h); time it with CUDA events."""
-    _ck(lib().b200sp_probe_gather(_ptr(table), table_elems, gathers, _ptr(sink), _stream(stream)), "b200sp_probe_gather")
+    """Enqueues the random-gather probe (see include/b200sp_tuning.h); time it with CUDA events."""
+    _ck(lib().b200sp_probe_gather(_dev(table, table_elems, 4, "probe table"), table_elems, gathers, _dev(sink, 1, 4, "probe sink"),
+                                  _stream(stream)), "b200sp_probe_gather")
 
 
 def b200sp_noalloc_max_items() -> int:
@@ -193,24 +269,28 @@ def b200sp_noalloc_max_items() -> int:
 
 
 def spmv_csr_host(m, n, nnz, row_ptr, col_idx, vals, x, y, alpha, beta, dtype, stream=None):
-    _ck(lib().spmv_csr_host(m, n, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype),
-                            _stream(stream)), "spmv_csr_host")
+    a = _csr_args(m, n, nnz, 0, row_ptr, col_idx, vals, x, y, dtype, "spmv_csr_host", conv=_host)
+    _ck(lib().spmv_csr_host(m, n, nnz, a[0], a[1], a[2], a[3], a[4], alpha, beta, _dt(dtype), _stream(stream)), "spmv_csr_host")
 
 
 def spmv_csr_vec_host(m, n, nnz, row_ptr, col_idx, vals, x_host, y_host, alpha, beta, dtype, stream=None):
     """Device-resident matrix, host x and y (one step of an iterative method)."""
-    _ck(lib().spmv_csr_vec_host(m, n, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(x_host), _ptr(y_host), alpha, beta, _dt(dtype),
-                                _stream(stream)), "spmv_csr_vec_host")
+    e = _esize(dtype)
+    _ck(lib().spmv_csr_vec_host(m, n, nnz, _dev(row_ptr, m + 1 if m > 0 else 0, 4, "spmv_csr_vec_host row_ptr"),
+                                _dev(col_idx, nnz, 4, "spmv_csr_vec_host col_idx"), _dev(vals, nnz, e, "spmv_csr_vec_host vals"),
+                                _host(x_host, n if nnz > 0 else 0, e, "spmv_csr_vec_host x"), _host(y_host, m, e, "spmv_csr_vec_host y"),
+                                alpha, beta, _dt(dtype), _stream(stream)), "spmv_csr_vec_host")
 
 
 def spmm_csr_host(m, n, nnz, k, row_ptr, col_idx, vals, B, Y, alpha, beta, dtype, stream=None):
-    _ck(lib().spmm_csr_host(m, n, nnz, k, _ptr(row_ptr), _ptr(col_idx), _ptr(vals), _ptr(B), _ptr(Y), alpha, beta, _dt(dtype),
-                            _stream(stream)), "spmm_csr_host")
+    a = _csr_args(m, n, nnz, k, row_ptr, col_idx, vals, B, Y, dtype, "spmm_csr_host", conv=_host)
+    _ck(lib().spmm_csr_host(m, n, nnz, k, a[0], a[1], a[2], a[3], a[4], alpha, beta, _dt(dtype), _stream(stream)), "spmm_csr_host")
 
 
 def b200sp_plan_create(m, n, nnz, row_ptr, stream=None) -> int:
     out = ctypes.c_void_p()
-    _ck(lib().b200sp_plan_create(ctypes.byref(out), m, n, nnz, _ptr(row_ptr), _stream(stream)), "b200sp_plan_create")
+    _ck(lib().b200sp_plan_create(ctypes.byref(out), m, n, nnz, _dev(row_ptr, m + 1 if m > 0 else 0, 4, "b200sp_plan_create row_ptr"),
+                                 _stream(stream)), "b200sp_plan_create")
     return out.value
 
 
@@ -225,16 +305,21 @@ def b200sp_plan_info(plan) -> dict:
 
 
 def b200sp_spmv(plan, col_idx, vals, x, y, alpha, beta, dtype, stream=None):
-    _ck(lib().b200sp_spmv(plan, _ptr(col_idx), _ptr(vals), _ptr(x), _ptr(y), alpha, beta, _dt(dtype), _stream(stream)), "b200sp_spmv")
+    I = b200sp_plan_info(plan)      # the plan knows m, n, nnz
+    a = _csr_args(I["m"], I["n"], I["nnz"], 0, None, col_idx, vals, x, y, dtype, "b200sp_spmv")
+    _ck(lib().b200sp_spmv(plan, a[1], a[2], a[3], a[4], alpha, beta, _dt(dtype), _stream(stream)), "b200sp_spmv")
 
 
 def b200sp_spmm(plan, k, col_idx, vals, B, Y, alpha, beta, dtype, stream=None):
-    _ck(lib().b200sp_spmm(plan, k, _ptr(col_idx), _ptr(vals), _ptr(B), _ptr(Y), alpha, beta, _dt(dtype), _stream(stream)), "b200sp_spmm")
+    I = b200sp_plan_info(plan)
+    a = _csr_args(I["m"], I["n"], I["nnz"], k, None, col_idx, vals, B, Y, dtype, "b200sp_spmm")
+    _ck(lib().b200sp_spmm(plan, k, a[1], a[2], a[3], a[4], alpha, beta, _dt(dtype), _stream(stream)), "b200sp_spmm")
 
 
 def b200sp_validate_csr(m, n, nnz, row_ptr, col_idx, stream=None) -> int:
     """Returns the status (0 = consistent, 6 = inconsistent CSR) instead of raising on a bad matrix."""
-    rc = lib().b200sp_validate_csr(m, n, nnz, _ptr(row_ptr), _ptr(col_idx), _stream(stream))
+    rc = lib().b200sp_validate_csr(m, n, nnz, _dev(row_ptr, m + 1, 4, "b200sp_validate_csr row_ptr"),
+                                   _dev(col_idx, nnz, 4, "b200sp_validate_csr col_idx"), _stream(stream))
     if rc not in (0, 6):
         raise B200spError(rc, "b200sp_validate_csr")
     return rc
@@ -247,6 +332,13 @@ def b200sp_check(stream=None):
 
 def b200sp_cache_clear():
     lib().b200sp_cache_clear()
+
+
+def b200sp_cache_drop(key):
+    """Forgets what the one-shot calls cached under this array's address (a row_ptr / row_idx / col_ptr tensor or array).
+    Call it before freeing or rewriting such an array: the caches are keyed on addresses, and an allocator that hands
+    the address out again would otherwise revive a stale plan."""
+    _ck(lib().b200sp_cache_drop(_ptr(key)), "b200sp_cache_drop")
 
 
 def b200sp_version() -> int:

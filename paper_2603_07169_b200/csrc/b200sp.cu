@@ -285,8 +285,13 @@ static int host_call(bool is_mm, int64_t m, int64_t n, int64_t nnz, int64_t k, c
   rc = pool_alloc(dev, (void**)&base, total, stream);
   if (rc != B200SP_OK) return rc;
   char* d_rp = base; char* d_ci = d_rp + up(b_rp); char* d_va = d_ci + up(b_ci); char* d_in = d_va + up(b_va); char* d_out = d_in + up(b_in);
-  b200sp_plan* p = nullptr;
-  auto done = [&](int code) { if (p) plan_free(p, true, stream); cudaFreeAsync(base, stream); cudaStreamSynchronize(stream); return code; };
+  // the plan is cached under the HOST address of row_ptr: a later call with the same address and sizes skips the plan pass
+  // (the header states that the contents must then be unchanged, as for the device entry points)
+  int cur_dev = 0;
+  CU(cudaGetDevice(&cur_dev));
+  const PlanKey key = std::make_tuple(cur_dev, (const void*)row_ptr, m, n, nnz);
+  b200sp_plan* p = cache_find(key);
+  auto done = [&](int code) { cudaFreeAsync(base, stream); cudaStreamSynchronize(stream); return code; };
 #define CUH(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return done(cuda_fail(e_, #call)); } while (0)
   CUH(cudaMemcpyAsync(d_rp, row_ptr, b_rp, cudaMemcpyHostToDevice, stream));
   if (nnz > 0) {
@@ -295,11 +300,18 @@ static int host_call(bool is_mm, int64_t m, int64_t n, int64_t nnz, int64_t k, c
     CUH(cudaMemcpyAsync(d_in, in, b_in, cudaMemcpyHostToDevice, stream));
   }
   if (beta != 0.0f) CUH(cudaMemcpyAsync(d_out, out, b_out, cudaMemcpyHostToDevice, stream));
-  rc = plan_build(&p, m, n, nnz, (const int32_t*)d_rp, stream);
-  if (rc != B200SP_OK) { p = nullptr; return done(rc); }
+  if (!p) {
+    rc = plan_build(&p, m, n, nnz, (const int32_t*)d_rp, stream);
+    if (rc != B200SP_OK) return done(rc);
+    p = cache_insert(key, p);
+  }
+  p->row_ptr = (const int32_t*)d_rp;             // this call's staging copy
+  if (p->probed_key == (const void*)col_idx) p->probed_col_idx = d_ci;   // the column-locality verdict follows the host pattern
+  else p->probed_col_idx = nullptr;
   rc = is_mm ? b200sp_spmm(p, k, (const int32_t*)d_ci, d_va, d_in, d_out, alpha, beta, dtype, stream)
              : b200sp_spmv(p, (const int32_t*)d_ci, d_va, d_in, d_out, alpha, beta, dtype, stream);
   if (rc != B200SP_OK) return done(rc);
+  if (p->probed_col_idx == (const void*)d_ci) p->probed_key = col_idx;
   CUH(cudaMemcpyAsync(out, d_out, b_out, cudaMemcpyDeviceToHost, stream));
   CUH(cudaStreamSynchronize(stream));
 #undef CUH
@@ -371,9 +383,43 @@ int b200sp_validate_csr(int64_t m, int64_t n, int64_t nnz, const int32_t* row_pt
   return h_bad ? B200SP_ERR_BAD_CSR : B200SP_OK;
 }
 
+// Drops what the one-shot entry points cached under this pointer on the current device: plans keyed on a row_ptr
+// (device or host address), COO row offsets keyed on a row_idx, CSC transpose plans keyed on a col_ptr.
+int b200sp_cache_drop(const void* key_ptr) {
+  if (!key_ptr) return B200SP_ERR_INVALID_ARG;
+  int dev = 0;
+  CU(cudaGetDevice(&dev));
+  std::vector<b200sp_plan*> plans;
+  std::vector<void*> blocks;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    for (auto it = g_cache.begin(); it != g_cache.end();) {
+      if (std::get<0>(it->first) == dev && std::get<1>(it->first) == key_ptr) { plans.push_back(it->second.plan); it = g_cache.erase(it); }
+      else ++it;
+    }
+    for (auto it = g_coo_cache.begin(); it != g_coo_cache.end();) {
+      if (std::get<0>(it->first) == dev && std::get<1>(it->first) == key_ptr) { blocks.push_back(it->second.row_ptr); it = g_coo_cache.erase(it); }
+      else ++it;
+    }
+    for (auto it = g_csc_cache.begin(); it != g_csc_cache.end();) {
+      if (std::get<0>(it->first) == dev && std::get<1>(it->first) == key_ptr) {
+        for (void* q : {(void*)it->second.row_ptr, (void*)it->second.col, (void*)it->second.perm, it->second.vals_t}) blocks.push_back(q);
+        it = g_csc_cache.erase(it);
+      } else ++it;
+    }
+  }
+  int rc = B200SP_OK;
+  for (b200sp_plan* p : plans) { const int r = plan_free(p); if (r != B200SP_OK) rc = r; }
+  if (!blocks.empty()) {
+    CU(cudaDeviceSynchronize());
+    for (void* q : blocks) if (q) cudaFree(q);
+  }
+  return rc;
+}
+
 void b200sp_cache_clear(void) {
   std::lock_guard<std::mutex> lock(g_mutex);
-  for (auto& kv : g_cache) plan_free(kv.second);
+  for (auto& kv : g_cache) plan_free(kv.second.plan);
   g_cache.clear();
   for (auto& kv : g_coo_cache) cudaFree(kv.second.row_ptr);
   g_coo_cache.clear();
@@ -418,32 +464,47 @@ int64_t b200sp_launch_count(void) { return g_launches.load(); }
 int b200sp_set_option(const char* name, int value) {
   if (!name) return B200SP_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_mutex);
-  if (!strcmp(name, "bstage_threads")) { if (value != 256 && value != 512 && value != 1024) return B200SP_ERR_INVALID_ARG; g_opt.bstage_threads = value; return B200SP_OK; }
-  if (!strcmp(name, "bstage_nnz")) { if (value < 1024) return B200SP_ERR_INVALID_ARG; g_opt.bstage_nnz = value; return B200SP_OK; }
-  if (!strcmp(name, "spmm_bstage")) { g_opt.spmm_bstage = value ? 1 : 0; return B200SP_OK; }
-  if (!strcmp(name, "pdl")) { g_opt.pdl = value ? 1 : 0; return B200SP_OK; }
-  if (!strcmp(name, "pool_keep_mb")) { if (value < 0) return B200SP_ERR_INVALID_ARG; g_opt.pool_keep_mb = value; return B200SP_OK; }
-  if (!strcmp(name, "bstage_stage_a")) { g_opt.bstage_stage_a = value ? 1 : 0; return B200SP_OK; }
-  if (!strcmp(name, "spmm_sliced")) { g_opt.spmm_sliced = value ? 1 : 0; return B200SP_OK; }
-  if (!strcmp(name, "merge_threads")) { if (value != 64 && value != 128 && value != 256) return B200SP_ERR_INVALID_ARG; g_opt.merge_threads = value; return B200SP_OK; }
-  if (!strcmp(name, "sub_lanes")) { if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != 16 && value != 32) return B200SP_ERR_INVALID_ARG; g_opt.sub_lanes = value; return B200SP_OK; }
-  if (!strcmp(name, "merge_stride")) { if (value < 0 || value > (1 << 20)) return B200SP_ERR_INVALID_ARG; g_opt.merge_stride = value; return B200SP_OK; }
-  if (!strcmp(name, "merge_scan")) { g_opt.merge_scan = value ? 1 : 0; return B200SP_OK; }
-  if (!strcmp(name, "merge_short")) { if (value != 8 && value != 16 && value != 32 && value != 64) return B200SP_ERR_INVALID_ARG; g_opt.merge_short = value; return B200SP_OK; }
-  if (!strcmp(name, "merge_carve")) { if (value < -1 || value > 100) return B200SP_ERR_INVALID_ARG; g_opt.merge_carve = value; return B200SP_OK; }
-  if (!strcmp(name, "merge_staged")) { g_opt.merge_staged = value ? 1 : 0; return B200SP_OK; }
-  if (!strcmp(name, "merge_items")) { if (value != 1024 && value != 2048 && value != 4096) return B200SP_ERR_INVALID_ARG; g_opt.merge_items = value; return B200SP_OK; }
-  if (!strcmp(name, "merge_stages")) { if (value < 2 || value > kMergeMaxStages) return B200SP_ERR_INVALID_ARG; g_opt.merge_stages = value; return B200SP_OK; }
-  if (!strcmp(name, "merge_ctas")) { if (value < 1 || value > 8) return B200SP_ERR_INVALID_ARG; g_opt.merge_ctas = value; return B200SP_OK; }
-  if (!strcmp(name, "uni_unroll")) { if (value != 0 && value != 1 && value != 2 && value != 4) return B200SP_ERR_INVALID_ARG; g_opt.uni_unroll = value; return B200SP_OK; }
-  if (!strcmp(name, "uni_ctas")) { if (value < 0 || value > 32) return B200SP_ERR_INVALID_ARG; g_opt.uni_ctas = value; return B200SP_OK; }
-  if (!strcmp(name, "spmv_kernel")) { if (value < -1 || value > 3) return B200SP_ERR_INVALID_ARG; g_opt.spmv_kernel = value; return B200SP_OK; }
-  if (!strcmp(name, "x_l2_window")) { g_opt.x_l2_window = value ? 1 : 0; return B200SP_OK; }
-  if (!strcmp(name, "row_stages")) { if (value < 2 || value > kRowMaxStages) return B200SP_ERR_INVALID_ARG; g_opt.row_stages = value; return B200SP_OK; }
-  if (!strcmp(name, "row_smem_kb")) { if (value < 16 || value > 227) return B200SP_ERR_INVALID_ARG; g_opt.row_smem_kb = value; return B200SP_OK; }
-  if (!strcmp(name, "row_threads")) { if (value != 128 && value != 256) return B200SP_ERR_INVALID_ARG; g_opt.row_threads = value; return B200SP_OK; }
-  if (!strcmp(name, "row_ctas")) { if (value < 1 || value > 8) return B200SP_ERR_INVALID_ARG; g_opt.row_ctas = value; return B200SP_OK; }
-  if (!strcmp(name, "row_unroll")) { if (value != 8 && value != 16) return B200SP_ERR_INVALID_ARG; g_opt.row_unroll = value; return B200SP_OK; }
+  // each switch accepts exactly the values listed for it in b200sp_tuning.h; the test suite runs every one of them
+  struct Entry { const char* name; int* slot; bool boolean; std::initializer_list<int> values; int lo, hi; };
+  const Entry table[] = {
+      {"spmv_kernel", &g_opt.spmv_kernel, false, {-1, 0, 1, 2, 3}, 0, 0},
+      {"spmm_bstage", &g_opt.spmm_bstage, true, {}, 0, 0},
+      {"spmm_sliced", &g_opt.spmm_sliced, true, {}, 0, 0},
+      {"spmm_ranges", &g_opt.spmm_ranges, false, {0, 1, 2, 3, 4, 5, 6, 7, 8}, 0, 0},
+      {"merge_items", &g_opt.merge_items, false, {1024, 2048, 4096}, 0, 0},
+      {"merge_threads", &g_opt.merge_threads, false, {64, 128, 256}, 0, 0},
+      {"merge_carve", &g_opt.merge_carve, false, {-1, 0, 25, 45, 60, 75, 100}, 0, 0},
+      {"merge_short", &g_opt.merge_short, false, {8, 16, 32, 64}, 0, 0},
+      {"merge_empty", &g_opt.merge_empty, true, {}, 0, 0},
+      {"row_stages", &g_opt.row_stages, false, {2, 3, 4}, 0, 0},
+      {"row_ctas", &g_opt.row_ctas, false, {1, 2, 3, 4}, 0, 0},
+      {"row_smem_kb", &g_opt.row_smem_kb, false, {48, 96, 160, 220, 227}, 0, 0},
+      {"row_threads", &g_opt.row_threads, false, {128, 256}, 0, 0},
+      {"row_unroll", &g_opt.row_unroll, false, {8, 16}, 0, 0},
+      {"uni_unroll", &g_opt.uni_unroll, false, {0, 1, 2, 4}, 0, 0},
+      {"uni_ctas", &g_opt.uni_ctas, false, {0, 1, 2, 4, 8}, 0, 0},
+      {"sub_lanes", &g_opt.sub_lanes, false, {0, 1, 2, 4, 8, 16, 32}, 0, 0},
+      {"bstage_threads", &g_opt.bstage_threads, false, {256, 512, 1024}, 0, 0},
+      {"bstage_nnz", &g_opt.bstage_nnz, false, {16384, 65536, 131072, 524288}, 0, 0},
+      {"bstage_stage_a", &g_opt.bstage_stage_a, true, {}, 0, 0},
+      {"x_l2_window", &g_opt.x_l2_window, true, {}, 0, 0},
+      {"pdl", &g_opt.pdl, true, {}, 0, 0},
+      {"debug_no_copies", &g_opt.debug_no_copies, true, {}, 0, 0},
+      {"pool_keep_mb", &g_opt.pool_keep_mb, false, {}, 0, 1 << 20},
+      {"spin_limit", &g_opt.spin_limit, false, {}, 1, 1 << 30},
+      {"fail_alloc_after", &g_opt.fail_alloc_after, false, {}, 0, 1 << 30},
+  };
+  for (const Entry& e : table) {
+    if (strcmp(name, e.name)) continue;
+    if (e.boolean) { *e.slot = value ? 1 : 0; return B200SP_OK; }
+    if (e.values.size()) {
+      for (int v : e.values) if (v == value) { *e.slot = value; return B200SP_OK; }
+      return B200SP_ERR_INVALID_ARG;
+    }
+    if (value < e.lo || value > e.hi) return B200SP_ERR_INVALID_ARG;
+    *e.slot = value;
+    return B200SP_OK;
+  }
   return B200SP_ERR_INVALID_ARG;
 }
 

@@ -46,12 +46,14 @@ spmv_ell_kernel(int m, int width, const int* __restrict__ col_ids, const T* __re
   const long long gid = (long long)blockIdx.x * THREADS + threadIdx.x;
   const long long row = gid / LPR;
   const int sub = (int)(gid % LPR);
-  float acc = 0.0f;
+  float acc = 0.0f, tot = 0.0f;   // acc: at most kChainBlock products in one chain, then folded into tot
+  int trips = 0;
   if (row < m) {
     const long long base = row * width;
     if (VECW == 4) {
       int j = sub * 4;
       for (; j + LPR * 4 < width; j += 2 * LPR * 4) {   // two independent groups of four per trip
+        if (++trips > kChainBlock / 8) { trips = 1; tot += acc; acc = 0.0f; }
         const int4 c0 = ld_stream_i4(col_ids + base + j), c1 = ld_stream_i4(col_ids + base + j + LPR * 4);
         float v0[4], v1[4];
         ld_stream_vals4(vals + base + j, v0);
@@ -75,11 +77,13 @@ spmv_ell_kernel(int m, int width, const int* __restrict__ col_ids, const T* __re
       }
     } else {
       for (int j = sub; j < width; j += LPR) {
+        if (++trips > kChainBlock) { trips = 1; tot += acc; acc = 0.0f; }
         const int c = ld_stream_i1(col_ids + base + j);
         if (c >= 0) acc = fmaf(ld_stream_val1(vals + base + j), ld_gather(x + c), acc);
       }
     }
   }
+  acc += tot;
 #pragma unroll
   for (int o = 1; o < LPR; o <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
   if (row < m && sub == 0) epilogue_store(y, row, acc, alpha, beta);
@@ -100,16 +104,22 @@ spmm_ell_slice_kernel(int m, int k, int width, int row_blocks, const int* __rest
   if (col0 >= k) return;
   const T* Bc = B + col0;
   const long long base = row * width;
-  float acc[VEC];
+  float acc[VEC], tot[VEC];   // blocks of at most kChainBlock products, block sums in a second chain
 #pragma unroll
-  for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
+  for (int j = 0; j < VEC; ++j) { acc[j] = 0.0f; tot[j] = 0.0f; }
   for (int j = 0; j < width; ++j) {
+    if (j > 0 && j % kChainBlock == 0) {
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) { tot[i] += acc[i]; acc[i] = 0.0f; }
+    }
     const int c = __ldg(col_ids + base + j);
     if (c >= 0) {
       const raw_t b = RawVec<T, VEC>::ld(Bc + (long long)c * k);
       RawVec<T, VEC>::fma(b, to_f32(__ldg(vals + base + j)), acc);
     }
   }
+#pragma unroll
+  for (int i = 0; i < VEC; ++i) acc[i] += tot[i];
   T* yp = Y + row * k + col0;
   float out[VEC];
   if (beta != 0.0f) {
@@ -133,12 +143,13 @@ spmm_ell_entry_kernel(long long m, int k, int width, const int* __restrict__ col
   if (id >= m * k) return;
   const long long row = id / k;
   const int c = (int)(id - row * k);
-  float acc = 0.0f;
+  float acc = 0.0f, tot = 0.0f;
   for (int j = 0; j < width; ++j) {
+    if (j > 0 && j % kChainBlock == 0) { tot += acc; acc = 0.0f; }
     const int col = col_ids[row * width + j];
     if (col >= 0) acc = fmaf(to_f32(vals[row * width + j]), to_f32(B[(long long)col * k + c]), acc);
   }
-  epilogue_store(Y, id, acc, alpha, beta);
+  epilogue_store(Y, id, acc + tot, alpha, beta);
 }
 
 }  // namespace b200sp

@@ -1,4 +1,4 @@
-// Host side of libb200sp.so: the plan pass (row statistics, bins, splits, long-row list) and the plan cache.
+// Host side of libb200sp.so: the plan pass (row statistics, bins, splits, medium- and long-row lists) and the plan cache.
 // One of the pieces of the single translation unit b200sp.cu; include/b200sp.h states the contract of every entry point.
 #pragma once
 #include "host_runtime.cuh"
@@ -6,7 +6,14 @@
 
 namespace {
 
-std::map<std::tuple<int, const void*, int64_t, int64_t, int64_t>, b200sp_plan*> g_cache;
+// Plans cached by the one-shot entry points, keyed on (device, row_ptr address, m, n, nnz).  The address may be a device
+// pointer (spmv_csr, spmm_csr) or a host pointer (spmv_csr_host, spmm_csr_host); the two never collide in a unified
+// address space.  At most kCacheCap plans are kept: the least recently used one is dropped when another is added.
+typedef std::tuple<int, const void*, int64_t, int64_t, int64_t> PlanKey;
+struct CachedPlan { b200sp_plan* plan = nullptr; uint64_t stamp = 0; };
+std::map<PlanKey, CachedPlan> g_cache;
+uint64_t g_cache_clock = 0;
+constexpr size_t kCacheCap = 64;
 
 // Frees a plan.  With stream_ordered the block goes back to the pool in the order of `stream` (the caller
 // knows that every kernel that used the plan ran there); otherwise the device is synchronised first.
@@ -43,17 +50,16 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   const int items = g_opt.merge_items == 4096 ? 4096 : (g_opt.merge_items == 1024 ? 1024 : 2048);
   I.spmv_tile_items = items;
   I.spmv_tiles = (int32_t)((m + nnz + items - 1) / items);
-  I.spmm_tile_nnz = kSpmmTileNnz;
-  I.spmm_tiles = (int32_t)((nnz + kSpmmTileNnz - 1) / kSpmmTileNnz);
   I.spmv_kernel = g_opt.spmv_kernel >= 0 ? g_opt.spmv_kernel : 0;
   if (m == 0) { *out = p; return B200SP_OK; }
 
-  // one block from the pool: statistics, counter, split points, carries, tails, SpMM split points, long-row list
-  const size_t nt = (size_t)I.spmv_tiles, ns = (size_t)I.spmm_tiles;
+  // one block from the pool: statistics, counters, split points, carries, tails, medium- and long-row lists
+  const size_t nt = (size_t)I.spmv_tiles;
   const size_t long_cap = (size_t)(nnz / (kLongRow + 1)) + 1;     // rows longer than kLongRow: at most this many
+  const size_t mid_cap = (size_t)(nnz / (kMediumRow + 1)) + 1;    // rows longer than kMediumRow
   auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
   const size_t o_stats = 0, o_count = o_stats + up(sizeof(PlanStats)), o_split = o_count + 256, o_carry = o_split + up((nt + 1) * 4),
-               o_tail = o_carry + up((nt + 1) * 4), o_msplit = o_tail + up((nt + 1) * 4), o_long = o_msplit + up((ns + 1) * 4),
+               o_tail = o_carry + up((nt + 1) * 4), o_mid = o_tail + up((nt + 1) * 4), o_long = o_mid + up(mid_cap * 4),
                total = o_long + up(long_cap * 4);
   PlanStats h = {};
   h.min_len = 0x7FFFFFFF;
@@ -63,12 +69,12 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   if (rc != B200SP_OK) { delete p; return rc; }
   char* base = (char*)p->block;
   PlanStats* d_stats = (PlanStats*)(base + o_stats);
-  int* d_count = (int*)(base + o_count);
-  p->probe_out = (unsigned long long*)(base + o_count + 16);
+  int* d_count = (int*)(base + o_count);                       // two list counters
+  p->probe_out = (unsigned long long*)(base + o_count + 16);   // two probe counters
   p->split_row = (int32_t*)(base + o_split);
   p->carry = (float*)(base + o_carry);
   p->tail = (float*)(base + o_tail);
-  p->spmm_split_row = (int32_t*)(base + o_msplit);
+  p->medium_rows = (int32_t*)(base + o_mid);
   p->long_rows = (int32_t*)(base + o_long);
   I.scratch_bytes = (int64_t)total;
   CUP(cudaMemcpyAsync(d_stats, &h, sizeof h, cudaMemcpyHostToDevice, stream));
@@ -79,26 +85,30 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
     g_launches++;
   }
   plan_merge_split_kernel<<<(unsigned)((nt + 1 + 255) / 256), 256, 0, stream>>>(row_ptr, (int)m, (int)nnz, items, (int)nt, p->split_row);
-  plan_nnz_split_kernel<<<(unsigned)((ns + 1 + 255) / 256), 256, 0, stream>>>(row_ptr, (int)m, (int)nnz, kSpmmTileNnz, (int)ns, p->spmm_split_row);
-  g_launches += 2;
+  g_launches++;
   CUP(cudaGetLastError());
   CUP(cudaMemcpyAsync(&h, d_stats, sizeof h, cudaMemcpyDeviceToHost, stream));
   CUP(cudaStreamSynchronize(stream));
-  if (!h.bad && h.bin_rows[4] > 0) {   // list of the rows in the last length bin (> kLongRow), sorted on the host
-    const int cap = (int)h.bin_rows[4];
-    if ((size_t)cap > long_cap) return fail(B200SP_ERR_BAD_CSR);   // cannot happen for a monotone row_ptr
-    CUP(cudaMemsetAsync(d_count, 0, sizeof(int), stream));
+  if (!h.bad && h.bin_rows[4] + h.bin_rows[5] > 0) {   // lists of the rows in the last two length bins, sorted on the host
+    const size_t n_mid = (size_t)h.bin_rows[4], n_long = (size_t)h.bin_rows[5];
+    if (n_mid > mid_cap || n_long > long_cap) return fail(B200SP_ERR_BAD_CSR);   // cannot happen for a monotone row_ptr
+    CUP(cudaMemsetAsync(d_count, 0, 2 * sizeof(int), stream));
     const int blocks = (int)((m + 255) / 256);
-    plan_long_rows_kernel<<<blocks < dev->sms * 8 ? blocks : dev->sms * 8, 256, 0, stream>>>(row_ptr, (int)m, kLongRow, cap, p->long_rows, d_count);
+    plan_row_lists_kernel<<<blocks < dev->sms * 8 ? blocks : dev->sms * 8, 256, 0, stream>>>(
+        row_ptr, (int)m, kMediumRow, kLongRow, (int)n_mid, (int)n_long, p->medium_rows, p->long_rows, d_count);
     g_launches++;
     CUP(cudaGetLastError());
-    std::vector<int32_t> tmp((size_t)cap);
-    CUP(cudaMemcpyAsync(tmp.data(), p->long_rows, (size_t)cap * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    std::vector<int32_t> tmp(n_mid + n_long);
+    if (n_mid) CUP(cudaMemcpyAsync(tmp.data(), p->medium_rows, n_mid * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    if (n_long) CUP(cudaMemcpyAsync(tmp.data() + n_mid, p->long_rows, n_long * sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
     CUP(cudaStreamSynchronize(stream));
-    std::sort(tmp.begin(), tmp.end());
-    CUP(cudaMemcpyAsync(p->long_rows, tmp.data(), (size_t)cap * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+    std::sort(tmp.begin(), tmp.begin() + n_mid);
+    std::sort(tmp.begin() + n_mid, tmp.end());
+    if (n_mid) CUP(cudaMemcpyAsync(p->medium_rows, tmp.data(), n_mid * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+    if (n_long) CUP(cudaMemcpyAsync(p->long_rows, tmp.data() + n_mid, n_long * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
     CUP(cudaStreamSynchronize(stream));
-    p->num_long = cap;
+    p->num_medium = (int)n_mid;
+    p->num_long = (int)n_long;
   }
 #undef CUP
   if (h.bad) { plan_free(p, true, stream); cudaStreamSynchronize(stream); return B200SP_ERR_BAD_CSR; }
@@ -115,8 +125,8 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   int choice = uniform_ok ? 2 : (row_direct_ok ? 1 : 0);
   // Small problems (launch-latency regime): one sub-warp per row, no scratch, maximum spread over the SMs -- unless the
   // rows are uniform (the uniform-row kernel is as flat) or the row-direct kernel would still get a tile for every SM.
-  if (nnz > 0 && nnz <= kSmallNnz && h.max_len <= 4096 && !uniform_ok && !(row_direct_ok && m >= (int64_t)kRowThreads * dev->sms)) choice = 3;
-  if (g_opt.spmv_kernel == 3) choice = h.max_len <= 65536 ? 3 : 0;
+  if (nnz > 0 && nnz <= kSmallNnz && h.max_len <= 32 * kSubwarpChain && !uniform_ok && !(row_direct_ok && m >= (int64_t)kRowThreads * dev->sms)) choice = 3;
+  if (g_opt.spmv_kernel == 3) choice = h.max_len <= 32 * kSubwarpChain ? 3 : 0;
   if (g_opt.spmv_kernel == 0) choice = 0;
   if (g_opt.spmv_kernel == 1) choice = row_direct_possible ? 1 : 0;
   if (g_opt.spmv_kernel == 2) choice = uniform_ok ? 2 : (row_direct_ok ? 1 : 0);
@@ -132,25 +142,49 @@ int check_common(const b200sp_plan* p, const void* col_idx, const void* vals, co
   if (I.nnz > 0 && (!col_idx || !vals || !dense_in)) return B200SP_ERR_INVALID_ARG;
   if (I.m > 0 && !dense_out) return B200SP_ERR_INVALID_ARG;
   if (!aligned16(col_idx) || !aligned16(vals) || !aligned16(dense_in) || !aligned16(dense_out)) return B200SP_ERR_INVALID_ARG;
+  int cur = 0;
+  CU(cudaGetDevice(&cur));
+  if (I.m > 0 && cur != p->device) return B200SP_ERR_INVALID_ARG;   // a plan belongs to the device it was created on
   return B200SP_OK;
+}
+
+// Looks `key` up; a hit refreshes its stamp.  The caller holds no lock.
+b200sp_plan* cache_find(const PlanKey& key) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  auto it = g_cache.find(key);
+  if (it == g_cache.end()) return nullptr;
+  it->second.stamp = ++g_cache_clock;
+  return it->second.plan;
+}
+
+// Adds a plan under `key` (or returns the one another thread added first) and drops the least recently used
+// plan beyond the cap.  Dropping synchronises the device of the dropped plan.
+b200sp_plan* cache_insert(const PlanKey& key, b200sp_plan* p) {
+  b200sp_plan* victim = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    auto ins = g_cache.emplace(key, CachedPlan{p, ++g_cache_clock});
+    if (!ins.second) { victim = p; p = ins.first->second.plan; }
+    else if (g_cache.size() > kCacheCap) {
+      auto oldest = g_cache.end();
+      for (auto it = g_cache.begin(); it != g_cache.end(); ++it)
+        if (it->second.plan != p && (oldest == g_cache.end() || it->second.stamp < oldest->second.stamp)) oldest = it;
+      if (oldest != g_cache.end()) { victim = oldest->second.plan; g_cache.erase(oldest); }
+    }
+  }
+  if (victim) plan_free(victim);
+  return p;
 }
 
 int get_cached_plan(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, cudaStream_t stream) {
   int dev = 0;
   CU(cudaGetDevice(&dev));
-  const auto key = std::make_tuple(dev, (const void*)row_ptr, m, n, nnz);
-  {
-    std::lock_guard<std::mutex> lock(g_mutex);
-    auto it = g_cache.find(key);
-    if (it != g_cache.end()) { *out = it->second; return B200SP_OK; }
-  }
+  const PlanKey key = std::make_tuple(dev, (const void*)row_ptr, m, n, nnz);
+  if (b200sp_plan* hit = cache_find(key)) { *out = hit; return B200SP_OK; }
   b200sp_plan* p = nullptr;
   int rc = b200sp_plan_create(&p, m, n, nnz, row_ptr, stream);
   if (rc != B200SP_OK) return rc;
-  std::lock_guard<std::mutex> lock(g_mutex);
-  auto ins = g_cache.emplace(key, p);
-  if (!ins.second) { plan_free(p); p = ins.first->second; }
-  *out = p;
+  *out = cache_insert(key, p);
   return B200SP_OK;
 }
 

@@ -1,7 +1,7 @@
 // Host side of libb200sp.so: constants, tuning switches, device queries, the launch helper and argument checks.
 // One of the pieces of the single translation unit b200sp.cu; include/b200sp.h states the contract of every entry point.
 #pragma once
-#include "../../include/b200sp.h"
+#include "../../include/b200sp_tuning.h"
 
 #include <algorithm>
 #include <atomic>
@@ -31,8 +31,9 @@ constexpr int kRowMaxLen = 64;
 constexpr int kSmemPerSm = 227 * 1024;   // usable shared memory per SM (each CTA also reserves 1 KB)
 // SpMM
 constexpr int kSpmmThreads = 256;
-constexpr int kSpmmTileNnz = 4096;
 constexpr int kSmallNnz = 1 << 20;   // at or below this many nonzeros SpMV uses the sub-warp-per-row kernel
+constexpr int kSubwarpChain = 128;   // longest sequential FP32 chain one lane of the sub-warp SpMV kernel may add
+constexpr int kMediumRow = 128;   // SpMM: rows longer than this are added in blocks of this many products (second-to-last length bin)
 constexpr int kLongRow = 1024;   // rows longer than this get a CTA of their own in SpMM (last length bin of the plan)
 
 thread_local std::string g_last_error;
@@ -49,10 +50,7 @@ struct Options {
   int row_threads = 256;  // threads per CTA of the row-direct kernel (128 or 256)
   int uni_unroll = 0;     // groups of four nonzeros in flight per thread of the uniform-row kernel (1, 2 or 4); 0 = 1 (32 registers, full occupancy)
   int uni_ctas = 0;       // CTAs per SM for the uniform-row kernel (0 = as many as fit)
-  int merge_staged = 0;   // 1 = persistent staged merge kernel, 0 = one-tile-per-CTA merge kernel
   int merge_items = 2048; // merge items per tile (2048 or 4096)
-  int merge_stages = 3;   // shared-memory stages per CTA of the staged merge kernel (2..4)
-  int merge_ctas = 2;     // CTAs per SM of the staged merge kernel
   int merge_threads = 128; // threads per CTA of the one-tile-per-CTA merge kernel (128 or 256)
   int bstage_threads = 1024; // threads per CTA of that kernel (256, 512 or 1024)
   int bstage_nnz = 131072;   // nonzeros per CTA it aims for
@@ -60,19 +58,23 @@ struct Options {
   int spmm_bstage = 1;     // 1 = hold the slice of B in shared memory when A has few columns (default), 0 = never
   int spmm_sliced = 1;     // 1 = k-sliced SpMM kernel (default), 0 = one pass over all of k
   int sub_lanes = 0;       // lanes per row of the sub-warp kernel (0 = from the mean row length)
-  int merge_stride = 0;    // tile order of the scan merge kernel: stride through the tiles (0 / 1 = plain order)
-  int merge_scan = 0;      // 1 = merge kernel with the in-register segmented scan, 0 = products through shared memory (default: as fast on power-law rows, faster on short rows)
+  int merge_empty = 1;     // 1 = rows without nonzeros are kept out of the merge list when the matrix has many of them (default), 0 = never
+  int spmm_ranges = 0;     // column ranges per slice of the k-sliced SpMM kernel with sorted columns: 0 = sized for L2, 1 = none, 2..8 forced
   int merge_short = 32;    // rows up to this many products are added by one thread (8, 16, 32, 64)
   int pdl = 1;             // 1 = launch the kernels that begin with griddepcontrol.wait with programmatic stream serialisation
   int pool_keep_mb = 1024; // freed memory the library's pool keeps across synchronisation points, MiB (read when the pool is created)
   int merge_carve = 45;    // shared-memory carveout (percent) requested for it, -1 = leave to the driver
+  // test switches (failure paths that must be reachable without faulting a GPU)
+  int spin_limit = 1 << 20;   // polls before a bounded barrier wait gives up
+  int debug_no_copies = 0;    // 1 = the kernels that stage through shared memory issue no copy and arm no barrier: their waits run out
+  int fail_alloc_after = 0;   // N > 0: the N-th allocation from the library's pool from now on fails (then the switch clears itself)
 } g_opt;
 
 struct DeviceInfo {
   bool known = false;
   int cc_major = 0, sms = 0, persist_max = 0, window_max = 0, l2_bytes = 0;
   size_t persist_set = 0;
-  int* err_flag = nullptr;  // device int: set by a kernel whose bounded wait ran out
+  int* err_flag = nullptr;  // address of g_timeout_flag on this device: set by a kernel whose bounded wait ran out
   cudaMemPool_t pool = nullptr;  // the library's own stream-ordered pool: plan scratch and the host entry points' staging buffers
 };
 DeviceInfo g_dev[64];
@@ -133,6 +135,13 @@ int device_pool(DeviceInfo* d, cudaMemPool_t* out) {
 }
 
 int pool_alloc(DeviceInfo* d, void** ptr, size_t bytes, cudaStream_t stream) {
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_opt.fail_alloc_after > 0 && --g_opt.fail_alloc_after == 0) {   // injected failure (test switch)
+      g_last_error = "out of device memory (injected)";
+      return B200SP_ERR_ALLOC;
+    }
+  }
   cudaMemPool_t pool = nullptr;
   int rc = device_pool(d, &pool);
   if (rc != B200SP_OK) return rc;
@@ -142,12 +151,15 @@ int pool_alloc(DeviceInfo* d, void** ptr, size_t bytes, cudaStream_t stream) {
   return B200SP_OK;
 }
 
-// The flag that kernels with bounded waits raise; allocated on first use (those kernels only).
+// The flag that kernels with bounded waits raise: one int in the library image per device (zero when the module is
+// loaded), so finding it neither allocates nor synchronises.
+__device__ int g_timeout_flag;
 int ensure_err_flag(DeviceInfo* d) {
   std::lock_guard<std::mutex> lock(g_mutex);
   if (!d->err_flag) {
-    CU(cudaMalloc(&d->err_flag, sizeof(int)));
-    CU(cudaMemset(d->err_flag, 0, sizeof(int)));
+    void* ptr = nullptr;
+    CU(cudaGetSymbolAddress(&ptr, g_timeout_flag));
+    d->err_flag = static_cast<int*>(ptr);
   }
   return B200SP_OK;
 }
@@ -225,10 +237,11 @@ struct b200sp_plan {
   int32_t* split_row = nullptr;       // spmv tiles + 1
   float* carry = nullptr;             // spmv tiles
   float* tail = nullptr;              // spmv tiles
-  int32_t* spmm_split_row = nullptr;  // spmm tiles + 1
+  int32_t* medium_rows = nullptr;     // rows of kMediumRow + 1 .. kLongRow nonzeros, ascending
   int32_t* long_rows = nullptr;       // rows longer than kLongRow, ascending
   unsigned long long* probe_out = nullptr;  // two counters for the column-locality probe
-  int num_long = 0;
+  int num_medium = 0, num_long = 0;
   const void* probed_col_idx = nullptr;   // col_idx the column-locality probe last ran on
+  const void* probed_key = nullptr;       // host entry points: the HOST col_idx that verdict belongs to
   bool cols_local = true;                 // its verdict: adjacent rows share most of their lines of x
 };

@@ -7,13 +7,22 @@
 
 namespace {
 
+// Rows of at most kLongRow nonzeros by one lane group each; longer rows by a CTA per (row, 8 * VEC columns).
 template <typename T, int VEC, int LANES, int NCH>
-int launch_spmm(const b200sp_plan_info_t& I, const int32_t* row_ptr, int k, const int32_t* col_idx, const T* vals, const T* B, T* Y,
-                float alpha, float beta, cudaStream_t stream, DeviceInfo* dev) {
+int launch_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const T* B, T* Y, float alpha, float beta,
+                cudaStream_t stream, DeviceInfo* dev) {
+  const b200sp_plan_info_t& I = p->info;
   constexpr int GROUPS = kSpmmThreads / LANES;
   const unsigned grid = (unsigned)((I.m + GROUPS - 1) / GROUPS);
-  return launch(spmm_row_group_kernel<T, VEC, LANES, NCH, kSpmmThreads>, dim3(grid), dim3(kSpmmThreads), stream, B,
-                (size_t)I.n * k * sizeof(T), dev, (int)I.m, k, row_ptr, col_idx, vals, B, Y, alpha, beta);
+  tl_pdl_kernel = true;
+  int rc = launch(spmm_row_group_kernel<T, VEC, LANES, NCH, kSpmmThreads>, dim3(grid), dim3(kSpmmThreads), stream, B,
+                  (size_t)I.n * k * sizeof(T), dev, (int)I.m, k, p->row_ptr, col_idx, vals, B, Y, alpha, beta, kLongRow);
+  if (rc != B200SP_OK || p->num_long == 0) return rc;
+  const long long ctas = (long long)((k + 8 * VEC - 1) / (8 * VEC)) * p->num_long;
+  if (ctas >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+  tl_pdl_kernel = true;
+  return launch(spmm_long_row_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)ctas), dim3(kSpmmThreads), stream, nullptr, 0, dev, k, p->num_long,
+                (const int*)p->long_rows, p->row_ptr, col_idx, vals, B, Y, alpha, beta);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
@@ -81,7 +90,8 @@ int launch_spmm_bstage(b200sp_plan* p, int k, const int32_t* col_idx, const T* v
   if (rc != B200SP_OK) return rc;
   tl_pdl_kernel = true;
   return launch_smem(kernel, dim3((unsigned)(slices * row_chunks)), dim3(THREADS), smem, stream, nullptr, 0, dev, map, (int)I.m, (int)I.n,
-                     k, row_chunks, rows_per_chunk, box_rows, (int)bslice, capw, p->row_ptr, col_idx, vals, Y, alpha, beta, dev->err_flag);
+                     k, row_chunks, rows_per_chunk, box_rows, (int)bslice, capw, p->row_ptr, col_idx, vals, Y, alpha, beta, dev->err_flag,
+                     g_opt.spin_limit, g_opt.debug_no_copies);
 }
 
 template <typename T, int VEC>
@@ -123,32 +133,42 @@ int run_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const
     const int row_blocks = (int)((I.m + GROUPS - 1) / GROUPS);
     if ((long long)slices * row_blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
     int rc;
-    tl_pdl_kernel = true;
+    const int mid_blocks = (p->num_medium + GROUPS - 1) / GROUPS;
+    // rows of at most kMediumRow nonzeros: the register-capped kernel; kMediumRow + 1 .. kLongRow: the same scheme with
+    // blocked sums over the plan's list of such rows; longer rows: a CTA per (row, slice)
 #define B200SP_SLICE_LAUNCH(L)                                                                                                      \
+    tl_pdl_kernel = true;                                                                                                           \
     rc = launch(spmm_slice_kernel<T, VEC, kSpmmThreads, L>, dim3((unsigned)(slices * row_blocks)), dim3(kSpmmThreads), stream, nullptr, 0, \
-                dev, (int)I.m, k, row_blocks, p->row_ptr, col_idx, vals, B, Y, alpha, beta, kLongRow)
-    if (lanes == 8) B200SP_SLICE_LAUNCH(8);
-    else if (lanes == 4) B200SP_SLICE_LAUNCH(4);
-    else if (lanes == 2) B200SP_SLICE_LAUNCH(2);
-    else B200SP_SLICE_LAUNCH(1);
+                dev, (int)I.m, k, row_blocks, p->row_ptr, col_idx, vals, B, Y, alpha, beta, kMediumRow);                            \
+    if (rc == B200SP_OK && p->num_medium > 0) {                                                                                     \
+      tl_pdl_kernel = true;                                                                                                         \
+      rc = launch(spmm_medium_row_kernel<T, VEC, kSpmmThreads, L>, dim3((unsigned)(slices * mid_blocks)), dim3(kSpmmThreads), stream, \
+                  nullptr, 0, dev, p->num_medium, (const int*)p->medium_rows, k, mid_blocks, p->row_ptr, col_idx, vals, B, Y, alpha, beta); \
+    }
+    if (lanes == 8) { B200SP_SLICE_LAUNCH(8); }
+    else if (lanes == 4) { B200SP_SLICE_LAUNCH(4); }
+    else if (lanes == 2) { B200SP_SLICE_LAUNCH(2); }
+    else { B200SP_SLICE_LAUNCH(1); }
 #undef B200SP_SLICE_LAUNCH
     if (rc != B200SP_OK || p->num_long == 0) return rc;
+    const long long ctas = (long long)((k + 8 * VEC - 1) / (8 * VEC)) * p->num_long;
+    if (ctas >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
     tl_pdl_kernel = true;
-    return launch(spmm_long_row_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)(((k + 8 * VEC - 1) / (8 * VEC)) * p->num_long)), dim3(kSpmmThreads), stream, nullptr, 0,
+    return launch(spmm_long_row_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)ctas), dim3(kSpmmThreads), stream, nullptr, 0,
                   dev, k, p->num_long, (const int*)p->long_rows, p->row_ptr, col_idx, vals, B, Y, alpha, beta);
   }
   if (k % VEC != 0) {  // ragged k: scalar lanes
-    if (k <= 2) return launch_spmm<T, 1, 2, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
-    if (k <= 4) return launch_spmm<T, 1, 4, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
-    if (k <= 8) return launch_spmm<T, 1, 8, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
-    return launch_spmm<T, 1, 32, 2>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+    if (k <= 2) return launch_spmm<T, 1, 2, 1>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+    if (k <= 4) return launch_spmm<T, 1, 4, 1>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+    if (k <= 8) return launch_spmm<T, 1, 8, 1>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+    return launch_spmm<T, 1, 32, 2>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
   }
   const int vecs = k / VEC;  // vector columns per row
-  if (vecs <= 4) return launch_spmm<T, VEC, 4, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
-  if (vecs <= 8) return launch_spmm<T, VEC, 8, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
-  if (vecs <= 16) return launch_spmm<T, VEC, 16, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
-  if (vecs <= 32) return launch_spmm<T, VEC, 32, 1>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
-  return launch_spmm<T, VEC, 32, 2>(I, p->row_ptr, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+  if (vecs <= 4) return launch_spmm<T, VEC, 4, 1>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+  if (vecs <= 8) return launch_spmm<T, VEC, 8, 1>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+  if (vecs <= 16) return launch_spmm<T, VEC, 16, 1>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+  if (vecs <= 32) return launch_spmm<T, VEC, 32, 1>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
+  return launch_spmm<T, VEC, 32, 2>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
 }
 
 }  // namespace

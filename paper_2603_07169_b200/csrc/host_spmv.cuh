@@ -5,8 +5,6 @@
 #include "spmv_kernels.cuh"
 #include "spmv_row_kernels.cuh"
 #include "spmv_uniform_kernels.cuh"
-#include "spmv_merge_stage_kernels.cuh"
-#include "spmv_merge_scan_kernels.cuh"
 
 namespace {
 
@@ -53,7 +51,7 @@ int launch_row_direct(b200sp_plan* p, const int32_t* col_idx, const T* vals, con
   if (rc_flag != B200SP_OK) return rc_flag;
   tl_pdl_kernel = true;
   return launch_smem(kernel, dim3(grid), dim3(THREADS), smem, stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz,
-                     p->row_ptr, col_idx, vals, x, y, alpha, beta, R, cap, tiles, stages, rot_lanes, dev->err_flag, 0);
+                     p->row_ptr, col_idx, vals, x, y, alpha, beta, R, cap, tiles, stages, rot_lanes, dev->err_flag, 0, g_opt.spin_limit, g_opt.debug_no_copies);
 }
 
 // The same kernel on an ELL matrix of at most kRowMaxLen slots per row (implicit row offsets, padding skipped).
@@ -89,7 +87,7 @@ int launch_row_direct_ell(int64_t m, int width, const int32_t* col_ids, const T*
   if (rc_flag != B200SP_OK) return rc_flag;
   tl_pdl_kernel = true;
   return launch_smem(kernel, dim3(grid), dim3(THREADS), smem, stream, nullptr, 0, dev, (int)m, (int)(m * width), (const int*)nullptr, col_ids,
-                     vals, x, y, alpha, beta, R, cap, tiles, stages, 0, dev->err_flag, width);
+                     vals, x, y, alpha, beta, R, cap, tiles, stages, 0, dev->err_flag, width, g_opt.spin_limit, g_opt.debug_no_copies);
 }
 
 template <typename T>
@@ -165,36 +163,7 @@ int run_spmv_merge(b200sp_plan* p, const int32_t* col_idx, const T* vals, const 
   const b200sp_plan_info_t& I = p->info;
   const int tiles = I.spmv_tiles;
   int rc;
-  if (g_opt.merge_staged) {
-    const int stages = g_opt.merge_stages, ctas = g_opt.merge_ctas;
-    auto kernel = spmv_merge_stage_kernel<T, ITEMS, kThreads, kShortMax>;
-    const size_t smem = (size_t)stages * merge_stage_bytes<T>(ITEMS);
-    if ((size_t)ctas * (smem + 2048) > (size_t)kSmemPerSm) return B200SP_ERR_UNSUPPORTED;
-    static int configured[64] = {};
-    int carve = (int)(((size_t)ctas * (smem + 2048) * 100 + (size_t)kSmemPerSm) / ((size_t)kSmemPerSm + 1024)) + 1;
-    if (carve > 100) carve = 100;
-    if (configured[p->device] != carve + 1) {
-      CU(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerSm - 2048));
-      CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve));
-      configured[p->device] = carve + 1;
-    }
-    rc = ensure_err_flag(dev);
-    if (rc != B200SP_OK) return rc;
-    const int grid = tiles < ctas * dev->sms ? tiles : ctas * dev->sms;
-    rc = launch_smem(kernel, dim3(grid), dim3(kThreads), smem, stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr,
-                     col_idx, vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail, tiles, stages, dev->err_flag);
-  } else if (g_opt.merge_scan && ITEMS <= 2048) {
-    constexpr int SCAN_ITEMS = ITEMS <= 2048 ? ITEMS : 2048;
-    auto kernel = spmv_merge_scan_kernel<T, SCAN_ITEMS, 128>;
-    if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
-    int stride = 1;   // tile order: a stride coprime to the tile count (1 = plain order)
-    if (g_opt.merge_stride > 1 && tiles > 2 * g_opt.merge_stride) {
-      stride = g_opt.merge_stride;
-      while (gcd_int(stride, tiles) != 1) ++stride;
-    }
-    rc = launch(kernel, dim3(tiles), dim3(128), stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx,
-                vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail, stride);
-  } else if (g_opt.merge_threads == 64) {
+  if (g_opt.merge_threads == 64) {
     auto kernel = spmv_merge_tile_kernel<T, ITEMS, 64, SHORT>;
     if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
     tl_pdl_kernel = true;
@@ -242,6 +211,9 @@ int run_spmv_subwarp(b200sp_plan* p, const int32_t* col_idx, const T* vals, cons
   const double mean = I.m > 0 ? (double)I.nnz / (double)I.m : 0.0;
   int lpr = g_opt.sub_lanes;
   if (lpr <= 0) lpr = mean <= 3 ? 1 : mean <= 6 ? 2 : mean <= 12 ? 4 : mean <= 24 ? 8 : mean <= 64 ? 16 : 32;
+  // no lane adds more than kSubwarpChain terms in sequence, whatever the mean says (the plan sends matrices with a row
+  // longer than 32 * kSubwarpChain to the merge-tile kernel)
+  while (lpr < 32 && ((long long)I.max_row_len + lpr - 1) / lpr > kSubwarpChain) lpr *= 2;
   switch (lpr) {
     case 1: return launch_subwarp<T, 1>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
     case 2: return launch_subwarp<T, 2>(p, col_idx, vals, x, y, alpha, beta, stream, dev);

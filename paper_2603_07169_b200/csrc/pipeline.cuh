@@ -1,5 +1,5 @@
 // mbarrier + bulk-copy (TMA, 1-D) helpers for the shared-memory staging pipelines.
-// Every wait is bounded: after kSpinLimit polls the caller records an error and leaves.
+// Every wait is bounded: after `limit` polls (option "spin_limit", default kSpinLimit) the caller records an error and leaves.
 #pragma once
 #include "common.cuh"
 
@@ -22,9 +22,9 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
                : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Returns false if the barrier did not flip within the poll limit.
-__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity) {
-  for (int spin = 0; spin < kSpinLimit; ++spin)
+// Returns false if the barrier did not flip within `limit` polls.
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity, int limit) {
+  for (int spin = 0; spin < limit; ++spin)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }

@@ -1,4 +1,4 @@
-// Plan pass (device side): row-length statistics and bins, nnz-balanced split points.
+// Plan pass (device side): row-length statistics and bins, merge-path split points, lists of medium and long rows.
 #pragma once
 #include "common.cuh"
 
@@ -9,39 +9,40 @@ struct PlanStats {
   int max_len;
   int bad;  // row_ptr not monotone (negative length seen)
   int pad;
-  unsigned long long bin_rows[5];
-  unsigned long long bin_nnz[5];
+  unsigned long long bin_rows[6];
+  unsigned long long bin_nnz[6];
 };
 
+// Row-length bins: 0, 1-4, 5-32, 33-128, 129-1024, > 1024.
 __device__ __forceinline__ int length_bin(int len) {
-  return len == 0 ? 0 : len <= 4 ? 1 : len <= 32 ? 2 : len <= 1024 ? 3 : 4;
+  return len == 0 ? 0 : len <= 4 ? 1 : len <= 32 ? 2 : len <= 128 ? 3 : len <= 1024 ? 4 : 5;
 }
 
-// One pass over row_ptr: min / max row length and the five length bins (rows, nnz per bin).
+// One pass over row_ptr: min / max row length and the six length bins (rows, nnz per bin).
 // Integer atomics only, so the result does not depend on scheduling.
 __global__ void __launch_bounds__(256) plan_stats_kernel(const int* __restrict__ row_ptr, int m, PlanStats* st) {
-  __shared__ unsigned long long s_rows[5], s_nnz[5];
+  __shared__ unsigned long long s_rows[6], s_nnz[6];
   __shared__ int s_min, s_max, s_bad;
-  if (threadIdx.x < 5) { s_rows[threadIdx.x] = 0; s_nnz[threadIdx.x] = 0; }
+  if (threadIdx.x < 6) { s_rows[threadIdx.x] = 0; s_nnz[threadIdx.x] = 0; }
   if (threadIdx.x == 0) { s_min = 0x7FFFFFFF; s_max = 0; s_bad = 0; }
   __syncthreads();
   int lmin = 0x7FFFFFFF, lmax = 0, bad = 0;
-  unsigned rows[5] = {0, 0, 0, 0, 0};
-  unsigned long long nz[5] = {0, 0, 0, 0, 0};
+  unsigned rows[6] = {0, 0, 0, 0, 0, 0};
+  unsigned long long nz[6] = {0, 0, 0, 0, 0, 0};
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < m; i += (long long)gridDim.x * blockDim.x) {
     const int len = row_ptr[i + 1] - row_ptr[i];
     if (len < 0) { bad = 1; continue; }
     lmin = min(lmin, len); lmax = max(lmax, len);
     const int b = length_bin(len);
 #pragma unroll
-    for (int j = 0; j < 5; ++j) if (b == j) { rows[j]++; nz[j] += (unsigned)len; }
+    for (int j = 0; j < 6; ++j) if (b == j) { rows[j]++; nz[j] += (unsigned)len; }
   }
   atomicMin(&s_min, lmin); atomicMax(&s_max, lmax); if (bad) atomicOr(&s_bad, 1);
 #pragma unroll
-  for (int j = 0; j < 5; ++j) if (rows[j]) { atomicAdd(&s_rows[j], (unsigned long long)rows[j]); atomicAdd(&s_nnz[j], nz[j]); }
+  for (int j = 0; j < 6; ++j) if (rows[j]) { atomicAdd(&s_rows[j], (unsigned long long)rows[j]); atomicAdd(&s_nnz[j], nz[j]); }
   __syncthreads();
   if (threadIdx.x == 0) { atomicMin(&st->min_len, s_min); atomicMax(&st->max_len, s_max); if (s_bad) atomicOr(&st->bad, 1); }
-  if (threadIdx.x < 5 && s_rows[threadIdx.x]) {
+  if (threadIdx.x < 6 && s_rows[threadIdx.x]) {
     atomicAdd(&st->bin_rows[threadIdx.x], s_rows[threadIdx.x]);
     atomicAdd(&st->bin_nnz[threadIdx.x], s_nnz[threadIdx.x]);
   }
@@ -65,29 +66,19 @@ __global__ void __launch_bounds__(256) plan_merge_split_kernel(const int* __rest
   split_row[t] = lo;
 }
 
-// nnz-only split for SpMM: unit u starts at nonzero u * tile_nnz; split_row[u] = the row holding it
-// (the last row whose start is <= that position; rows of length 0 are skipped over).
-__global__ void __launch_bounds__(256) plan_nnz_split_kernel(const int* __restrict__ row_ptr, int m, int nnz, int tile_nnz,
-                                                             int tiles, int* __restrict__ split_row) {
-  const int t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t > tiles) return;
-  long long p = (long long)t * tile_nnz;
-  if (p >= nnz) { split_row[t] = m; return; }
-  int lo = 0, hi = m;  // find the largest r with row_ptr[r] <= p  (then row_ptr[r+1] > p)
-  while (lo < hi) {
-    const int mid = (lo + hi) >> 1;
-    if ((long long)row_ptr[mid + 1] <= p) lo = mid + 1; else hi = mid;
-  }
-  split_row[t] = lo;
-}
-
-// Rows longer than `thresh`, appended to a list (order of the list only affects scheduling, never a value).
-__global__ void __launch_bounds__(256) plan_long_rows_kernel(const int* __restrict__ row_ptr, int m, int thresh, int capacity,
-                                                             int* __restrict__ list, int* __restrict__ count) {
+// Rows of mid_thresh + 1 .. long_thresh nonzeros and rows longer than long_thresh, each appended to a list of its own
+// (count[0], count[1]; the host sorts the lists, and their order only affects scheduling, never a value).
+__global__ void __launch_bounds__(256) plan_row_lists_kernel(const int* __restrict__ row_ptr, int m, int mid_thresh, int long_thresh,
+                                                             int mid_cap, int long_cap, int* __restrict__ mid_list,
+                                                             int* __restrict__ long_list, int* __restrict__ count) {
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < m; i += (long long)gridDim.x * blockDim.x) {
-    if (row_ptr[i + 1] - row_ptr[i] > thresh) {
+    const int len = row_ptr[i + 1] - row_ptr[i];
+    if (len > long_thresh) {
+      const int slot = atomicAdd(count + 1, 1);
+      if (slot < long_cap) long_list[slot] = (int)i;
+    } else if (len > mid_thresh) {
       const int slot = atomicAdd(count, 1);
-      if (slot < capacity) list[slot] = (int)i;
+      if (slot < mid_cap) mid_list[slot] = (int)i;
     }
   }
 }

@@ -42,26 +42,42 @@ template <> struct VecLoad<bf16_t, 1> {
   static __device__ __forceinline__ void st(bf16_t* p, const float (&v)[1]) { store_elem(p, v[0]); }
 };
 
+// No lane adds more than kChainBlock products in one sequential FP32 chain: longer rows are added block by block
+// and the block sums are added in a second chain, so the worst-case rounding error of a row of L products is
+// (kChainBlock + L / kChainBlock) * 2^-24 * sum|a b| instead of L * 2^-24 * sum|a b|.
+constexpr int kChainBlock = 128;
+
 // One group of LANES lanes per row; the group sweeps k in chunks of LANES * VEC columns, NCH chunks
 // at a time held in registers (the row's nonzeros are re-read from L1 for each further block of chunks).
+// Rows longer than long_thresh are left to spmm_long_row_kernel.
 template <typename T, int VEC, int LANES, int NCH, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 spmm_row_group_kernel(int m, int k, const int* __restrict__ row_ptr, const int* __restrict__ col_idx, const T* __restrict__ vals,
-                      const T* __restrict__ B, T* __restrict__ Y, float alpha, float beta) {
+                      const T* __restrict__ B, T* __restrict__ Y, float alpha, float beta, int long_thresh) {
   constexpr int GROUPS = THREADS / LANES;
+  grid_dependency_wait();
   const int g = threadIdx.x / LANES, lane = threadIdx.x % LANES;
   const long long row = (long long)blockIdx.x * GROUPS + g;
   if (row >= m) return;
   const int rs = row_ptr[row], re = row_ptr[row + 1];
+  if (re - rs > long_thresh) return;
   constexpr int SPAN = LANES * VEC;  // columns covered by one chunk
   for (int c0 = 0; c0 < k; c0 += SPAN * NCH) {
-    float acc[NCH][VEC];
+    float acc[NCH][VEC], tot[NCH][VEC];
 #pragma unroll
     for (int h = 0; h < NCH; ++h)
 #pragma unroll
-      for (int j = 0; j < VEC; ++j) acc[h][j] = 0.0f;
+      for (int j = 0; j < VEC; ++j) { acc[h][j] = 0.0f; tot[h][j] = 0.0f; }
     int p = rs;
+    int fold = 0;
     for (; p + 4 <= re; p += 4) {  // four independent B rows in flight per lane
+      if (++fold > kChainBlock / 4) {   // a block of products is complete: its sum joins the second-level chain
+        fold = 1;
+#pragma unroll
+        for (int h = 0; h < NCH; ++h)
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) { tot[h][j] += acc[h][j]; acc[h][j] = 0.0f; }
+      }
       int cc[4]; float vv[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) { cc[u] = __ldg(col_idx + p + u); vv[u] = to_f32(__ldg(vals + p + u)); }
@@ -104,6 +120,8 @@ spmm_row_group_kernel(int m, int k, const int* __restrict__ row_ptr, const int* 
       if (col < k) {
         float out[VEC];
         T* yp = Y + row * k + col;
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) acc[h][j] += tot[h][j];
         if (beta != 0.0f) {
           float old[VEC];
           VecLoad<T, VEC>::ld_plain(yp, old);
@@ -178,6 +196,46 @@ __device__ __forceinline__ void ld_a4(const int* col_idx, const bf16_t* vals, in
 // row's (col, val) pairs with the same 128-bit loads (a broadcast, served by L1), and each lane keeps its
 // VEC columns of the slice in FP32 registers with four independent 16-byte reads of B in flight.
 // Rows longer than long_thresh are left to spmm_long_row_kernel.
+// acc += sum over nonzeros [p, pe) of vals[q] * (this lane's VEC columns of row col_idx[q] of B): scalar steps up to the
+// first multiple of four, then four independent 16-byte reads of B in flight per lane.
+template <typename T, int VEC>
+__device__ __forceinline__ void slice_accumulate(const int* __restrict__ col_idx, const T* __restrict__ vals, const T* __restrict__ Bc, int k,
+                                                 int p, int pe, float (&acc)[VEC]) {
+  typedef typename RawVec<T, VEC>::type raw_t;
+  for (; p < pe && (p & 3); ++p) {   // up to the first multiple of four
+    const raw_t b = RawVec<T, VEC>::ld(Bc + (long long)__ldg(col_idx + p) * k);
+    RawVec<T, VEC>::fma(b, to_f32(__ldg(vals + p)), acc);
+  }
+  for (; p + 4 <= pe; p += 4) {
+    int c[4]; float v[4];
+    ld_a4(col_idx, vals, p, c, v);
+    raw_t b[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) b[u] = RawVec<T, VEC>::ld(Bc + (long long)c[u] * k);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) RawVec<T, VEC>::fma(b[u], v[u], acc);
+  }
+  for (; p < pe; ++p) {
+    const raw_t b = RawVec<T, VEC>::ld(Bc + (long long)__ldg(col_idx + p) * k);
+    RawVec<T, VEC>::fma(b, to_f32(__ldg(vals + p)), acc);
+  }
+}
+
+template <typename T, int VEC>
+__device__ __forceinline__ void slice_store(T* yp, const float (&acc)[VEC], float alpha, float beta) {
+  float out[VEC];
+  if (beta != 0.0f) {
+    float old[VEC];
+    VecLoad<T, VEC>::ld_plain(yp, old);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) out[j] = alpha * acc[j] + beta * old[j];
+  } else {
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) out[j] = alpha * acc[j];
+  }
+  VecLoad<T, VEC>::st(yp, out);
+}
+
 template <typename T, int VEC, int THREADS, int LANES>
 __global__ void __launch_bounds__(THREADS, 2048 / THREADS)
 spmm_slice_kernel(int m, int k, int row_blocks, const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
@@ -229,8 +287,42 @@ spmm_slice_kernel(int m, int k, int row_blocks, const int* __restrict__ row_ptr,
   VecLoad<T, VEC>::st(yp, out);
 }
 
-// One CTA per (long row, slice): the CTA's groups of eight lanes stride over the row's nonzeros, then the
-// per-group partial sums are added in group order through shared memory (fixed order: reproducible).
+// The same lanes-along-k scheme for the rows of kChainBlock + 1 .. long-row threshold products, taken from the plan's list of
+// such rows: the row is added in blocks of at most kChainBlock products (blocks end on multiples of four) and the block
+// sums join a second-level chain.  A kernel of its own so that the second set of accumulators costs the register-capped
+// kernel above nothing.
+template <typename T, int VEC, int THREADS, int LANES>
+__global__ void __launch_bounds__(THREADS)
+spmm_medium_row_kernel(int num_rows, const int* __restrict__ rows, int k, int row_blocks, const int* __restrict__ row_ptr,
+                       const int* __restrict__ col_idx, const T* __restrict__ vals, const T* __restrict__ B, T* __restrict__ Y,
+                       float alpha, float beta) {
+  constexpr int GROUPS = THREADS / LANES, KS = LANES * VEC;
+  grid_dependency_wait();
+  const int slice = blockIdx.x / row_blocks, rb = blockIdx.x - slice * row_blocks;
+  const int g = threadIdx.x / LANES, l8 = threadIdx.x % LANES;
+  const int idx = rb * GROUPS + g;
+  if (idx >= num_rows) return;
+  const long long row = rows[idx];
+  const int rs = __ldg(row_ptr + row), re = __ldg(row_ptr + row + 1);
+  const int col0 = slice * KS + l8 * VEC;
+  if (col0 >= k) return;
+  const T* Bc = B + col0;
+  float acc[VEC], tot[VEC];
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) { acc[j] = 0.0f; tot[j] = 0.0f; }
+  for (int p = rs; p < re;) {
+    const int pe = min(re, (p + kChainBlock) & ~3);
+    slice_accumulate<T, VEC>(col_idx, vals, Bc, k, p, pe, acc);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) { tot[j] += acc[j]; acc[j] = 0.0f; }
+    p = pe;
+  }
+  slice_store<T, VEC>(Y + row * k + col0, tot, alpha, beta);
+}
+
+// One CTA per (long row, slice): the CTA's groups of eight lanes stride over the row's nonzeros (sums in blocks of
+// kChainBlock / 2 products, block sums in a second chain), then the per-group partial sums are combined pairwise through
+// shared memory in a fixed tree (reproducible; five levels instead of a chain of 32).
 template <typename T, int VEC, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 spmm_long_row_kernel(int k, int num_long, const int* __restrict__ long_rows, const int* __restrict__ row_ptr,
@@ -246,12 +338,18 @@ spmm_long_row_kernel(int k, int num_long, const int* __restrict__ long_rows, con
   const int col0 = slice * KS + l8 * VEC;
   const bool active = col0 < k;
   const T* Bc = B + col0;
-  float acc[VEC];
+  float acc[VEC], tot[VEC];
 #pragma unroll
-  for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
+  for (int j = 0; j < VEC; ++j) { acc[j] = 0.0f; tot[j] = 0.0f; }
+  int fold = 0;
   for (int p = rs + g; p < re; p += GROUPS) {
     const int c = __ldg(col_idx + p);
     const float v = to_f32(__ldg(vals + p));
+    if (++fold > kChainBlock / 2) {
+      fold = 1;
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) { tot[j] += acc[j]; acc[j] = 0.0f; }
+    }
     if (active) {
       float b[VEC];
       VecLoad<T, VEC>::ld(Bc + (long long)c * k, b);
@@ -260,15 +358,15 @@ spmm_long_row_kernel(int k, int num_long, const int* __restrict__ long_rows, con
     }
   }
 #pragma unroll
-  for (int j = 0; j < VEC; ++j) part[g][l8 * VEC + j] = acc[j];
+  for (int j = 0; j < VEC; ++j) part[g][l8 * VEC + j] = acc[j] + tot[j];
   __syncthreads();
+  for (int half = GROUPS / 2; half > 0; half >>= 1) {
+    for (int i = threadIdx.x; i < half * KS; i += THREADS) part[i / KS][i % KS] += part[i / KS + half][i % KS];
+    __syncthreads();
+  }
   if (threadIdx.x < KS) {
     const int col = slice * KS + threadIdx.x;
-    if (col < k) {
-      float s = 0.0f;
-      for (int gg = 0; gg < GROUPS; ++gg) s += part[gg][threadIdx.x];
-      epilogue_store(Y, row * k + col, s, alpha, beta);
-    }
+    if (col < k) epilogue_store(Y, row * k + col, part[0][threadIdx.x], alpha, beta);
   }
 }
 

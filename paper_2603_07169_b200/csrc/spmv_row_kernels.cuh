@@ -50,13 +50,14 @@ __device__ __forceinline__ float row_batch(const int* __restrict__ cp, const T* 
   return acc;
 }
 
+// spin_limit bounds every barrier wait (polls); a wait that runs out sets *err and the CTA leaves.
 // ELL = true: the matrix is ELL (row-major m x ell_width, padding col_id < 0): row i starts at i * ell_width,
 // row_ptr is not read (the pointer may be null) and padded entries are skipped.
 template <typename T, int THREADS, int UNROLL, bool ROT, bool ELL = false>
 __global__ void __launch_bounds__(THREADS)
 spmv_row_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
                      const T* __restrict__ vals, const T* __restrict__ x, T* __restrict__ y, float alpha, float beta,
-                     int R, int cap, int num_tiles, int stages, int rot_lanes, int* __restrict__ err, int ell_width = 0) {
+                     int R, int cap, int num_tiles, int stages, int rot_lanes, int* __restrict__ err, int ell_width, int spin_limit, int no_copies) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ __align__(8) unsigned long long full_bar[kRowMaxStages];
   const int tid = threadIdx.x;
@@ -109,7 +110,8 @@ spmv_row_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const int*
       bulk_copy_g2s(smem_addr(val_s), vals + a0, (unsigned)bulk_nz * (unsigned)sizeof(T), bar);
     }
   };
-  if (tid == 0) {
+  // no_copies (a test switch): the producer issues nothing at all, so no copy can be in flight when the waits below run out
+  if (tid == 0 && !no_copies) {
     load_bounds(0);
     for (int i = 0; i < stages && i < my_tiles; ++i) { issue(i, i); load_bounds(i + 1); }
   }
@@ -129,14 +131,14 @@ spmv_row_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const int*
     // y0 does not depend on the stage: fetch it before waiting
     float yold = 0.0f;
     if (beta != 0.0f && tid < rows) yold = to_f32(y[r0 + tid]);
-    const bool arrived = mbar_wait_bounded(smem_addr(&full_bar[s]), parity);
+    const bool arrived = mbar_wait_bounded(smem_addr(&full_bar[s]), parity, spin_limit);
     if (!__syncthreads_and(arrived)) {   // uniform decision: a wait ran out of polls
       if (tid == 0) atomicExch(err, 1);
       // give the copies already issued a bounded chance to land before the CTA (and its shared memory) goes away
       int s2 = s; unsigned par2 = parity;
       for (int k = 1; k < stages && i + k < my_tiles; ++k) {
         if (++s2 == stages) { s2 = 0; par2 ^= 1; }
-        (void)mbar_wait_bounded(smem_addr(&full_bar[s2]), par2);
+        (void)mbar_wait_bounded(smem_addr(&full_bar[s2]), par2, spin_limit);
       }
       return;
     }
@@ -156,7 +158,7 @@ spmv_row_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const int*
       store_elem(y + r0 + tid, r);
     }
     __syncthreads();   // every thread is done with stage s
-    if (tid == 0 && i + stages < my_tiles) { issue(i + stages, s); load_bounds(i + stages + 1); }
+    if (tid == 0 && !no_copies && i + stages < my_tiles) { issue(i + stages, s); load_bounds(i + stages + 1); }
     if (++s == stages) { s = 0; parity ^= 1; }
   }
 }

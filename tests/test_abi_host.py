@@ -14,7 +14,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def declared_functions():
-    text = open(os.path.join(ROOT, "include", "b200sp.h")).read()
+    text = "".join(open(os.path.join(ROOT, "include", f)).read() for f in sorted(os.listdir(os.path.join(ROOT, "include"))) if f.endswith(".h"))
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     names = re.findall(r"\b([a-z_0-9]+)\s*\(", text)
     return sorted({n for n in names if n.startswith(("spmv_", "spmm_", "b200sp_"))})
@@ -88,6 +88,26 @@ def test_binding_raises_with_status():
     with pytest.raises(b200sp.B200spError) as e:
         b200sp.spmv_csr(-1, 0, 0, None, None, None, None, None, 1.0, 0.0, "f32", stream=0)
     assert e.value.status == BAD
+
+
+def test_device_entry_points_refuse_host_arrays_before_anything_is_launched():
+    """A numpy array (or a CPU tensor) handed to a device entry point would make a kernel dereference a host address; the
+    binding refuses it with INVALID_ARG and the library is never entered."""
+    import torch
+    n0 = b200sp.b200sp_launch_count()
+    a = np.zeros(64, np.int32)
+    f = np.zeros(64, np.float32)
+    for bad in (a, torch.zeros(64, dtype=torch.int32)):
+        with pytest.raises(b200sp.B200spError) as e:
+            b200sp.spmv_csr(4, 4, 4, bad, a, f, f, f, 1.0, 0.0, "f32", stream=0)
+        assert e.value.status == BAD
+    with pytest.raises(b200sp.B200spError) as e:
+        b200sp.spmm_csr(4, 4, 4, 8, a, a, f, f, f, 1.0, 0.0, "f32", stream=0)
+    assert e.value.status == BAD
+    with pytest.raises(b200sp.B200spError) as e:       # host entry point: too short an array is refused as well
+        b200sp.spmv_csr_host(100, 100, 400, a, a, f, f, f, 1.0, 0.0, "f32", stream=0)
+    assert e.value.status == BAD
+    assert b200sp.b200sp_launch_count() == n0
 
 
 def test_product_path_does_not_import_the_oracle():

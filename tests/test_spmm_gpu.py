@@ -51,16 +51,37 @@ def test_long_rows_and_both_kernels(sliced, dtype):
         b200sp.b200sp_set_option("spmm_sliced", 1)
 
 
-@pytest.mark.parametrize("k", [64, 256])
-def test_longest_sequential_rows_positive_data(k):
-    """Rows of exactly 1024 nonzeros are the longest that one lane group adds in sequence; with all-positive data nothing
-    cancels, so this is the case that comes closest to the FP32 bound (chain bound 1024 * 2^-24 * S; measured 0.2-0.25 of 1e-5 * S)."""
+@pytest.mark.parametrize("sliced", [1, 0])
+@pytest.mark.parametrize("k", [3, 17, 64, 256])
+def test_positive_data_chains_stay_below_the_literal_fp32_bound(k, sliced):
+    """All-positive data, where rounding errors do not cancel.  No lane adds more than about 128 products in one chain:
+    rows of up to 128 nonzeros are added in sequence, rows of 129-1024 in blocks of 128 whose sums form a second chain,
+    longer rows by a CTA with blocks of 64 and a pairwise tree.  Rows of 128, 129, 1024, 1025 and 20,000 nonzeros, with k a
+    multiple of the vector width and not (k = 3, 17: scalar lanes)."""
     rng = np.random.default_rng(5)
-    A = gen.random_csr(400, 4000, np.full(400, 1024), seed=1024)
+    lens = np.concatenate([np.full(100, 128), np.full(100, 129), np.full(60, 1024), np.full(10, 1025), [20000], np.full(50, 7)])
+    n = 30000
+    b200sp.b200sp_set_option("spmm_sliced", sliced)
+    try:
+        A = gen.random_csr(len(lens), n, lens, seed=1024)
+        A.vals[:] = rng.random(A.nnz).astype(np.float32) + 0.01
+        B = rng.random(n * k).astype(np.float32) + 0.01
+        Y, Y_ref, S = run_spmm(A, B, k, None, 1.0, 0.0, "f32")
+        r = assert_within(Y, Y_ref, S, "f32", what="positive data k=%d sliced=%d" % (k, sliced))
+        assert r < 0.5, "k=%d sliced=%d: ratio %.3g" % (k, sliced, r)
+    finally:
+        b200sp.b200sp_set_option("spmm_sliced", 1)
+
+
+def test_positive_data_few_columns_kernel():
+    """The kernel that holds a slice of B in shared memory, rows of up to 2048 positive products (duplicates allowed)."""
+    rng = np.random.default_rng(6)
+    lens = np.concatenate([np.full(50, 2048), np.full(50, 1500), np.full(2000, 20), [6000]])
+    A = gen.random_csr(len(lens), 2048, lens, seed=3, allow_dup=True)
     A.vals[:] = rng.random(A.nnz).astype(np.float32) + 0.01
-    B = rng.random(4000 * k).astype(np.float32) + 0.01
-    Y, Y_ref, S = run_spmm(A, B, k, None, 1.0, 0.0, "f32")
-    assert assert_within(Y, Y_ref, S, "f32", what="1024-term rows, positive data") < 0.5
+    B = rng.random(2048 * 64).astype(np.float32) + 0.01
+    Y, Y_ref, S = run_spmm(A, B, 64, None, 1.0, 0.0, "f32")
+    assert assert_within(Y, Y_ref, S, "f32", what="positive data, B in shared memory") < 0.5
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
@@ -103,15 +124,25 @@ def test_workload_scaled(name):
         assert_within(Y, Y_ref, S, dtype, what="%s %s" % (name, dtype))
 
 
-@pytest.mark.parametrize("name", ["c5k64", "c5k256"])
-def test_workload_full_size_sampled_rows(name):
-    """Full size; the oracle computes 2048 sampled output rows (plus the first and last) one by one."""
-    w = gen.workload(name)
+def test_workload_full_size_every_entry_k64():
+    """c5 with k = 64 at full size, both dtypes: every one of the 33.5 M output entries against the oracle."""
+    w = gen.workload("c5k64")
+    for dtype in w.dtypes:
+        Y, Y_ref, S = run_spmm(w.A, w.B, w.k, None, w.alpha, w.beta, dtype)
+        assert_within(Y, Y_ref, S, dtype, what="c5k64 %s full, all rows" % dtype)
+        del Y, Y_ref, S
+
+
+def test_workload_full_size_sampled_rows_k256():
+    """c5 with k = 256 at full size; the oracle computes 8192 sampled output rows (plus the first and last of every block of
+    2^16 rows) one by one."""
+    w = gen.workload("c5k256")
     rng = np.random.default_rng(11)
-    rows = np.unique(np.concatenate([[0, w.A.m - 1], rng.integers(0, w.A.m, 2048)])).astype(np.int64)
+    edges = np.arange(0, w.A.m + 1, 1 << 16)
+    rows = np.unique(np.concatenate([edges[:-1], edges[1:] - 1, rng.integers(0, w.A.m, 8192)])).astype(np.int64)
     for dtype in w.dtypes:
         Y, Y_ref, S = run_spmm(w.A, w.B, w.k, None, w.alpha, w.beta, dtype, rows=rows)
-        assert_within(Y, Y_ref, S, dtype, what="%s %s full" % (name, dtype))
+        assert_within(Y, Y_ref, S, dtype, what="c5k256 %s full" % dtype)
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
