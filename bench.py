@@ -2,13 +2,15 @@
 """Benchmark of the CSR SpMV / SpMM hot path on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extras]
+    python bench.py --probes          the hardware rates behind the secondary bounds (gather, stream, full-line reads)
+    python bench.py --paper-sweep     the paper's own SpMV / SpMM sizes, speed-up over a naive kernel and its score P
 
 Headline (one JSON line on stdout): effective HBM GB/s of CSR SpMV on the uniform 16-nonzeros-per-row
 workload (m = n = 2^20, FP32, alpha 1.5, beta 0.5), i.e. algorithmic bytes per call divided by the
 device time per call, through the C ABI (spmv_csr) with a cached plan.  One "step" is one spmv_csr
-call (merge-tile kernel + carry fix-up kernel).  Inputs are resident in HBM; to keep every call
-cold, the steps rotate over R independent device copies of all operands whose total size is several
-times the L2 capacity, so no flush sits inside the timed region.  The same line carries the
+call; on this workload (equal rows) that is one launch of the uniform-row kernel.  Inputs are resident
+in HBM; to keep every call cold, the steps rotate over R independent device copies of all operands whose
+total size is several times the L2 capacity, so no flush sits inside the timed region.  The same line carries the
 roofline fraction against the measured copy bandwidth, an end-to-end figure through spmv_csr_host
 (host buffers, copies inside the timed region), the CPU oracle timed on the host cores, the other
 workloads (BF16, R-MAT, 27-point stencil, SpMM) as extras, and the SM clocks sampled while running.
@@ -34,16 +36,19 @@ if ROOT not in sys.path:
 METRIC = "SpMV/SpMM effective HBM GB/s (fraction of B200 peak); GFLOP/s at 2*nnz*k"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes (read + write) per launch of the dominant kernel from an ncu capture, keyed by
-# (workload, dtype); None where no capture has been made.  Sources: the summaries under profiles/.
-NCU_TRAFFIC_BYTES = {
-    ("c2", "f32"): 148_018_944,     # profiles/spmv_uniform_vec_c2_f32.md
-    ("c2", "bf16"): 108_764_928,    # profiles/spmv_uniform_vec_c2_bf16.md
-    ("c3", "f32"): 305_641_216,     # profiles/spmv_merge_tile_c3_f32.md
-    ("c4", "bf16"): 690_968_832,    # profiles/spmv_row_tile_c4_bf16.md
-    ("c1", "f32"): 3_163_648,       # profiles/spmv_row_tile_c1_f32.md
-    ("c5k64", "f32"): 1_274_698_040,  # profiles/spmm_slice_c5k64_f32.md
-}
+def ncu_record(workload: str, dtype: str):
+    """What one ncu capture of the dominant kernel of (workload, dtype) measured, per launch: profiles/traffic.json, written
+    from ncu's CSV by `python -m paper_2603_07169_b200.ncu_summary` (None if there is no capture)."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        return json.load(f).get("%s_%s" % (workload, dtype))
+
+
+def ncu_traffic(workload: str, dtype: str):
+    rec = ncu_record(workload, dtype)
+    return None if rec is None else rec.get("dram_bytes")
 
 
 def measured_peaks():
@@ -215,7 +220,7 @@ def measure(w, dtype, steps, warmup, dev, l2_bytes, barrier=None, min_copies=2, 
     res["cusparse_ms"] = None
     if cusparse is not None:
         try:
-            res["cusparse_ms"] = cusparse.time(sets[0], w, dtype, min(steps, 20), stream)
+            res["cusparse_ms"] = cusparse.time(sets, w, dtype, min(steps, 20), stream)
         except Exception as ex:  # pragma: no cover
             res["cusparse_ms"] = "unavailable: %r" % (ex,)
     res["_sets"] = sets
@@ -338,6 +343,107 @@ def probe_gather_rate(n_elems: int, dev) -> float:
     return 5 * gathers / (a.elapsed_time(b) * 1e-3)
 
 
+def run_probes(dev, l2_bytes):
+    """The hardware rates that bound the kernels, each measured by a library probe kernel that does nothing else (CUDA events,
+    median of 7 repetitions, a buffer larger than L2 rewritten between repetitions so that every repetition starts cold)."""
+    import torch
+    import paper_2603_07169_b200 as b200sp
+    stream = torch.cuda.current_stream()
+    sink = torch.zeros(1, dtype=torch.float32, device=dev)
+    flush = torch.empty(max(2 * l2_bytes, 256 << 20) // 4, dtype=torch.float32, device=dev)
+    props = torch.cuda.get_device_properties(dev)
+    sms = props.multi_processor_count
+    clock_hz = float(getattr(props, "clock_rate", 1965000)) * 1e3      # kHz -> Hz (maximum SM clock)
+
+    def timed(fn, reps=7):
+        fn()
+        ts = []
+        for _ in range(reps):
+            flush.fill_(1.0)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            b.synchronize()
+            ts.append(a.elapsed_time(b) * 1e-3)
+        ts.sort()
+        return ts[len(ts) // 2]
+
+    out = {"device": props.name, "sms": sms, "l2_mb": round(l2_bytes / 1e6, 1), "rows": []}
+
+    def row(name, value, unit, note=""):
+        out["rows"].append({"probe": name, "value": round(value, 2), "unit": unit, "note": note})
+
+    # streaming reads
+    for nbytes, label in ((1 << 30, "1 GiB"), (134_217_728, "134 MB (the CSR arrays of the uniform workload)"), (688_000_000, "688 MB (the stencil workload)")):
+        buf = torch.zeros(nbytes // 4, dtype=torch.int32, device=dev)
+        t = timed(lambda: b200sp.b200sp_probe_stream(buf, buf.numel() * 4, sink, stream))
+        row("streaming read, 128-bit loads, %s" % label, buf.numel() * 4 / t * 1e-9, "GB/s", "%.1f us" % (t * 1e6))
+        del buf
+    # random gathers
+    gathers = 1 << 26
+    for elems, eb, smem, label in ((16384, 4, 0, "4-byte gathers, table 64 KB (fits L1)"), (1 << 20, 4, 0, "4-byte gathers, table 4 MB (fits L2, not L1)"),
+                                   (1 << 22, 4, 0, "4-byte gathers, table 16 MB"), (1 << 20, 2, 0, "2-byte gathers, table 2 MB"),
+                                   (8192, 4, 1, "4-byte gathers, table 32 KB held in shared memory"),
+                                   (32768, 4, 1, "4-byte gathers, table 128 KB held in shared memory")):
+        table = torch.zeros(elems, dtype=torch.float32 if eb == 4 else torch.int16, device=dev)
+        t = timed(lambda: b200sp.b200sp_probe_gather_ex(table, elems, gathers, eb, smem, sink, stream))
+        rate = gathers / t
+        row("random " + label, rate * 1e-9, "G gathers/s", "%.2f per clock per SM at %d MHz" % (rate / sms / (clock_hz), int(clock_hz // 1e6)))
+        del table
+    # random full-line reads (SpMM's reads of B): lines in flight per group of eight lanes, in registers or through cp.async
+    reads = 1 << 25
+    for lines, label in ((1 << 19, "64 MB of lines (one k-slice of B of the SpMM workload)"), (1 << 17, "16 MB of lines (L2-resident)")):
+        buf = torch.zeros(lines * 32, dtype=torch.int32, device=dev)
+        for inflight, to_smem in ((4, 0), (8, 0), (16, 0), (4, 1), (8, 1), (16, 1)):
+            t = timed(lambda: b200sp.b200sp_probe_lines(buf, lines, reads, sink, inflight, to_smem, stream))
+            row("random 128-byte line reads by groups of 8 lanes, %d in flight per group %s, %s" % (inflight, "to shared memory (cp.async)" if to_smem else "to registers", label),
+                reads * 128 / t * 1e-12, "TB/s", "%.1f bytes per clock per SM" % (reads * 128 / t / sms / clock_hz))
+        del buf
+    return out
+
+
+def request_bound(rec, w, dtype, gather_rate):
+    """A bound from MEASURED L1-to-L2 traffic instead of one miss per nonzero: the ncu capture of this workload counts the
+    sectors the L1s asked L2 for; the CSR stream's share of them arrives four sectors to a request (128-bit coalesced loads of
+    whole lines), every other sector is a request of its own, and the SMs issue requests at the probe's rate."""
+    if not rec or "l2_sectors_read_by_l1" not in rec:
+        return {}
+    A = w.A
+    e = 4 if dtype == "f32" else 2
+    stream_sectors = (A.nnz * (4 + e) + (A.m + 1) * 4) / 32.0
+    sectors = float(rec["l2_sectors_read_by_l1"])
+    requests = max(sectors - stream_sectors, 0.0) + stream_sectors / 4.0
+    return {"request_bound_ms": round(requests / gather_rate * 1e3, 5), "l1_hit_pct_ncu": rec.get("l1_hit_pct"),
+            "request_bound_note": "L1-to-L2 requests counted by ncu (%.3g sectors, CSR stream four to a request) at the probe's request rate" % sectors}
+
+
+_LINES_RATE = {}
+
+
+def probe_lines_rate(dev, lines=1 << 19) -> float:
+    """Bytes per second of random 128-byte line reads by groups of eight lanes with four lines in flight per group (the access
+    pattern of the k-sliced SpMM kernel's reads of B), from a buffer of `lines` lines; measured once per process."""
+    import torch
+    import paper_2603_07169_b200 as b200sp
+    if dev not in _LINES_RATE:
+        buf = torch.zeros(lines * 32, dtype=torch.int32, device=dev)
+        sink = torch.zeros(1, dtype=torch.float32, device=dev)
+        stream = torch.cuda.current_stream()
+        reads = 1 << 25
+        for _ in range(2):
+            b200sp.b200sp_probe_lines(buf, lines, reads, sink, 4, 0, stream)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(3):
+            b200sp.b200sp_probe_lines(buf, lines, reads, sink, 4, 0, stream)
+        b.record(stream)
+        b.synchronize()
+        _LINES_RATE[dev] = 3 * reads * 128 / (a.elapsed_time(b) * 1e-3)
+        del buf
+    return _LINES_RATE[dev]
+
+
 class CuSparse:
     """cuSPARSE generic API through ctypes, timed on the same device buffers as a comparison point only."""
     R_32F, R_16BF, IDX_32I, ORDER_ROW = 0, 14, 2, 2
@@ -361,56 +467,66 @@ class CuSparse:
         if rc != 0:
             raise RuntimeError("cuSPARSE status %d" % rc)
 
-    def time(self, s, w, dtype, steps, stream):
-        """Median-free mean time per call (ms) of cusparseSpMV / cusparseSpMM on device set s (preprocess excluded)."""
+    def time(self, sets, w, dtype, steps, stream):
+        """Mean time per call (ms) of cusparseSpMV / cusparseSpMM over the device sets `sets` in rotation (cold L2 like our own
+        timing; buffer sizing and preprocess excluded)."""
         import torch
         c, L = self.c, self.lib
         A = w.A
         vt = self.R_32F if dtype == "f32" else self.R_16BF
         vp = c.c_void_p
+        if not isinstance(sets, (list, tuple)):
+            sets = [sets]
         self._ck(L.cusparseSetStream(self.h, vp(stream.cuda_stream)))
-        mat = vp()
-        self._ck(L.cusparseCreateCsr(c.byref(mat), c.c_int64(A.m), c.c_int64(A.n), c.c_int64(A.nnz), vp(s.rp.data_ptr()), vp(s.ci.data_ptr()),
-                                     vp(s.va.data_ptr()), self.IDX_32I, self.IDX_32I, 0, vt))
         alpha, beta = c.c_float(w.alpha), c.c_float(w.beta)
-        size = c.c_size_t(0)
-        out = s.out.clone()
-        if w.k:
-            dB, dC = vp(), vp()
-            self._ck(L.cusparseCreateDnMat(c.byref(dB), c.c_int64(A.n), c.c_int64(w.k), c.c_int64(w.k), vp(s.inp.data_ptr()), vt, self.ORDER_ROW))
-            self._ck(L.cusparseCreateDnMat(c.byref(dC), c.c_int64(A.m), c.c_int64(w.k), c.c_int64(w.k), vp(out.data_ptr()), vt, self.ORDER_ROW))
-            args = (self.h, 0, 0, c.byref(alpha), mat, dB, c.byref(beta), dC, self.R_32F, 0)
-            self._ck(L.cusparseSpMM_bufferSize(*args, c.byref(size)))
-            buf = torch.empty(max(size.value, 16), dtype=torch.uint8, device=s.va.device)
-            if hasattr(L, "cusparseSpMM_preprocess"):
-                self._ck(L.cusparseSpMM_preprocess(*args, vp(buf.data_ptr())))
-            run = lambda: L.cusparseSpMM(*args, vp(buf.data_ptr()))
-        else:
-            dX, dY = vp(), vp()
-            self._ck(L.cusparseCreateDnVec(c.byref(dX), c.c_int64(A.n), vp(s.inp.data_ptr()), vt))
-            self._ck(L.cusparseCreateDnVec(c.byref(dY), c.c_int64(A.m), vp(out.data_ptr()), vt))
-            args = (self.h, 0, c.byref(alpha), mat, dX, c.byref(beta), dY, self.R_32F, 0)
-            self._ck(L.cusparseSpMV_bufferSize(*args, c.byref(size)))
-            buf = torch.empty(max(size.value, 16), dtype=torch.uint8, device=s.va.device)
-            if hasattr(L, "cusparseSpMV_preprocess"):
-                self._ck(L.cusparseSpMV_preprocess(*args, vp(buf.data_ptr())))
-            run = lambda: L.cusparseSpMV(*args, vp(buf.data_ptr()))
-        for _ in range(3):
-            self._ck(run())
+        runs, keep, mats = [], [], []
+        for s in sets:
+            mat = vp()
+            self._ck(L.cusparseCreateCsr(c.byref(mat), c.c_int64(A.m), c.c_int64(A.n), c.c_int64(A.nnz), vp(s.rp.data_ptr()), vp(s.ci.data_ptr()),
+                                         vp(s.va.data_ptr()), self.IDX_32I, self.IDX_32I, 0, vt))
+            mats.append(mat)
+            size = c.c_size_t(0)
+            out = s.out.clone()
+            if w.k:
+                dB, dC = vp(), vp()
+                self._ck(L.cusparseCreateDnMat(c.byref(dB), c.c_int64(A.n), c.c_int64(w.k), c.c_int64(w.k), vp(s.inp.data_ptr()), vt, self.ORDER_ROW))
+                self._ck(L.cusparseCreateDnMat(c.byref(dC), c.c_int64(A.m), c.c_int64(w.k), c.c_int64(w.k), vp(out.data_ptr()), vt, self.ORDER_ROW))
+                args = (self.h, 0, 0, c.byref(alpha), mat, dB, c.byref(beta), dC, self.R_32F, 0)
+                self._ck(L.cusparseSpMM_bufferSize(*args, c.byref(size)))
+                buf = torch.empty(max(size.value, 16), dtype=torch.uint8, device=s.va.device)
+                if hasattr(L, "cusparseSpMM_preprocess"):
+                    self._ck(L.cusparseSpMM_preprocess(*args, vp(buf.data_ptr())))
+                runs.append(lambda args=args, buf=buf: L.cusparseSpMM(*args, vp(buf.data_ptr())))
+            else:
+                dX, dY = vp(), vp()
+                self._ck(L.cusparseCreateDnVec(c.byref(dX), c.c_int64(A.n), vp(s.inp.data_ptr()), vt))
+                self._ck(L.cusparseCreateDnVec(c.byref(dY), c.c_int64(A.m), vp(out.data_ptr()), vt))
+                args = (self.h, 0, c.byref(alpha), mat, dX, c.byref(beta), dY, self.R_32F, 0)
+                self._ck(L.cusparseSpMV_bufferSize(*args, c.byref(size)))
+                buf = torch.empty(max(size.value, 16), dtype=torch.uint8, device=s.va.device)
+                if hasattr(L, "cusparseSpMV_preprocess"):
+                    self._ck(L.cusparseSpMV_preprocess(*args, vp(buf.data_ptr())))
+                runs.append(lambda args=args, buf=buf: L.cusparseSpMV(*args, vp(buf.data_ptr())))
+            keep.append((out, buf))
+        for i in range(max(3, len(runs))):
+            self._ck(runs[i % len(runs)]())
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
-        for _ in range(steps):
-            self._ck(run())
+        for i in range(steps):
+            self._ck(runs[i % len(runs)]())
         b.record(stream)
         b.synchronize()
-        L.cusparseDestroySpMat(mat)
+        for mat in mats:
+            L.cusparseDestroySpMat(mat)
+        del keep
         return a.elapsed_time(b) / steps
 
 
-def paper_sweep(args, dev, l2_bytes):
+def paper_sweep(quick, dev, l2_bytes):
     """The experiment the paper ran for this operator (Table 6, tasks 12 / 13; Fig. 3a): its own sizes, speed-up over a
     naive baseline kernel and the complexity-weighted score P = sum T(N_i) S_i / sum T(N_i) (Section 3.3, Eq. 1-2),
-    for this library and for cuSPARSE.  T(N) = nnz for SpMV and nnz * K for SpMM, as in the table."""
+    for this library and for cuSPARSE.  T(N) = nnz for SpMV and nnz * K for SpMM, as in the table.  `quick` leaves out the
+    two largest SpMM sizes (2^16 and 2^18 rows).  Returns the record."""
     import torch
     import gen
     import paper_2603_07169_b200 as b200sp
@@ -459,7 +575,7 @@ def paper_sweep(args, dev, l2_bytes):
 
     out = {}
     spmm_rows = [2 ** 10, 2 ** 12, 2 ** 14, 2 ** 16, 2 ** 18]
-    for op, rows_list, k in (("spmv", [2 ** e for e in range(10, 16)], 0), ("spmm", spmm_rows if not args.quick else spmm_rows[:3], 4096)):
+    for op, rows_list, k in (("spmv", [2 ** e for e in range(10, 16)], 0), ("spmm", spmm_rows if not quick else spmm_rows[:3], 4096)):
         for dtype in ("f32", "bf16"):
             rec = {"rows": [], "nnz": [], "ours_us": [], "naive_us": [], "cusparse_us": []}
             for rows in rows_list:
@@ -487,7 +603,7 @@ def paper_sweep(args, dev, l2_bytes):
                 cu = None
                 if cusp is not None:
                     try:
-                        cu = round(cusp.time(sets[0], w, dtype, steps, stream) * 1e3, 3)
+                        cu = round(cusp.time(sets, w, dtype, steps, stream) * 1e3, 3)
                     except Exception:
                         cu = None
                 rec["cusparse_us"].append(cu)
@@ -503,9 +619,11 @@ def paper_sweep(args, dev, l2_bytes):
                 rec["speedup_cusparse"] = [round(v, 3) for v in Sc]
                 rec["P_cusparse"] = round(sum(t * v for t, v in zip(T, Sc)) / sum(T), 3)
             out["%s_%s" % (op, dtype)] = rec
-    print(json.dumps({"paper_sweep": out, "note": "rows x 2048 at density 0.01 (K = 4096 for SpMM); speed-ups over the naive one-thread-per-row "
-                      "(per-entry) kernel; P per the paper's Eq. 1-2 with T = nnz (x K); operands rotate over independent copies; SpMV ours / naive are "
-                      "per-call device times of 100 calls replayed from a CUDA graph, cuSPARSE and SpMM are launched from the host"}))
+    out["note"] = ("rows x 2048 at density 0.01 (K = 4096 for SpMM%s); speed-ups over the naive one-thread-per-row (per-entry) kernel; "
+                   "P per the paper's Eq. 1-2 with T = nnz (x K); operands rotate over independent copies; SpMV ours / naive are per-call "
+                   "device times of 100 calls replayed from a CUDA graph, cuSPARSE and SpMM are launched from the host"
+                   % (", SpMM rows 2^10, 2^12, 2^14 only" if quick else ""))
+    return out
 
 
 def run_reference(args):
@@ -554,6 +672,7 @@ def main():
     ap.add_argument("--dtype", default="f32")
     ap.add_argument("--paper-sweep", action="store_true", help="the paper's own SpMV / SpMM sizes with speed-up over a naive kernel and its score P")
     ap.add_argument("--quick", action="store_true", help="with --paper-sweep: skip the two largest SpMM sizes")
+    ap.add_argument("--probes", action="store_true", help="measure the hardware rates behind the secondary bounds and print them")
     ap.add_argument("--opt", action="append", default=[], help="library tuning switch name=value (b200sp_set_option), repeatable")
     ap.add_argument("--profile", action="store_true",
                     help="short run for a profiler: the timed loop of one workload only (no clock loop, e2e, extras, CPU baseline)")
@@ -587,7 +706,11 @@ def main():
 
     if args.paper_sweep:
         if rank == 0:
-            paper_sweep(args, dev, l2)
+            print(json.dumps({"paper_sweep": paper_sweep(args.quick, dev, l2)}))
+        return
+    if args.probes:
+        if rank == 0:
+            print(json.dumps({"probes": run_probes(dev, l2)}))
         return
     sampler = ClockSampler(local)
     sampler.start()
@@ -680,6 +803,7 @@ def main():
         todo = [("c2", "bf16"), ("c3", "f32"), ("c3p", "f32"), ("c4", "bf16"), ("c1", "f32"), ("c5k64", "f32"), ("c5k64", "bf16"),
                 ("c5k256", "f32"), ("c5k256", "bf16")]
         cache = {args.workload: w}
+        window_ab = {}
         for name, dt in todo:
             if (name, dt) == (args.workload, dtype):
                 continue
@@ -697,12 +821,33 @@ def main():
                 if name == "c1":   # launch-latency regime: per-call device time from a CUDA graph, and the floors on the same box
                     extras["c1_f32"].update(latency_floor(r["_call"], r["_sets"], dev, r["algorithmic_bytes"]))
                 if not ww.k:   # SpMV: time at the measured L1-miss gather rate for this x
-                    extras["%s_%s" % (name, dt)]["gather_bound_ms"] = round(ww.A.nnz / probe_gather_rate(ww.A.n, dev) * 1e3, 5)
+                    rate = probe_gather_rate(ww.A.n, dev)
+                    ex_ = extras["%s_%s" % (name, dt)]
+                    ex_["gather_bound_ms"] = round(ww.A.nnz / rate * 1e3, 5)
+                    ex_.update(request_bound(ncu_record(name, dt), ww, dt, rate))
+                else:          # SpMM: time of its reads of B (nnz * k * e bytes, one 128-byte line per nonzero and slice) at the measured rate of such reads
+                    lr = probe_lines_rate(dev)
+                    ex_ = extras["%s_%s" % (name, dt)]
+                    ex_["line_read_bound_ms"] = round(ww.A.nnz * ww.k * (4 if dt == "f32" else 2) / lr * 1e3, 5)
+                    ex_["line_read_rate_tbs"] = round(lr * 1e-12, 2)
                 del r
                 b200sp.b200sp_cache_clear()
                 torch.cuda.empty_cache()
             except Exception as ex:  # pragma: no cover
                 extras["%s_%s" % (name, dt)] = {"error": repr(ex)}
+            if (name, dt) in (("c3", "f32"), ("c2", "bf16"), ("c5k64", "f32")) and "ms_per_step" in extras.get("%s_%s" % (name, dt), {}):
+                try:   # the L2 access-policy window on the gathered operand, off / on
+                    b200sp.b200sp_set_option("x_l2_window", 1)
+                    r1 = measure(ww, dt, min(steps, 50), 5, dev, l2)
+                    window_ab["%s_%s" % (name, dt)] = {"window_off_ms": extras["%s_%s" % (name, dt)]["ms_per_step"], "window_on_ms": round(r1["ms_per_step"], 5)}
+                    del r1
+                except Exception as ex:  # pragma: no cover
+                    window_ab["%s_%s" % (name, dt)] = {"error": repr(ex)}
+                finally:
+                    b200sp.b200sp_set_option("x_l2_window", 0)
+                    b200sp.b200sp_cache_clear()
+                    torch.cuda.empty_cache()
+        extras["x_l2_window_ab"] = dict(window_ab, note="per-launch access-policy window (persisting hits) over x, or over B for SpMM; default off")
         # the COO and ELL front ends on the same matrices (paper tasks 8 and 14)
         for name, dt in (("c2", "f32"), ("c4", "bf16")):
             for kind in ("coo", "ell"):
@@ -715,6 +860,14 @@ def main():
                     torch.cuda.empty_cache()
                 except Exception as ex:  # pragma: no cover
                     extras["%s_%s_%s" % (kind, name, dt)] = {"error": repr(ex)}
+        # the paper's own experiment at its sizes (Table 6, tasks 12 / 13; score P of Section 3.3), short form
+        try:
+            cache = {}
+            sw = paper_sweep(True, dev, l2)
+            extras["paper_sweep_quick"] = {k: ({kk: v[kk] for kk in ("rows", "ours_us", "naive_us", "cusparse_us", "P_ours", "P_cusparse") if kk in v}
+                                               if isinstance(v, dict) else v) for k, v in sw.items()}
+        except Exception as ex:  # pragma: no cover
+            extras["paper_sweep_quick"] = {"error": repr(ex)}
     sampler.stop()
 
     # ---- CPU baseline: the oracle on the host cores, same workload (rank 0, N = 1 only)
@@ -755,14 +908,15 @@ def main():
                 "data": "synthetic", "config": config, "clocks": clocks, "e2e": e2e,
                 "gpu_launches": int(head["launches"]),
                 "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                             "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dtype)), "peak_kind": "of " + peak_kind,
+                             "traffic": ncu_traffic(args.workload, dtype), "peak_kind": "of " + peak_kind,
                              "frac_of_nominal_7700": achieved / 7700.0,
                              "note": "algorithmic bytes per step over event time per step (the step is the SpMV kernel; plan cached)",
+                             "binding_bound": "secondary" if (gather_rate is not None and A.nnz / gather_rate * 1e3 > head["algorithmic_bytes"] / peak * 1e-6) else "hbm",
                              "secondary": None if gather_rate is None else {
                                  "bound": "L1-miss gather (one L2 request per random x read)", "gathers_per_s": gather_rate,
                                  "ms_at_bound": A.nnz / gather_rate * 1e3, "frac_of_bound": (A.nnz / gather_rate * 1e3) / (head["ms_total"] / steps),
                                  "note": "measured live with b200sp_probe_gather on a table the size of x"}},
-                "cusparse": {"ms_per_step": head["cusparse_ms"], "note": "cusparseSpMV/SpMM, default algorithm, preprocess excluded, warm (one operand set); comparison point only"},
+                "cusparse": {"ms_per_step": head["cusparse_ms"], "note": "cusparseSpMV/SpMM, default algorithm, preprocess excluded, over the same rotated operand copies (cold L2); comparison point only"},
                 "cpu_baseline": cpu, "extra": extras}
         print(json.dumps(line))
     if world > 1:

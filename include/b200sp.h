@@ -96,7 +96,7 @@ typedef struct {
  * caching allocator does this readily), the stale plan would be used and the result would be wrong
  * without any error.  Call b200sp_cache_drop(row_ptr) before releasing or rewriting a row_ptr array (or
  * b200sp_cache_clear for everything), or use the plan API, which has no hidden state.  The cache holds
- * at most 64 plans and drops the least recently used one beyond that (dropping synchronises the device).
+ * at most 1024 plans and drops the least recently used one beyond that (dropping synchronises the device).
  * Two calls that use the same cached plan must not overlap on the GPU (they share its scratch).
  * dtype is a b200sp_dtype. */
 int spmv_csr(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx,
@@ -206,7 +206,8 @@ int spmv_csr_vec_host(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr,
  * B200SP_ERR_BAD_CSR if any check fails. */
 int b200sp_validate_csr(int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, const int32_t* col_idx, void* stream);
 
-void b200sp_cache_clear(void);                 /* destroys every plan cached by the one-shot calls and trims the library's memory pools */
+void b200sp_cache_clear(void);                 /* destroys every plan cached by the one-shot calls, trims the library's memory pools and
+                                                  releases the L2 set aside for access-policy windows (option "x_l2_window") */
 /* Forgets what the one-shot entry points cached under this address on the current device: the plan keyed on a row_ptr
  * (device address, or host address for the *_host calls), the row offsets keyed on a COO row_idx, the transpose plan
  * keyed on a CSC col_ptr.  Synchronises the device if anything was dropped.  Unknown addresses are not an error. */

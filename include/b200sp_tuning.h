@@ -23,15 +23,19 @@ extern "C" {
  *                    3 = sub-warp per row; a kernel the matrix is not eligible for falls back to an eligible one
  *   "spmm_bstage"    1 = SpMM keeps a slice of B in shared memory when A has few columns (default), 0 = never
  *   "spmm_sliced"    1 = SpMM walks k in 128-byte slices so that a slice of B can stay in L2 (default), 0 = one pass
- *   "spmm_ranges"    SpMM with sorted columns: 0 = choose the number of column ranges per slice so that a range of B
- *                    fits in L2 (default), 1 = never split, 2..8 = this many ranges
+ *   "spmm_stage_a"   the k-sliced SpMM kernel's warps first copy their rows' (col, val) pairs into shared memory: 1 = yes, 0 = no,
+ *                    2 = for BF16 storage only (default: measured 5-6 % faster there and 2-3 % slower for FP32)
+ *   "spmm_ranges"    k-sliced SpMM on rows with ascending columns, one launch per column range so that the rows of B a
+ *                    launch gathers from stay in L2: 1 = no ranges (default: measured slower, see the benchmarks' record),
+ *                    0 = as many as make a range of B fit L2, 2, 3, 4 or 8 = that many
  *  merge-tile SpMV kernel
  *   "merge_items"    merge items per tile: 1024, 2048 (default) or 4096
  *   "merge_threads"  threads per CTA: 64, 128 (default) or 256
  *   "merge_carve"    shared-memory carveout in percent requested for it: 0, 25, 45 (default), 60, 75, 100 or -1 = leave to the driver
  *   "merge_short"    rows of up to this many products are added by one thread: 8, 16, 32 (default) or 64
- *   "merge_empty"    1 = when many rows have no nonzeros they are kept out of the merge list and their y is written by a
- *                    pass of its own (default), 0 = every row is a merge item
+ *   "merge_empty"    1 = when a quarter or more of the rows have no nonzeros the merge list holds only the other rows, and y
+ *                    of the empty rows is written by a pass of its own, 0 = every row is a merge item (default: the list
+ *                    measured 3 % slower on the power-law workload with 61 % empty rows)
  *  row-direct SpMV kernel
  *   "row_stages"     shared-memory stages per CTA, 2 (default) .. 4
  *   "row_ctas"       CTAs per SM the tiles are sized for, 1..4, default 3
@@ -63,15 +67,30 @@ extern "C" {
  *                      with nothing in flight; the launch raises the flag that b200sp_check reports and its output is undefined
  *   "fail_alloc_after" N > 0: the N-th allocation the library makes from its memory pool from now on fails with
  *                      B200SP_ERR_ALLOC (the switch then clears itself); 0 = off (default)
- * "spmv_kernel" and "merge_items" apply to plans created afterwards, the others to the next call. */
+ * "spmv_kernel", "merge_items" and "merge_empty" apply to plans created afterwards, the others to the next call. */
 int b200sp_set_option(const char* name, int value);
 
-/* Measurement aid (no counterpart in the paper): enqueues `gathers` independent 4-byte reads of
- * table[h(i) mod table_elems] (table_elems a power of two, h a hash computed in registers), eight in
- * flight per thread, on as many CTAs as fit.  Timed by the caller with events it gives the rate at
- * which the SMs take random reads that miss L1, i.e. the bound on gathering x from a vector much
- * larger than L1.  `table` (table_elems floats) and `sink` (one float) are device pointers. */
+/* ---- measurement probes (no counterpart in the paper's operations) ----------------------------------------------
+ * Each enqueues one kernel that does nothing but the access pattern named, so that the caller, timing it with events,
+ * gets the hardware rate that bounds the corresponding library kernel.  All pointers are device pointers; `sink` is
+ * one float that is (practically) never written.
+ *
+ * b200sp_probe_gather: `gathers` independent 4-byte reads of table[h(i) mod table_elems] (table_elems a power of two,
+ *   h a hash computed in registers), eight in flight per thread, on as many CTAs as fit: the rate at which the SMs
+ *   take random reads that miss L1, i.e. the bound on gathering x from a vector much larger than L1.
+ * b200sp_probe_gather_ex: the same with entries of elem_bytes = 2 or 4 bytes and, with in_shared_memory = 1, with
+ *   the table (at most 224 KB) first copied into each CTA's shared memory and gathered from there.
+ * b200sp_probe_stream: reads `bytes` (a multiple of 16; buf 16-byte aligned) once with coalesced 128-bit loads: what
+ *   a pure stream of the CSR arrays reaches at that size.
+ * b200sp_probe_lines: `reads` random 128-byte lines out of `lines` (a power of two), each by a group of eight lanes
+ *   with 16 bytes per lane and in_flight = 4, 8 or 16 lines in flight per group, into registers or, with
+ *   to_shared_memory = 1, into shared memory with cp.async: the L2-to-SM rate of SpMM's reads of B (the k-sliced kernel
+ *   keeps four lines per group in registers). */
 int b200sp_probe_gather(const float* table, int64_t table_elems, int64_t gathers, float* sink, void* stream);
+int b200sp_probe_gather_ex(const void* table, int64_t table_elems, int64_t gathers, int elem_bytes, int in_shared_memory, float* sink,
+                           void* stream);
+int b200sp_probe_stream(const void* buf, int64_t bytes, float* sink, void* stream);
+int b200sp_probe_lines(const void* buf, int64_t lines, int64_t reads, int in_flight, int to_shared_memory, float* sink, void* stream);
 
 #ifdef __cplusplus
 }

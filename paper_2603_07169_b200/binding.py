@@ -20,7 +20,7 @@ EXPORTS = (
     "spmv_csr", "spmm_csr", "b200sp_plan_create", "b200sp_plan_destroy", "b200sp_plan_info", "b200sp_spmv",
     "b200sp_spmm", "spmv_csr_host", "spmm_csr_host", "b200sp_validate_csr", "b200sp_cache_clear",
     "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_launch_count", "b200sp_set_option",
-    "b200sp_check", "b200sp_cache_drop", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell", "spmv_csc", "spmm_csc", "spmv_csr_vec_host",
+    "b200sp_check", "b200sp_cache_drop", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_probe_gather_ex", "b200sp_probe_stream", "b200sp_probe_lines", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell", "spmv_csc", "spmm_csc", "spmv_csr_vec_host",
 )
 
 
@@ -81,6 +81,12 @@ def lib() -> ctypes.CDLL:
         L.b200sp_noalloc_max_items.restype = i64
         L.b200sp_probe_gather.argtypes = [p, i64, i64, p, p]
         L.b200sp_probe_gather.restype = i32
+        L.b200sp_probe_gather_ex.argtypes = [p, i64, i64, i32, i32, p, p]
+        L.b200sp_probe_gather_ex.restype = i32
+        L.b200sp_probe_stream.argtypes = [p, i64, p, p]
+        L.b200sp_probe_stream.restype = i32
+        L.b200sp_probe_lines.argtypes = [p, i64, i64, i32, i32, p, p]
+        L.b200sp_probe_lines.restype = i32
         L.spmm_csr_host.argtypes = L.spmm_csr.argtypes
         L.b200sp_plan_create.argtypes = [ctypes.POINTER(p), i64, i64, i64, p, p]
         L.b200sp_plan_destroy.argtypes = [p]
@@ -262,6 +268,21 @@ def b200sp_probe_gather(table, table_elems, gathers, sink, stream=None):
     """Enqueues the random-gather probe (see include/b200sp_tuning.h); time it with CUDA events."""
     _ck(lib().b200sp_probe_gather(_dev(table, table_elems, 4, "probe table"), table_elems, gathers, _dev(sink, 1, 4, "probe sink"),
                                   _stream(stream)), "b200sp_probe_gather")
+
+
+def b200sp_probe_gather_ex(table, table_elems, gathers, elem_bytes, in_shared_memory, sink, stream=None):
+    _ck(lib().b200sp_probe_gather_ex(_dev(table, table_elems, elem_bytes, "probe table"), table_elems, gathers, elem_bytes, in_shared_memory,
+                                     _dev(sink, 1, 4, "probe sink"), _stream(stream)), "b200sp_probe_gather_ex")
+
+
+def b200sp_probe_stream(buf, nbytes, sink, stream=None):
+    _ck(lib().b200sp_probe_stream(_dev(buf, nbytes // max(buf.element_size(), 1), buf.element_size(), "probe buffer"), nbytes,
+                                  _dev(sink, 1, 4, "probe sink"), _stream(stream)), "b200sp_probe_stream")
+
+
+def b200sp_probe_lines(buf, lines, reads, sink, in_flight=4, to_shared_memory=0, stream=None):
+    _ck(lib().b200sp_probe_lines(_dev(buf, lines * 128 // max(buf.element_size(), 1), buf.element_size(), "probe buffer"), lines, reads,
+                                 in_flight, to_shared_memory, _dev(sink, 1, 4, "probe sink"), _stream(stream)), "b200sp_probe_lines")
 
 
 def b200sp_noalloc_max_items() -> int:

@@ -40,12 +40,32 @@ static int run_spmv_noalloc(int64_t m, int64_t nnz, const int32_t* row_ptr, cons
                   kItems, tiles, (int*)sc->split_row);
   if (rc != B200SP_OK) return rc;
   rc = launch(spmv_merge_tile_kernel<T, kItems, kThreads, kShortMax>, dim3(tiles), dim3(kThreads), stream, nullptr, 0, dev, (int)m,
-              (int)nnz, row_ptr, col_idx, vals, x, y, alpha, beta, (const int*)sc->split_row, sc->carry, sc->tail);
+              (int)nnz, row_ptr, col_idx, vals, x, y, alpha, beta, (const int*)sc->split_row, sc->carry, sc->tail, (const int*)nullptr);
   if (rc != B200SP_OK) return rc;
   if (tiles > 1)
     rc = launch(spmv_carry_fixup_kernel<T, kItems>, dim3((tiles + 127) / 128), dim3(128), stream, nullptr, 0, dev, tiles, row_ptr,
-                (const int*)sc->split_row, (const float*)sc->carry, (const float*)sc->tail, y, alpha, beta);
+                (const int*)sc->split_row, (const float*)sc->carry, (const float*)sc->tail, y, alpha, beta, (const int*)nullptr);
   return rc;
+}
+
+// launcher of the gather probe (b200sp_tuning.h)
+template <typename E, bool SMEM>
+static int run_probe_gather(const void* table, int64_t table_elems, int64_t gathers, float* sink, cudaStream_t stream, DeviceInfo* dev) {
+  auto kernel = probe_gather_kernel<E, SMEM>;
+  const size_t smem = SMEM ? (size_t)table_elems * sizeof(E) : 0;
+  int d = 0;
+  CU(cudaGetDevice(&d));
+  if (SMEM) {
+    if (smem > (size_t)kSmemPerSm - 2048) return B200SP_ERR_INVALID_ARG;
+    CU(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  } else {
+    CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 0));
+  }
+  int nb = 0;
+  CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kernel, 256, smem));
+  if (nb < 1) nb = 1;
+  return launch_smem(kernel, dim3((unsigned)(dev->sms * nb)), dim3(256), smem, stream, nullptr, 0, dev, (const E*)table,
+                     (unsigned)(table_elems - 1), (long long)gathers, sink);
 }
 
 extern "C" {
@@ -182,23 +202,58 @@ int b200sp_spmm_naive(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_
                 row_ptr, col_idx, (const bf16_t*)vals, (const bf16_t*)B, (bf16_t*)Y, alpha, beta);
 }
 
-int b200sp_probe_gather(const float* table, int64_t table_elems, int64_t gathers, float* sink, void* stream) {
-  if (!table || !sink || table_elems <= 0 || (table_elems & (table_elems - 1)) != 0 || table_elems > ((int64_t)1 << 31) || gathers < 0)
+// ---- measurement probes (b200sp_tuning.h) ----
+int b200sp_probe_gather_ex(const void* table, int64_t table_elems, int64_t gathers, int elem_bytes, int in_shared_memory, float* sink,
+                           void* stream) {
+  if (!table || !sink || table_elems <= 0 || (table_elems & (table_elems - 1)) != 0 || table_elems > ((int64_t)1 << 31) || gathers < 0 ||
+      (elem_bytes != 2 && elem_bytes != 4))
     return B200SP_ERR_INVALID_ARG;
   DeviceInfo* dev = nullptr;
   int rc = device_info(&dev);
   if (rc != B200SP_OK) return rc;
-  static int per_sm[64] = {};
-  int d = 0;
-  CU(cudaGetDevice(&d));
-  if (!per_sm[d]) {
-    CU(cudaFuncSetAttribute(probe_gather_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, 0));
-    int nb = 0;
-    CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, probe_gather_kernel, 256, 0));
-    per_sm[d] = nb > 0 ? nb : 1;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (elem_bytes == 4)
+    return in_shared_memory ? run_probe_gather<float, true>(table, table_elems, gathers, sink, st, dev)
+                            : run_probe_gather<float, false>(table, table_elems, gathers, sink, st, dev);
+  return in_shared_memory ? run_probe_gather<unsigned short, true>(table, table_elems, gathers, sink, st, dev)
+                          : run_probe_gather<unsigned short, false>(table, table_elems, gathers, sink, st, dev);
+}
+
+int b200sp_probe_gather(const float* table, int64_t table_elems, int64_t gathers, float* sink, void* stream) {
+  return b200sp_probe_gather_ex(table, table_elems, gathers, 4, 0, sink, stream);
+}
+
+int b200sp_probe_stream(const void* buf, int64_t bytes, float* sink, void* stream) {
+  if (!buf || !sink || bytes < 0 || (bytes & 15) || !aligned16(buf)) return B200SP_ERR_INVALID_ARG;
+  DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  return launch(probe_stream_kernel, dim3((unsigned)(dev->sms * 8)), dim3(256), (cudaStream_t)stream, nullptr, 0, dev, (const int4*)buf,
+                (long long)(bytes / 16), sink);
+}
+
+int b200sp_probe_lines(const void* buf, int64_t lines, int64_t reads, int in_flight, int to_shared_memory, float* sink, void* stream) {
+  if (!buf || !sink || lines <= 0 || (lines & (lines - 1)) != 0 || lines > ((int64_t)1 << 31) || reads < 0 || !aligned16(buf) ||
+      (in_flight != 4 && in_flight != 8 && in_flight != 16))
+    return B200SP_ERR_INVALID_ARG;
+  DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  const dim3 grid((unsigned)(dev->sms * 8)), block(256);
+  const unsigned mask = (unsigned)(lines - 1);
+  const size_t smem = to_shared_memory ? (size_t)256 * in_flight * 16 : 0;
+#define B200SP_PROBE_LINES(U, A) return launch_smem(probe_lines_kernel<U, A>, grid, block, smem, st, nullptr, 0, dev, (const int4*)buf, mask, (long long)reads, sink)
+  if (to_shared_memory) {
+    if (in_flight == 4) B200SP_PROBE_LINES(4, true);
+    if (in_flight == 8) B200SP_PROBE_LINES(8, true);
+    CU(cudaFuncSetAttribute(probe_lines_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    B200SP_PROBE_LINES(16, true);
   }
-  return launch(probe_gather_kernel, dim3((unsigned)(dev->sms * per_sm[d])), dim3(256), (cudaStream_t)stream, nullptr, 0, dev, table,
-                (unsigned)(table_elems - 1), (long long)gathers, sink);
+  if (in_flight == 4) B200SP_PROBE_LINES(4, false);
+  if (in_flight == 8) B200SP_PROBE_LINES(8, false);
+  B200SP_PROBE_LINES(16, false);
+#undef B200SP_PROBE_LINES
 }
 
 int64_t b200sp_noalloc_max_items(void) { return (int64_t)kNoAllocMaxTiles * kItems; }
@@ -425,8 +480,21 @@ void b200sp_cache_clear(void) {
   g_coo_cache.clear();
   for (auto& kv : g_csc_cache) csc_free(kv.second);
   g_csc_cache.clear();
-  for (DeviceInfo& d : g_dev)
+  int cur = 0;
+  const bool have_cur = cudaGetDevice(&cur) == cudaSuccess;
+  for (int i = 0; i < 64; ++i) {
+    DeviceInfo& d = g_dev[i];
     if (d.pool) cudaMemPoolTrimTo(d.pool, 0);
+    if (d.persist_set > 0 && have_cur) {   // give the L2 set aside for the access-policy windows back
+      if (cudaSetDevice(i) == cudaSuccess) {
+        cudaCtxResetPersistingL2Cache();
+        cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, 0);
+        d.persist_set = 0;
+      }
+      cudaSetDevice(cur);
+    }
+  }
+  (void)cudaGetLastError();
 }
 
 const char* b200sp_status_string(int s) {
@@ -470,7 +538,8 @@ int b200sp_set_option(const char* name, int value) {
       {"spmv_kernel", &g_opt.spmv_kernel, false, {-1, 0, 1, 2, 3}, 0, 0},
       {"spmm_bstage", &g_opt.spmm_bstage, true, {}, 0, 0},
       {"spmm_sliced", &g_opt.spmm_sliced, true, {}, 0, 0},
-      {"spmm_ranges", &g_opt.spmm_ranges, false, {0, 1, 2, 3, 4, 5, 6, 7, 8}, 0, 0},
+      {"spmm_stage_a", &g_opt.spmm_stage_a, false, {0, 1, 2}, 0, 0},
+      {"spmm_ranges", &g_opt.spmm_ranges, false, {0, 1, 2, 3, 4, 8}, 0, 0},
       {"merge_items", &g_opt.merge_items, false, {1024, 2048, 4096}, 0, 0},
       {"merge_threads", &g_opt.merge_threads, false, {64, 128, 256}, 0, 0},
       {"merge_carve", &g_opt.merge_carve, false, {-1, 0, 25, 45, 60, 75, 100}, 0, 0},

@@ -13,23 +13,27 @@ typedef std::tuple<int, const void*, int64_t, int64_t, int64_t> PlanKey;
 struct CachedPlan { b200sp_plan* plan = nullptr; uint64_t stamp = 0; };
 std::map<PlanKey, CachedPlan> g_cache;
 uint64_t g_cache_clock = 0;
-constexpr size_t kCacheCap = 64;
+constexpr size_t kCacheCap = 1024;
 
 // Frees a plan.  With stream_ordered the block goes back to the pool in the order of `stream` (the caller
 // knows that every kernel that used the plan ran there); otherwise the device is synchronised first.
 int plan_free(b200sp_plan* p, bool stream_ordered = false, cudaStream_t stream = nullptr) {
   if (!p) return B200SP_OK;
   int rc = B200SP_OK;
-  if (p->block) {
+  if (p->block || p->cuts_block || p->compact_block) {
     cudaError_t e = cudaSuccess;
     if (stream_ordered) {
-      e = cudaFreeAsync(p->block, stream);
+      if (p->block) e = cudaFreeAsync(p->block, stream);
+      if (p->cuts_block && e == cudaSuccess) e = cudaFreeAsync(p->cuts_block, stream);
+      if (p->compact_block && e == cudaSuccess) e = cudaFreeAsync(p->compact_block, stream);
     } else {
       int cur = 0;
       e = cudaGetDevice(&cur);
       if (e == cudaSuccess && cur != p->device) e = cudaSetDevice(p->device);
       if (e == cudaSuccess) e = cudaDeviceSynchronize();
-      if (e == cudaSuccess) e = cudaFree(p->block);
+      if (e == cudaSuccess && p->block) e = cudaFree(p->block);
+      if (e == cudaSuccess && p->cuts_block) e = cudaFree(p->cuts_block);
+      if (e == cudaSuccess && p->compact_block) e = cudaFree(p->compact_block);
       if (cur != p->device) cudaSetDevice(cur);
     }
     if (e != cudaSuccess) rc = cuda_fail(e, "freeing a plan");
@@ -47,7 +51,7 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   p->row_ptr = row_ptr;
   b200sp_plan_info_t& I = p->info;
   I.m = m; I.n = n; I.nnz = nnz;
-  const int items = g_opt.merge_items == 4096 ? 4096 : (g_opt.merge_items == 1024 ? 1024 : 2048);
+  const int items = g_opt.merge_items;
   I.spmv_tile_items = items;
   I.spmv_tiles = (int32_t)((m + nnz + items - 1) / items);
   I.spmv_kernel = g_opt.spmv_kernel >= 0 ? g_opt.spmv_kernel : 0;
@@ -109,6 +113,30 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
     CUP(cudaStreamSynchronize(stream));
     p->num_medium = (int)n_mid;
     p->num_long = (int)n_long;
+  }
+  // Many rows without nonzeros (a quarter or more): the merge list is built over the rows that have nonzeros only, and the
+  // split points are searched again over that list.
+  if (!h.bad && g_opt.merge_empty && nnz > 0 && (int64_t)h.bin_rows[0] * 4 >= m) {
+    const int64_t mc = m - (int64_t)h.bin_rows[0];
+    const int blocks = (int)((m + kCompactBlock - 1) / kCompactBlock);
+    const size_t o_id = 0, o_rp = o_id + up((size_t)mc * 4), o_bc = o_rp + up((size_t)(mc + 1) * 4), tot2 = o_bc + up((size_t)(blocks + 1) * 4);
+    rc = pool_alloc(dev, &p->compact_block, tot2, stream);
+    if (rc != B200SP_OK) return fail(rc);
+    char* b2 = (char*)p->compact_block;
+    p->compact_row_id = (int32_t*)(b2 + o_id);
+    p->compact_row_ptr = (int32_t*)(b2 + o_rp);
+    int* d_bc = (int*)(b2 + o_bc);
+    plan_compact_count_kernel<<<blocks, 256, 0, stream>>>(row_ptr, (int)m, d_bc);
+    plan_compact_scan_kernel<<<1, 1024, 0, stream>>>(d_bc, blocks);
+    plan_compact_write_kernel<<<blocks, 256, 0, stream>>>(row_ptr, (int)m, (int)nnz, d_bc, p->compact_row_id, p->compact_row_ptr);
+    const size_t ntc = (size_t)((mc + nnz + items - 1) / items);     // fewer items, fewer tiles: the arrays sized above suffice
+    plan_merge_split_kernel<<<(unsigned)((ntc + 1 + 255) / 256), 256, 0, stream>>>(p->compact_row_ptr, (int)mc, (int)nnz, items, (int)ntc, p->split_row);
+    g_launches += 4;
+    CUP(cudaGetLastError());
+    CUP(cudaStreamSynchronize(stream));
+    p->compact_rows = (int)mc;
+    I.spmv_tiles = (int32_t)ntc;
+    I.scratch_bytes += (int64_t)tot2;
   }
 #undef CUP
   if (h.bad) { plan_free(p, true, stream); cudaStreamSynchronize(stream); return B200SP_ERR_BAD_CSR; }

@@ -31,6 +31,7 @@ constexpr int kRowMaxLen = 64;
 constexpr int kSmemPerSm = 227 * 1024;   // usable shared memory per SM (each CTA also reserves 1 KB)
 // SpMM
 constexpr int kSpmmThreads = 256;
+constexpr int kSpmmStageCap = 128;   // (col, val) pairs a warp of the k-sliced SpMM kernel can stage in shared memory
 constexpr int kSmallNnz = 1 << 20;   // at or below this many nonzeros SpMV uses the sub-warp-per-row kernel
 constexpr int kSubwarpChain = 128;   // longest sequential FP32 chain one lane of the sub-warp SpMV kernel may add
 constexpr int kMediumRow = 128;   // SpMM: rows longer than this are added in blocks of this many products (second-to-last length bin)
@@ -50,7 +51,7 @@ struct Options {
   int row_threads = 256;  // threads per CTA of the row-direct kernel (128 or 256)
   int uni_unroll = 0;     // groups of four nonzeros in flight per thread of the uniform-row kernel (1, 2 or 4); 0 = 1 (32 registers, full occupancy)
   int uni_ctas = 0;       // CTAs per SM for the uniform-row kernel (0 = as many as fit)
-  int merge_items = 2048; // merge items per tile (2048 or 4096)
+  int merge_items = 2048; // merge items per tile (1024, 2048 or 4096)
   int merge_threads = 128; // threads per CTA of the one-tile-per-CTA merge kernel (128 or 256)
   int bstage_threads = 1024; // threads per CTA of that kernel (256, 512 or 1024)
   int bstage_nnz = 131072;   // nonzeros per CTA it aims for
@@ -58,8 +59,9 @@ struct Options {
   int spmm_bstage = 1;     // 1 = hold the slice of B in shared memory when A has few columns (default), 0 = never
   int spmm_sliced = 1;     // 1 = k-sliced SpMM kernel (default), 0 = one pass over all of k
   int sub_lanes = 0;       // lanes per row of the sub-warp kernel (0 = from the mean row length)
-  int merge_empty = 1;     // 1 = rows without nonzeros are kept out of the merge list when the matrix has many of them (default), 0 = never
-  int spmm_ranges = 0;     // column ranges per slice of the k-sliced SpMM kernel with sorted columns: 0 = sized for L2, 1 = none, 2..8 forced
+  int merge_empty = 0;     // 1 = when a quarter or more of the rows have no nonzeros the merge list holds only the others, 0 = every row is a merge item (default: measured 3 % slower on the power-law workload, where the extra pass over y costs more than the skipped items save)
+  int spmm_stage_a = 2;    // the k-sliced SpMM kernel's warps stage their rows' (col, val) pairs in shared memory: 1 = yes, 0 = no (broadcast loads from global memory), 2 = for BF16 storage only (default)
+  int spmm_ranges = 1;     // column ranges per slice of the k-sliced SpMM kernel with sorted columns: 1 = none (default), 0 = as many as make a range of B fit L2, 2, 3, 4, 8 = forced
   int merge_short = 32;    // rows up to this many products are added by one thread (8, 16, 32, 64)
   int pdl = 1;             // 1 = launch the kernels that begin with griddepcontrol.wait with programmatic stream serialisation
   int pool_keep_mb = 1024; // freed memory the library's pool keeps across synchronisation points, MiB (read when the pool is created)
@@ -242,6 +244,16 @@ struct b200sp_plan {
   unsigned long long* probe_out = nullptr;  // two counters for the column-locality probe
   int num_medium = 0, num_long = 0;
   const void* probed_col_idx = nullptr;   // col_idx the column-locality probe last ran on
+  // merge list over the rows that have nonzeros (matrices with many empty rows)
+  void* compact_block = nullptr;          // one pool block: row ids, their offsets, block counts
+  int compact_rows = 0;                   // 0 = the merge list is the matrix's own row list
+  int32_t* compact_row_id = nullptr;      // compact_rows matrix row numbers, ascending
+  int32_t* compact_row_ptr = nullptr;     // compact_rows + 1 offsets
+  // column ranges of the k-sliced SpMM kernel (rows with ascending columns): built on the first SpMM call with a given col_idx
+  void* cuts_block = nullptr;             // (ranges - 1) * m cut positions, a pool block of its own
+  const void* cuts_col_idx = nullptr;     // col_idx they were computed from
+  int cuts_ranges = 0;                    // number of ranges they describe (0 = none computed)
+  bool cols_sorted = false;               // every row's columns ascend
   const void* probed_key = nullptr;       // host entry points: the HOST col_idx that verdict belongs to
   bool cols_local = true;                 // its verdict: adjacent rows share most of their lines of x
 };

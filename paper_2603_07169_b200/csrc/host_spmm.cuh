@@ -94,6 +94,46 @@ int launch_spmm_bstage(b200sp_plan* p, int k, const int32_t* col_idx, const T* v
                      g_opt.spin_limit, g_opt.debug_no_copies);
 }
 
+// Column ranges for the k-sliced kernel: how many, and the per-row cut positions (computed once per col_idx; one small
+// kernel and one synchronisation of the stream).  Returns 1 in *ranges when the ranges do not apply: B's slice fits L2,
+// the rows' columns are not in ascending order, or the switch says so.
+int spmm_column_ranges(b200sp_plan* p, const int32_t* col_idx, int slice_bytes, cudaStream_t stream, DeviceInfo* dev, int* ranges) {
+  const b200sp_plan_info_t& I = p->info;
+  *ranges = 1;
+  int want = g_opt.spmm_ranges;
+  if (want == 0) {
+    // a range of B (n / ranges rows of slice_bytes) should take at most this share of L2: the L2 of this part keeps a line
+    // read by all SMs in both of its halves, and the streams of A and Y pass through it as well
+    const double budget = 0.3 * (double)dev->l2_bytes;
+    want = (int)(((double)I.n * slice_bytes + budget - 1) / budget);
+    if (want > 8) want = 8;
+  }
+  if (want <= 1 || I.n < want || I.m < 1) return B200SP_OK;
+  if (p->cuts_col_idx == (const void*)col_idx && p->cuts_ranges == want) { if (p->cols_sorted) *ranges = want; return B200SP_OK; }
+  if (p->cuts_block) { CU(cudaFreeAsync(p->cuts_block, stream)); p->cuts_block = nullptr; p->cuts_ranges = 0; p->cuts_col_idx = nullptr; }
+  const size_t bytes = (size_t)(want - 1) * (size_t)I.m * 4 + 256;
+  void* blk = nullptr;
+  int rc = pool_alloc(dev, &blk, bytes, stream);
+  if (rc != B200SP_OK) return rc;
+  int* flag = (int*)((char*)blk + (size_t)(want - 1) * (size_t)I.m * 4);
+  int h = 0;
+  cudaError_t e = cudaMemsetAsync(flag, 0, sizeof(int), stream);
+  if (e == cudaSuccess) {
+    spmm_range_cuts_kernel<<<(unsigned)((I.m + 255) / 256), 256, 0, stream>>>((int)I.m, (int)I.n, want, p->row_ptr, col_idx, (int*)blk, flag);
+    g_launches++;
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&h, flag, sizeof(int), cudaMemcpyDeviceToHost, stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) { cudaFreeAsync(blk, stream); return cuda_fail(e, "column ranges"); }
+  p->cuts_block = blk;
+  p->cuts_col_idx = col_idx;
+  p->cuts_ranges = want;
+  p->cols_sorted = h == 0;
+  if (p->cols_sorted) *ranges = want;
+  return B200SP_OK;
+}
+
 template <typename T, int VEC>
 int run_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const T* B, T* Y, float alpha, float beta,
              cudaStream_t stream, DeviceInfo* dev) {
@@ -134,12 +174,42 @@ int run_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const
     if ((long long)slices * row_blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
     int rc;
     const int mid_blocks = (p->num_medium + GROUPS - 1) / GROUPS;
+    int ranges = 1;
+    if (lanes == 8) {
+      rc = spmm_column_ranges(p, col_idx, 8 * 16, stream, dev, &ranges);
+      if (rc != B200SP_OK) return rc;
+    }
+    if (ranges > 1) {
+      // one launch per column range; FP32 partial sums for BF16 storage come from the pool and go back in stream order
+      float* partial = nullptr;
+      if (sizeof(T) == 2) {
+        rc = pool_alloc(dev, (void**)&partial, (size_t)I.m * (size_t)k * sizeof(float), stream);
+        if (rc != B200SP_OK) return rc;
+      }
+      for (int r = 0; r < ranges && rc == B200SP_OK; ++r) {
+        tl_pdl_kernel = true;
+        rc = launch(spmm_slice_range_kernel<T, VEC, kSpmmThreads, 8>, dim3((unsigned)(slices * row_blocks)), dim3(kSpmmThreads), stream, nullptr, 0,
+                    dev, (int)I.m, k, row_blocks, r, ranges, (const int*)p->cuts_block, p->row_ptr, col_idx, vals, B, Y, partial, alpha, beta,
+                    kMediumRow);
+      }
+      if (partial) { const cudaError_t e = cudaFreeAsync(partial, stream); if (e != cudaSuccess && rc == B200SP_OK) rc = cuda_fail(e, "cudaFreeAsync"); }
+      if (rc == B200SP_OK && p->num_medium > 0) {
+        tl_pdl_kernel = true;
+        rc = launch(spmm_medium_row_kernel<T, VEC, kSpmmThreads, 8>, dim3((unsigned)(slices * mid_blocks)), dim3(kSpmmThreads), stream,
+                    nullptr, 0, dev, p->num_medium, (const int*)p->medium_rows, k, mid_blocks, p->row_ptr, col_idx, vals, B, Y, alpha, beta);
+      }
+    } else
     // rows of at most kMediumRow nonzeros: the register-capped kernel; kMediumRow + 1 .. kLongRow: the same scheme with
     // blocked sums over the plan's list of such rows; longer rows: a CTA per (row, slice)
 #define B200SP_SLICE_LAUNCH(L)                                                                                                      \
     tl_pdl_kernel = true;                                                                                                           \
-    rc = launch(spmm_slice_kernel<T, VEC, kSpmmThreads, L>, dim3((unsigned)(slices * row_blocks)), dim3(kSpmmThreads), stream, nullptr, 0, \
-                dev, (int)I.m, k, row_blocks, p->row_ptr, col_idx, vals, B, Y, alpha, beta, kMediumRow);                            \
+    if ((g_opt.spmm_stage_a == 1 || (g_opt.spmm_stage_a == 2 && sizeof(T) == 2)) && L > 1)                                          \
+      rc = launch(spmm_slice_staged_kernel<T, VEC, kSpmmThreads, (L > 1 ? L : 2), kSpmmStageCap>, dim3((unsigned)(slices * row_blocks)),  \
+                  dim3(kSpmmThreads), stream, B, (size_t)I.n * k * sizeof(T), dev, (int)I.m, (int)I.nnz, k, row_blocks, p->row_ptr, col_idx, vals, B, Y, alpha, \
+                  beta, kMediumRow);                                                                                                \
+    else                                                                                                                            \
+      rc = launch(spmm_slice_kernel<T, VEC, kSpmmThreads, L>, dim3((unsigned)(slices * row_blocks)), dim3(kSpmmThreads), stream, B,       \
+                  (size_t)I.n * k * sizeof(T), dev, (int)I.m, k, row_blocks, p->row_ptr, col_idx, vals, B, Y, alpha, beta, kMediumRow);                          \
     if (rc == B200SP_OK && p->num_medium > 0) {                                                                                     \
       tl_pdl_kernel = true;                                                                                                         \
       rc = launch(spmm_medium_row_kernel<T, VEC, kSpmmThreads, L>, dim3((unsigned)(slices * mid_blocks)), dim3(kSpmmThreads), stream, \

@@ -5,6 +5,7 @@
 #include "spmv_kernels.cuh"
 #include "spmv_row_kernels.cuh"
 #include "spmv_uniform_kernels.cuh"
+#include "probe_kernels.cuh"
 
 namespace {
 
@@ -157,36 +158,46 @@ int run_spmv_uniform(b200sp_plan* p, const int32_t* col_idx, const T* vals, cons
   return B200SP_ERR_UNSUPPORTED;
 }
 
+// y of the rows that are not in a merge list of non-empty rows: y = beta * y (zero when beta == 0).
+template <typename T>
+int run_empty_rows(b200sp_plan* p, T* y, float beta, cudaStream_t stream, DeviceInfo* dev) {
+  const b200sp_plan_info_t& I = p->info;
+  if (beta == 0.0f) return run_scale<T>(I.m, y, 0.0f, stream, dev);
+  long long blocks = (I.m + 255) / 256;
+  if (blocks > (long long)dev->sms * 16) blocks = (long long)dev->sms * 16;
+  return launch(scale_empty_rows_kernel<T>, dim3((unsigned)blocks), dim3(256), stream, nullptr, 0, dev, (long long)I.m, p->row_ptr, y, beta);
+}
+
 template <typename T, int ITEMS, int SHORT = kShortMax>
 int run_spmv_merge(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
                    cudaStream_t stream, DeviceInfo* dev) {
   const b200sp_plan_info_t& I = p->info;
   const int tiles = I.spmv_tiles;
-  int rc;
-  if (g_opt.merge_threads == 64) {
-    auto kernel = spmv_merge_tile_kernel<T, ITEMS, 64, SHORT>;
-    if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
-    tl_pdl_kernel = true;
-    rc = launch(kernel, dim3(tiles), dim3(64), stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx,
-                vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail);
-  } else if (g_opt.merge_threads == 128) {
-    auto kernel = spmv_merge_tile_kernel<T, ITEMS, 128, SHORT>;
-    if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
-    tl_pdl_kernel = true;
-    rc = launch(kernel, dim3(tiles), dim3(128), stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx,
-                vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail);
-  } else {
-    auto kernel = spmv_merge_tile_kernel<T, ITEMS, kThreads, kShortMax>;
-    if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));
-    tl_pdl_kernel = true;
-    rc = launch(kernel, dim3(tiles), dim3(kThreads), stream, x, (size_t)I.n * sizeof(T), dev, (int)I.m, (int)I.nnz, p->row_ptr, col_idx,
-                vals, x, y, alpha, beta, (const int*)p->split_row, p->carry, p->tail);
+  const int rows = p->compact_rows > 0 ? p->compact_rows : (int)I.m;
+  const int* rp = p->compact_rows > 0 ? p->compact_row_ptr : p->row_ptr;
+  const int* rid = p->compact_rows > 0 ? p->compact_row_id : nullptr;
+  int rc = B200SP_OK;
+  if (rid) {
+    rc = run_empty_rows<T>(p, y, beta, stream, dev);
+    if (rc != B200SP_OK) return rc;
   }
+#define B200SP_MERGE_LAUNCH(TH)                                                                                                          \
+  {                                                                                                                                      \
+    auto kernel = spmv_merge_tile_kernel<T, ITEMS, TH, SHORT>;                                                                           \
+    if (g_opt.merge_carve >= 0) CU(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, g_opt.merge_carve));    \
+    tl_pdl_kernel = true;                                                                                                                \
+    rc = launch(kernel, dim3(tiles), dim3(TH), stream, x, (size_t)I.n * sizeof(T), dev, rows, (int)I.nnz, rp, col_idx, vals, x, y, alpha, \
+                beta, (const int*)p->split_row, p->carry, p->tail, rid);                                                                 \
+  }
+  if (g_opt.merge_threads == 64) B200SP_MERGE_LAUNCH(64)
+  else if (g_opt.merge_threads == 128) B200SP_MERGE_LAUNCH(128)
+  else B200SP_MERGE_LAUNCH(256)
+#undef B200SP_MERGE_LAUNCH
   if (rc != B200SP_OK) return rc;
   if (tiles > 1) {
     tl_pdl_kernel = true;
-    rc = launch(spmv_carry_fixup_kernel<T, ITEMS>, dim3((tiles + 127) / 128), dim3(128), stream, nullptr, 0, dev, tiles,
-                p->row_ptr, (const int*)p->split_row, (const float*)p->carry, (const float*)p->tail, y, alpha, beta);
+    rc = launch(spmv_carry_fixup_kernel<T, ITEMS>, dim3((tiles + 127) / 128), dim3(128), stream, nullptr, 0, dev, tiles, rp,
+                (const int*)p->split_row, (const float*)p->carry, (const float*)p->tail, y, alpha, beta, rid);
   }
   return rc;
 }
@@ -224,6 +235,22 @@ int run_spmv_subwarp(b200sp_plan* p, const int32_t* col_idx, const T* vals, cons
   }
 }
 
+// The merge-tile kernel by tile size and by the length up to which one thread adds a row.
+template <typename T>
+int run_spmv_merge_any(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, T* y, float alpha, float beta,
+                       cudaStream_t stream, DeviceInfo* dev) {
+  const int items = p->info.spmv_tile_items, sh = g_opt.merge_short;
+#define B200SP_MERGE_BY_SHORT(FN, ITEMS)                                                      \
+  if (sh == 8) return FN<T, ITEMS, 8>(p, col_idx, vals, x, y, alpha, beta, stream, dev);      \
+  if (sh == 16) return FN<T, ITEMS, 16>(p, col_idx, vals, x, y, alpha, beta, stream, dev);    \
+  if (sh == 64) return FN<T, ITEMS, 64>(p, col_idx, vals, x, y, alpha, beta, stream, dev);    \
+  return FN<T, ITEMS, 32>(p, col_idx, vals, x, y, alpha, beta, stream, dev)
+  if (items == 4096) return run_spmv_merge<T, 4096>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  if (items == 1024) return run_spmv_merge<T, 1024>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  B200SP_MERGE_BY_SHORT(run_spmv_merge, 2048);
+#undef B200SP_MERGE_BY_SHORT
+}
+
 // The row-direct kernel gives its shared memory to stages and leaves little L1; that pays only when the gather of x is
 // local (adjacent rows share lines).  The first call with a given col_idx samples that property (one small kernel, one
 // synchronisation); matrices with scattered columns go to the merge-tile kernel instead.
@@ -258,20 +285,13 @@ int run_spmv(b200sp_plan* p, const int32_t* col_idx, const T* vals, const T* x, 
     const int rc = probe_col_locality(p, col_idx, stream);
     if (rc != B200SP_OK) return rc;
     if (!p->cols_local) {
-      if (I.spmv_tile_items == 4096) return run_spmv_merge<T, 4096>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
-      if (I.spmv_tile_items == 1024) return run_spmv_merge<T, 1024>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
-      return run_spmv_merge<T, 2048>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+      return run_spmv_merge_any<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
     }
   }
   if (I.spmv_kernel == 3) return run_spmv_subwarp<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (I.spmv_kernel == 2) return run_spmv_uniform<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
   if (I.spmv_kernel == 1) return run_spmv_row_direct<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
-  if (I.spmv_tile_items == 4096) return run_spmv_merge<T, 4096>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
-  if (I.spmv_tile_items == 1024) return run_spmv_merge<T, 1024>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
-  if (g_opt.merge_short == 8) return run_spmv_merge<T, 2048, 8>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
-  if (g_opt.merge_short == 16) return run_spmv_merge<T, 2048, 16>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
-  if (g_opt.merge_short == 64) return run_spmv_merge<T, 2048, 64>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
-  return run_spmv_merge<T, 2048>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
+  return run_spmv_merge_any<T>(p, col_idx, vals, x, y, alpha, beta, stream, dev);
 }
 
 }  // namespace

@@ -66,6 +66,84 @@ __global__ void __launch_bounds__(256) plan_merge_split_kernel(const int* __rest
   split_row[t] = lo;
 }
 
+// ---- list of the rows that have nonzeros (for matrices with many empty rows) ----
+// Three passes: non-empty rows per block of kCompactBlock rows; an exclusive scan of the block counts by one CTA; then every
+// block writes its rows' numbers and offsets at its place.  Integer work only; the order of the list is the row order.
+constexpr int kCompactBlock = 1024;
+
+__global__ void __launch_bounds__(256) plan_compact_count_kernel(const int* __restrict__ row_ptr, int m, int* __restrict__ block_count) {
+  __shared__ int s_count;
+  if (threadIdx.x == 0) s_count = 0;
+  __syncthreads();
+  const long long base = (long long)blockIdx.x * kCompactBlock;
+  int c = 0;
+  for (int j = threadIdx.x; j < kCompactBlock; j += 256) {
+    const long long r = base + j;
+    if (r < m && row_ptr[r + 1] > row_ptr[r]) ++c;
+  }
+  atomicAdd(&s_count, c);
+  __syncthreads();
+  if (threadIdx.x == 0) block_count[blockIdx.x] = s_count;
+}
+
+// block_count[b] <- sum of block_count[0 .. b-1]; block_count[blocks] <- total.  One CTA of 1024 threads.
+__global__ void __launch_bounds__(1024) plan_compact_scan_kernel(int* __restrict__ block_count, int blocks) {
+  __shared__ int s_warp[32];
+  __shared__ int s_base;
+  if (threadIdx.x == 0) s_base = 0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int b0 = 0; b0 < blocks; b0 += 1024) {
+    const int b = b0 + threadIdx.x;
+    const int v = b < blocks ? block_count[b] : 0;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int w = s_warp[lane];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, w, o); if (lane >= o) w += t; }
+      s_warp[lane] = w;
+    }
+    __syncthreads();
+    const int before = s_base + (warp > 0 ? s_warp[warp - 1] : 0) + incl - v;
+    if (b < blocks) block_count[b] = before;
+    __syncthreads();
+    if (threadIdx.x == 1023) s_base = before + v;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) block_count[blocks] = s_base;
+}
+
+__global__ void __launch_bounds__(256) plan_compact_write_kernel(const int* __restrict__ row_ptr, int m, int nnz, const int* __restrict__ block_offset,
+                                                                 int* __restrict__ row_id, int* __restrict__ row_ptr_c) {
+  __shared__ int s_warp[8];
+  const long long base = (long long)blockIdx.x * kCompactBlock;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int out = block_offset[blockIdx.x];
+  for (int j0 = 0; j0 < kCompactBlock; j0 += 256) {     // rows in order: four rounds of 256 consecutive rows
+    const long long r = base + j0 + threadIdx.x;
+    int rs = 0, flag = 0;
+    if (r < m) { rs = row_ptr[r]; flag = row_ptr[r + 1] > rs ? 1 : 0; }
+    const unsigned ballot = __ballot_sync(0xFFFFFFFFu, flag);
+    if (lane == 0) s_warp[warp] = __popc(ballot);
+    __syncthreads();
+    int before = 0, round_total = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { const int c = s_warp[w]; if (w < warp) before += c; round_total += c; }
+    if (flag) {
+      const int slot = out + before + __popc(ballot & ((1u << lane) - 1u));
+      row_id[slot] = (int)r;
+      row_ptr_c[slot] = rs;
+    }
+    out += round_total;
+    __syncthreads();
+  }
+  if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) row_ptr_c[out] = nnz;
+}
+
 // Rows of mid_thresh + 1 .. long_thresh nonzeros and rows longer than long_thresh, each appended to a list of its own
 // (count[0], count[1]; the host sorts the lists, and their order only affects scheduling, never a value).
 __global__ void __launch_bounds__(256) plan_row_lists_kernel(const int* __restrict__ row_ptr, int m, int mid_thresh, int long_thresh,

@@ -1,0 +1,102 @@
+// Measurement probes: the hardware rates that bound the SpMV / SpMM kernels, measured by kernels that do nothing else.
+// They have no counterpart in the paper's operations; the paper's Appendix A sorts kernels by which rate limits them
+// (compute, memory latency, memory bandwidth), and these probes give the denominators for this part.
+//   probe_gather_kernel   random reads of a table: the rate at which an SM takes L1 misses (table >> L1), L1 hits (table fits L1)
+//                         or shared-memory reads (table staged in shared memory) -- the bound on gathering x
+//   probe_stream_kernel   coalesced 128-bit reads of a buffer: what a pure stream of the CSR arrays can reach at a given size
+//   probe_lines_kernel    random reads of whole 128-byte lines by groups of eight lanes: the L2-to-SM path that SpMM's reads of B use
+#pragma once
+#include "common.cuh"
+
+namespace b200sp {
+
+__device__ __forceinline__ unsigned probe_hash(unsigned long long i) {
+  unsigned long long z = i * 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z ^= z >> 27;
+  return (unsigned)(z >> 20);
+}
+
+// `gathers` independent reads of table[hash(i) & mask] (mask + 1 a power of two), eight in flight per thread, indices made in
+// registers so that nothing but the gather touches memory.  ELEM = 4 or 2 bytes per entry.  SMEM: the table (at most
+// smem_elems entries) is first copied into shared memory and gathered from there.
+template <typename E, bool SMEM>
+__global__ void __launch_bounds__(256) probe_gather_kernel(const E* __restrict__ table, unsigned mask, long long gathers,
+                                                           float* __restrict__ sink) {
+  extern __shared__ __align__(16) unsigned char probe_smem[];
+  const E* src = table;
+  if (SMEM) {
+    E* t = reinterpret_cast<E*>(probe_smem);
+    for (unsigned i = threadIdx.x; i <= mask; i += blockDim.x) t[i] = table[i];
+    __syncthreads();
+    src = t;
+  }
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  float s = 0.0f;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < gathers; i += stride * 8) {
+    E v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const unsigned idx = probe_hash((unsigned long long)(i + u * stride)) & mask;
+      v[u] = (i + u * stride < gathers) ? (SMEM ? src[idx] : __ldg(src + idx)) : E(0);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) s += (float)v[u];
+  }
+  if (s == 1.2345e-30f) *sink = s;   // keeps the loads alive; practically never true
+}
+
+// Streams `bytes` (a multiple of 16) once with coalesced 128-bit loads that do not allocate in L1.
+__global__ void __launch_bounds__(256) probe_stream_kernel(const int4* __restrict__ buf, long long vecs, float* __restrict__ sink) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  int acc = 0;
+  long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  for (; i + 3 * stride < vecs; i += 4 * stride) {
+    const int4 a = ld_stream_i4((const int*)(buf + i)), b = ld_stream_i4((const int*)(buf + i + stride));
+    const int4 c = ld_stream_i4((const int*)(buf + i + 2 * stride)), d = ld_stream_i4((const int*)(buf + i + 3 * stride));
+    acc ^= a.x ^ a.y ^ a.z ^ a.w ^ b.x ^ b.y ^ b.z ^ b.w ^ c.x ^ c.y ^ c.z ^ c.w ^ d.x ^ d.y ^ d.z ^ d.w;
+  }
+  for (; i < vecs; i += stride) { const int4 a = ld_stream_i4((const int*)(buf + i)); acc ^= a.x ^ a.y ^ a.z ^ a.w; }
+  if (acc == 0x5A5A1234) *sink = (float)acc;
+}
+
+// `reads` random 128-byte lines of a buffer of `lines` lines (a power of two): every group of eight lanes reads one line, 16 bytes
+// per lane, U lines in flight per group -- the access pattern of the k-sliced SpMM kernel's reads of B (which keeps U = 4 in
+// registers).  ASYNC: the lines go to shared memory with cp.async (16 bytes per lane) instead of registers, so the bytes in
+// flight are bounded by shared memory rather than by the register file.
+template <int U, bool ASYNC>
+__global__ void __launch_bounds__(256) probe_lines_kernel(const int4* __restrict__ buf, unsigned line_mask, long long reads,
+                                                          float* __restrict__ sink) {
+  extern __shared__ __align__(16) unsigned char probe_smem[];
+  const long long groups = ((long long)gridDim.x * blockDim.x) >> 3;
+  const long long g = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
+  const int l8 = threadIdx.x & 7;
+  int acc = 0;
+  int4* mine = reinterpret_cast<int4*>(probe_smem) + (size_t)threadIdx.x * U;
+  for (long long i = g; i < reads; i += groups * U) {
+    if (ASYNC) {
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const unsigned line = probe_hash((unsigned long long)(i + u * groups)) & line_mask;
+        const unsigned dst = (unsigned)__cvta_generic_to_shared(mine + u);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(buf + (size_t)line * 8 + l8) : "memory");
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+#pragma unroll
+      for (int u = 0; u < U; ++u) { const int4 v = mine[u]; acc ^= v.x ^ v.y ^ v.z ^ v.w; }
+    } else {
+      int4 v[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const unsigned line = probe_hash((unsigned long long)(i + u * groups)) & line_mask;
+        v[u] = (i + u * groups < reads) ? __ldg(buf + (size_t)line * 8 + l8) : make_int4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) acc ^= v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+    }
+  }
+  if (acc == 0x5A5A1234) *sink = (float)acc;
+}
+
+}  // namespace b200sp

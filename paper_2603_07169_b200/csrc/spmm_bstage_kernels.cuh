@@ -32,20 +32,6 @@ template <typename T> struct RawFromSmem;
 template <> struct RawFromSmem<float> { typedef float4 type; };
 template <> struct RawFromSmem<bf16_t> { typedef uint4 type; };
 
-// four consecutive (col, val) pairs from a shared-memory buffer (index a multiple of 4)
-__device__ __forceinline__ void lds_a4(const int* col_s, const float* val_s, int q, int (&c)[4], float (&v)[4]) {
-  const int4 cc = *(const int4*)(col_s + q);
-  const float4 vv = *(const float4*)(val_s + q);
-  c[0] = cc.x; c[1] = cc.y; c[2] = cc.z; c[3] = cc.w; v[0] = vv.x; v[1] = vv.y; v[2] = vv.z; v[3] = vv.w;
-}
-__device__ __forceinline__ void lds_a4(const int* col_s, const bf16_t* val_s, int q, int (&c)[4], float (&v)[4]) {
-  const int4 cc = *(const int4*)(col_s + q);
-  const uint2 vv = *(const uint2*)(val_s + q);
-  c[0] = cc.x; c[1] = cc.y; c[2] = cc.z; c[3] = cc.w;
-  v[0] = __uint_as_float(vv.x << 16); v[1] = __uint_as_float(vv.x & 0xFFFF0000u);
-  v[2] = __uint_as_float(vv.y << 16); v[3] = __uint_as_float(vv.y & 0xFFFF0000u);
-}
-
 // Dynamic shared memory: [ slice of B: bslice_bytes | per warp: (capw + 4) ints, (capw + 4) values ]; capw + 4 is a multiple of 8.
 template <typename T, int VEC, int LANES, int THREADS>
 __global__ void __launch_bounds__(THREADS)

@@ -11,6 +11,8 @@
 // A row cut by a tile boundary is not written by the tiles: each tile stores the partial sum of its
 // unfinished last row in carry[t], the tile that holds the row's end stores its part in tail[t], and
 // the fix-up kernel adds these in tile order and applies the epilogue once.  No atomics on floats.
+// The merge list's rows are either the matrix's own rows (row_id == nullptr) or, for matrices with many empty rows, the rows that
+// have nonzeros (m of them, row_ptr their m + 1 offsets, row_id[r] the matrix row of list row r).
 #pragma once
 #include "common.cuh"
 
@@ -22,7 +24,8 @@ template <typename T, int ITEMS, int THREADS, int SHORT_MAX>
 __global__ void __launch_bounds__(THREADS)
 spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const int* __restrict__ col_idx,
                        const T* __restrict__ vals, const T* __restrict__ x, T* __restrict__ y, float alpha, float beta,
-                       const int* __restrict__ split_row, float* __restrict__ carry, float* __restrict__ tail) {
+                       const int* __restrict__ split_row, float* __restrict__ carry, float* __restrict__ tail,
+                       const int* __restrict__ row_id) {
   constexpr int G = 4;                      // nonzeros per vector load
   constexpr int PROD_N = ITEMS + 2 * G;     // products of one tile, counted from the aligned start
   constexpr int MAX_LONG = ITEMS / (SHORT_MAX + 1) + 2;
@@ -102,7 +105,7 @@ spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const in
       float acc = 0.0f;
       for (int q = s - a0; q < re - a0; ++q) acc += prod[pad_index(q)];
       if (rs < p0) tail[t] = acc;            // row began in an earlier tile: completed by the fix-up kernel
-      else epilogue_store(y, r, acc, alpha, beta);
+      else epilogue_store(y, row_id ? (long long)__ldg(row_id + r) : (long long)r, acc, alpha, beta);
     } else {
       const int slot = atomicAdd(&n_long, 1);  // order of the list does not affect any value
       long_rows[slot] = rs < p0 ? -r - 1 : r;
@@ -122,7 +125,7 @@ spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const in
     acc = warp_sum(acc);
     if (lane == 0) {
       if (r < 0) tail[t] = acc;
-      else epilogue_store(y, r, acc, alpha, beta);
+      else epilogue_store(y, row_id ? (long long)__ldg(row_id + r) : (long long)r, acc, alpha, beta);
     }
   }
   if (warp == WARPS - 1) {
@@ -142,7 +145,8 @@ spmv_merge_tile_kernel(int m, int nnz, const int* __restrict__ row_ptr, const in
 template <typename T, int ITEMS>
 __global__ void __launch_bounds__(128)
 spmv_carry_fixup_kernel(int tiles, const int* __restrict__ row_ptr, const int* __restrict__ split_row,
-                        const float* __restrict__ carry, const float* __restrict__ tail, T* __restrict__ y, float alpha, float beta) {
+                        const float* __restrict__ carry, const float* __restrict__ tail, T* __restrict__ y, float alpha, float beta,
+                        const int* __restrict__ row_id) {
   grid_dependency_wait();
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t < 1 || t >= tiles) return;
@@ -155,7 +159,14 @@ spmv_carry_fixup_kernel(int tiles, const int* __restrict__ row_ptr, const int* _
   float acc = 0.0f;
   for (int u = tf; u < t; ++u) acc += carry[u];
   acc += tail[t];
-  epilogue_store(y, r0, acc, alpha, beta);
+  epilogue_store(y, row_id ? (long long)row_id[r0] : (long long)r0, acc, alpha, beta);
+}
+
+// y[i] = beta * y[i] for the rows without nonzeros (beta != 0): the pass that goes with a merge list of non-empty rows.
+template <typename T>
+__global__ void __launch_bounds__(256) scale_empty_rows_kernel(long long m, const int* __restrict__ row_ptr, T* __restrict__ y, float beta) {
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < m; i += (long long)gridDim.x * blockDim.x)
+    if (row_ptr[i] == row_ptr[i + 1]) epilogue_store(y, i, 0.0f, 0.0f, beta);
 }
 
 // y = beta * y (or 0 when beta == 0): used when alpha == 0 or the matrix has no nonzeros.

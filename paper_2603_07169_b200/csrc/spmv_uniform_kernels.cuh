@@ -63,29 +63,6 @@ spmv_uniform_vec_kernel(long long quads, const int* __restrict__ col_idx, const 
   }
 }
 
-// Measurement aid: `gathers` independent 4-byte reads of table[hash(i) & mask] (mask + 1 a power of two),
-// eight in flight per thread, indices made in registers so that nothing but the gather touches memory.
-// Timed by the caller, it gives the rate at which an SM can take random reads that miss L1 -- the bound
-// that applies to x gathers over a vector much larger than L1.
-__global__ void __launch_bounds__(256) probe_gather_kernel(const float* __restrict__ table, unsigned mask, long long gathers,
-                                                           float* __restrict__ sink) {
-  const long long stride = (long long)gridDim.x * blockDim.x;
-  float s = 0.0f;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < gathers; i += stride * 8) {
-    float v[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      unsigned long long z = (unsigned long long)(i + u * stride) * 0x9E3779B97F4A7C15ull;
-      z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
-      z ^= z >> 27;
-      v[u] = (i + u * stride < gathers) ? __ldg(table + ((unsigned)(z >> 20) & mask)) : 0.0f;
-    }
-#pragma unroll
-    for (int u = 0; u < 8; ++u) s += v[u];
-  }
-  if (s == 1.2345e-30f) *sink = s;   // keeps the loads alive; practically never true
-}
-
 }  // namespace b200sp
 
 namespace b200sp {

@@ -144,22 +144,29 @@ def test_workloads_full_size(name):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("empty", [1, 0])
 @pytest.mark.parametrize("items", [1024, 2048, 4096])
-def test_merge_kernel_tile_sizes(items, dtype):
-    """The merge-tile kernel at its three tile sizes on power-law rows, every row length, and a long run of empty rows."""
+def test_merge_kernel_tile_sizes(items, empty, dtype):
+    """The merge-tile kernel at its three tile sizes on power-law rows, every row length, and a long run of empty rows, with
+    and without the list of non-empty rows."""
     b200sp.b200sp_set_option("spmv_kernel", 0)
     b200sp.b200sp_set_option("merge_items", items)
+    b200sp.b200sp_set_option("merge_empty", empty)
     try:
         rng = np.random.default_rng(items)
         for name, lens in (("power_law", (rng.pareto(1.1, 40000) * 2).astype(np.int64).clip(0, 60000)),
                            ("every_length", np.arange(300)), ("empty_run", np.concatenate([np.zeros(20000, np.int64), [5000, 1, 0, 7]]))):
             A = gen.random_csr(len(lens), 3001, lens, seed=7)
             x = rng.standard_normal(3001).astype(np.float32)
+            y0 = rng.standard_normal(len(lens)).astype(np.float32)
             y, y_ref, S = run_spmv(A, x, None, 1.0, 0.0, dtype)
             assert_within(y, y_ref, S, dtype, what="%s items=%d" % (name, items))
+            y, y_ref, S = run_spmv(A, x, y0, 2.0, -0.5, dtype)
+            y0f = y0 if dtype == "f32" else gen.bf16_to_f32(gen.to_bf16(y0))
+            assert_within(y, y_ref, S, dtype, 2.0, np.abs(0.5 * y0f.astype(np.float64)), what="%s items=%d ab" % (name, items))
         b200sp.b200sp_check()
     finally:
-        for k, v in (("spmv_kernel", -1), ("merge_items", 2048)):
+        for k, v in (("spmv_kernel", -1), ("merge_items", 2048), ("merge_empty", 0)):
             b200sp.b200sp_set_option(k, v)
 
 
@@ -283,7 +290,16 @@ def test_plan_info_matches_numpy():
     for j, (lo, hi) in enumerate(edges):
         sel = (L >= lo) & (L <= hi)
         assert info["bin_rows"][j] == sel.sum() and info["bin_nnz"][j] == L[sel].sum()
-    assert info["spmv_tiles"] == -(-(A.m + A.nnz) // info["spmv_tile_items"]) and info["spmv_tile_items"] in (2048, 4096)
+    assert info["spmv_tile_items"] in (1024, 2048, 4096)
+    assert info["spmv_tiles"] == -(-(A.m + A.nnz) // info["spmv_tile_items"])
+    b200sp.b200sp_set_option("merge_empty", 1)      # the merge list over the non-empty rows only (61 % of this matrix's rows are empty)
+    try:
+        plan = b200sp.b200sp_plan_create(A.m, A.n, A.nnz, d_rp)
+        info2 = b200sp.b200sp_plan_info(plan)
+        b200sp.b200sp_plan_destroy(plan)
+    finally:
+        b200sp.b200sp_set_option("merge_empty", 0)
+    assert info2["spmv_tiles"] == -(-(int((L > 0).sum()) + A.nnz) // info2["spmv_tile_items"])
     assert info["spmv_kernel"] == 0          # power-law rows: merge-tile kernel
     w = gen.workload("c4", scale_down=2)
     plan = b200sp.b200sp_plan_create(w.A.m, w.A.n, w.A.nnz, to_dev(w.A.row_ptr))
