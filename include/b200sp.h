@@ -138,11 +138,12 @@ int b200sp_spmm(b200sp_plan* plan, int64_t k, const int32_t* col_idx, const void
  * out-of-range row indices return B200SP_ERR_UNSUPPORTED.  b200sp_cache_clear drops the cached offsets.
  *
  * CSC (tasks 10 / 11: values, row_indices, col_offsets of cols + 1 entries): the first call for a given
- * (device, col_ptr, row_idx, m, n, nnz) copies the pattern to the host, builds the row-major order of the
- * entries there (a stable counting sort by row, so a row's entries are added in ascending column order on every
- * run), uploads it and caches it together with a scratch array of nnz values; it synchronises the stream.
- * Every call then permutes vals into that order with one kernel and runs the CSR kernels.  Inconsistent
- * col_ptr / row_idx return B200SP_ERR_BAD_CSR.  Calls that share a cached pattern must not overlap on the GPU.
+ * (device, col_ptr, row_idx, m, n, nnz) builds the row-major order of the entries on the device (row counts, an
+ * exclusive scan, placement, and a sort of every row's entries by their CSC position, so that a row's entries are
+ * added in ascending column order on every run) and caches it together with a scratch array of nnz values; it
+ * synchronises the stream twice.  Every call then permutes vals into that order with one kernel and runs the
+ * CSR kernels.  Inconsistent col_ptr / row_idx return B200SP_ERR_BAD_CSR.  Calls that share a cached pattern
+ * must not overlap on the GPU.
  *
  * ELL: row-major, row i occupies entries [i*width, (i+1)*width) of col_ids and vals; an entry is padding
  * when its col_id is negative (its value is ignored, whatever it holds).  m * width < 2^31.  No plan, no
@@ -215,6 +216,10 @@ int b200sp_cache_drop(const void* key_ptr);
 const char* b200sp_status_string(int status);  /* static string, never NULL */
 const char* b200sp_last_cuda_error(void);      /* message of this thread's last failing CUDA call, "" if none */
 int b200sp_version(void);                      /* major * 10000 + minor * 100 + patch */
+/* 1 if the library was built with -DB200SP_BOUNDS_CHECK (libb200sp_check.so): every SpMV / SpMM call then validates the matrix
+ * on the device as b200sp_validate_csr does (one more kernel and one synchronisation of the stream per call) and returns
+ * B200SP_ERR_BAD_CSR, launching nothing else, if row_ptr or a column index is out of range.  0 for the ordinary build. */
+int b200sp_checked_build(void);
 
 /* Synchronises `stream`, then reports whether any kernel of this library on the current device gave up
  * on a bounded wait (a staged copy that never signalled its barrier): B200SP_ERR_TIMEOUT if so (the

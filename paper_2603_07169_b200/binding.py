@@ -12,14 +12,15 @@ import os
 from typing import Optional
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libb200sp.so")
+# B200SP_LIBRARY selects another build of the same library by file name (libb200sp_check.so: the checked build)
+LIB_PATH = os.path.join(_HERE, os.environ.get("B200SP_LIBRARY", "libb200sp.so"))
 
 F32, BF16 = 0, 1
 
 EXPORTS = (
     "spmv_csr", "spmm_csr", "b200sp_plan_create", "b200sp_plan_destroy", "b200sp_plan_info", "b200sp_spmv",
     "b200sp_spmm", "spmv_csr_host", "spmm_csr_host", "b200sp_validate_csr", "b200sp_cache_clear",
-    "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_launch_count", "b200sp_set_option",
+    "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_checked_build", "b200sp_launch_count", "b200sp_set_option",
     "b200sp_check", "b200sp_cache_drop", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_probe_gather_ex", "b200sp_probe_stream", "b200sp_probe_lines", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell", "spmv_csc", "spmm_csc", "spmv_csr_vec_host",
 )
 
@@ -102,6 +103,7 @@ def lib() -> ctypes.CDLL:
         L.b200sp_status_string.restype = ctypes.c_char_p
         L.b200sp_last_cuda_error.restype = ctypes.c_char_p
         L.b200sp_version.restype = i32
+        L.b200sp_checked_build.restype = i32
         L.b200sp_launch_count.restype = i64
         L.b200sp_set_option.argtypes = [ctypes.c_char_p, i32]
         L.b200sp_check.argtypes = [p]
@@ -364,6 +366,10 @@ def b200sp_cache_drop(key):
 
 def b200sp_version() -> int:
     return lib().b200sp_version()
+
+
+def b200sp_checked_build() -> int:
+    return lib().b200sp_checked_build()
 
 
 def b200sp_launch_count() -> int:

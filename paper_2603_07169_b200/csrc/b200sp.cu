@@ -48,6 +48,21 @@ static int run_spmv_noalloc(int64_t m, int64_t nnz, const int32_t* row_ptr, cons
   return rc;
 }
 
+// ---- checked build (-DB200SP_BOUNDS_CHECK): every compute call first verifies on the device that row_ptr is monotone
+// with the right ends and that every column index lies in [0, n), synchronises, and refuses an inconsistent matrix with
+// B200SP_ERR_BAD_CSR before any kernel that would index with it is launched.  A stand-in for a memory checker: nothing
+// traps, the first bad matrix is reported by a status code.  The ordinary build compiles this away.
+static int checked_build_validate(const b200sp_plan* p, const int32_t* col_idx, void* stream) {
+#ifdef B200SP_BOUNDS_CHECK
+  const b200sp_plan_info_t& I = p->info;
+  if (I.m == 0) return B200SP_OK;
+  return b200sp_validate_csr(I.m, I.n, I.nnz, p->row_ptr, col_idx, stream);
+#else
+  (void)p; (void)col_idx; (void)stream;
+  return B200SP_OK;
+#endif
+}
+
 // launcher of the gather probe (b200sp_tuning.h)
 template <typename E, bool SMEM>
 static int run_probe_gather(const void* table, int64_t table_elems, int64_t gathers, float* sink, cudaStream_t stream, DeviceInfo* dev) {
@@ -94,6 +109,8 @@ int b200sp_spmv(b200sp_plan* plan, const int32_t* col_idx, const void* vals, con
   DeviceInfo* dev = nullptr;
   rc = device_info(&dev);
   if (rc != B200SP_OK) return rc;
+  rc = checked_build_validate(plan, col_idx, stream);
+  if (rc != B200SP_OK) return rc;
   if (dtype == B200SP_F32) return run_spmv<float>(plan, col_idx, (const float*)vals, (const float*)x, (float*)y, alpha, beta, (cudaStream_t)stream, dev);
   return run_spmv<bf16_t>(plan, col_idx, (const bf16_t*)vals, (const bf16_t*)x, (bf16_t*)y, alpha, beta, (cudaStream_t)stream, dev);
 }
@@ -105,6 +122,8 @@ int b200sp_spmm(b200sp_plan* plan, int64_t k, const int32_t* col_idx, const void
   if (k <= 0 || k >= ((int64_t)1 << 31) || plan->info.m * k >= ((int64_t)1 << 40)) return B200SP_ERR_INVALID_ARG;
   DeviceInfo* dev = nullptr;
   rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  rc = checked_build_validate(plan, col_idx, stream);
   if (rc != B200SP_OK) return rc;
   if (dtype == B200SP_F32) return run_spmm<float, 4>(plan, (int)k, col_idx, (const float*)vals, (const float*)B, (float*)Y, alpha, beta, (cudaStream_t)stream, dev);
   return run_spmm<bf16_t, 8>(plan, (int)k, col_idx, (const bf16_t*)vals, (const bf16_t*)B, (bf16_t*)Y, alpha, beta, (cudaStream_t)stream, dev);
@@ -458,7 +477,7 @@ int b200sp_cache_drop(const void* key_ptr) {
     }
     for (auto it = g_csc_cache.begin(); it != g_csc_cache.end();) {
       if (std::get<0>(it->first) == dev && std::get<1>(it->first) == key_ptr) {
-        for (void* q : {(void*)it->second.row_ptr, (void*)it->second.col, (void*)it->second.perm, it->second.vals_t}) blocks.push_back(q);
+        blocks.push_back(it->second.block);
         it = g_csc_cache.erase(it);
       } else ++it;
     }
@@ -527,6 +546,13 @@ int b200sp_check(void* stream_v) {
 
 const char* b200sp_last_cuda_error(void) { return g_last_error.c_str(); }
 int b200sp_version(void) { return kVersion; }
+int b200sp_checked_build(void) {
+#ifdef B200SP_BOUNDS_CHECK
+  return 1;
+#else
+  return 0;
+#endif
+}
 int64_t b200sp_launch_count(void) { return g_launches.load(); }
 
 int b200sp_set_option(const char* name, int value) {

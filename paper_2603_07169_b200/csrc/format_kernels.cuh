@@ -6,6 +6,7 @@
 // implicit offsets i * width; its kernels skip the padded entries.
 #pragma once
 #include "common.cuh"
+#include "plan_kernels.cuh"
 #include "spmm_kernels.cuh"
 
 namespace b200sp {
@@ -27,6 +28,144 @@ __global__ void __launch_bounds__(256) coo_row_ptr_kernel(const int* __restrict_
     if (p + 1 < nnz && row_idx[p + 1] < r) b = 1;
   }
   if (b) atomicOr(bad, 1);
+}
+
+// ---- CSC front end: the transpose plan, built on the device ----
+// The row-major order of a CSC pattern: entry q of the row-major list is CSC entry perm[q], rows ascending and, inside a row,
+// CSC positions ascending (= columns ascending, duplicates in their stored order), so that a row's sum is added in the same
+// order on every run.  Steps: check the pattern; count the entries of each row (integer atomics: the counts do not depend on
+// scheduling); exclusive scan -> row offsets; place every entry in its row's range at a slot claimed with an integer atomic
+// (the order inside a row is arbitrary at this point); sort each row's range by CSC position (which makes it unique); look up each
+// entry's column in col_ptr.
+
+__global__ void __launch_bounds__(256) csc_check_kernel(const int* __restrict__ col_ptr, const int* __restrict__ row_idx, int m, int n, int nnz,
+                                                        int* __restrict__ bad) {
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  int b = 0;
+  if (i0 == 0 && (col_ptr[0] != 0 || col_ptr[n] != nnz)) b = 1;
+  for (long long j = i0; j < n; j += stride) if (col_ptr[j + 1] < col_ptr[j]) b = 1;
+  for (long long p = i0; p < nnz; p += stride) { const int r = row_idx[p]; if (r < 0 || r >= m) b = 1; }
+  if (b) atomicOr(bad, 1);
+}
+
+__global__ void __launch_bounds__(256) csc_count_rows_kernel(const int* __restrict__ row_idx, long long nnz, int* __restrict__ count) {
+  for (long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x; p < nnz; p += (long long)gridDim.x * blockDim.x)
+    atomicAdd(count + row_idx[p], 1);
+}
+
+// Exclusive scan of an int array in three passes (blocks of kScanBlock entries): block sums; their exclusive scan by one CTA
+// (plan_compact_scan_kernel); every block's own scan plus its offset.  out may alias in.  out[count] is not written.
+constexpr int kScanBlock = 1024;
+
+__global__ void __launch_bounds__(256) scan_block_sums_kernel(const int* __restrict__ in, long long count, int* __restrict__ block_sum) {
+  __shared__ int s_sum;
+  if (threadIdx.x == 0) s_sum = 0;
+  __syncthreads();
+  const long long base = (long long)blockIdx.x * kScanBlock;
+  int c = 0;
+  for (int j = threadIdx.x; j < kScanBlock; j += 256) if (base + j < count) c += in[base + j];
+  atomicAdd(&s_sum, c);
+  __syncthreads();
+  if (threadIdx.x == 0) block_sum[blockIdx.x] = s_sum;
+}
+
+__global__ void __launch_bounds__(256) scan_apply_kernel(const int* in, long long count, const int* __restrict__ block_offset, int* out) {
+  __shared__ int s_warp[8];
+  const long long base = (long long)blockIdx.x * kScanBlock;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int running = block_offset[blockIdx.x];
+  for (int j0 = 0; j0 < kScanBlock; j0 += 256) {
+    const long long i = base + j0 + threadIdx.x;
+    const int v = i < count ? in[i] : 0;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    int before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { const int c = s_warp[w]; if (w < warp) before += c; total += c; }
+    if (i < count) out[i] = running + before + incl - v;
+    running += total;
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(256) csc_place_kernel(const int* __restrict__ row_idx, long long nnz, const int* __restrict__ row_ptr_t,
+                                                        int* __restrict__ fill, int* __restrict__ perm) {
+  for (long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x; p < nnz; p += (long long)gridDim.x * blockDim.x) {
+    const int r = row_idx[p];
+    perm[row_ptr_t[r] + atomicAdd(fill + r, 1)] = (int)p;
+  }
+}
+
+// Sorts every row's range of perm ascending.  A CTA owns 256 consecutive rows: rows of at most 32 entries are sorted by one
+// thread each (insertion sort), longer rows one after another by the whole CTA with a bitonic network, in shared memory when the
+// row fits (4096 entries), else in place in global memory.  Positions are distinct, so the result is unique.
+__global__ void __launch_bounds__(256) csc_sort_rows_kernel(int m, const int* __restrict__ row_ptr_t, int* __restrict__ perm) {
+  constexpr int CAP = 4096;
+  __shared__ int buf[CAP];
+  const long long row0 = (long long)blockIdx.x * 256;
+  {
+    const long long r = row0 + threadIdx.x;
+    if (r < m) {
+      const int s = row_ptr_t[r], e = row_ptr_t[r + 1];
+      if (e - s <= 32) {
+        for (int i = s + 1; i < e; ++i) {
+          const int v = perm[i];
+          int j = i - 1;
+          while (j >= s && perm[j] > v) { perm[j + 1] = perm[j]; --j; }
+          perm[j + 1] = v;
+        }
+      }
+    }
+  }
+  for (int t = 0; t < 256; ++t) {
+    const long long r = row0 + t;
+    if (r >= m) break;
+    const int s = row_ptr_t[r], len = row_ptr_t[r + 1] - s;
+    if (len <= 32) continue;                       // uniform over the CTA: every thread reads the same bounds
+    int pow2 = 64;
+    while (pow2 < len) pow2 <<= 1;
+    const bool in_smem = len <= CAP;
+    __syncthreads();
+    if (in_smem) {
+      for (int i = threadIdx.x; i < len; i += 256) buf[i] = perm[s + i];
+      __syncthreads();
+    }
+    int* const data = in_smem ? buf : perm + s;
+    // bitonic network in the form whose comparisons all ascend (each merge starts with a mirrored step), so entries past len,
+    // which would only ever be the larger partner, need not exist
+    for (int size = 2; size <= pow2; size <<= 1) {
+      const int half = size >> 1;
+      for (int i = threadIdx.x; i < pow2 / 2; i += 256) {
+        const int blk = i / half, off = i - blk * half;
+        const int lo = blk * size + off, hi = blk * size + size - 1 - off;
+        if (hi < len) { const int a = data[lo], b = data[hi]; if (a > b) { data[lo] = b; data[hi] = a; } }
+      }
+      __syncthreads();
+      for (int stride = half >> 1; stride > 0; stride >>= 1) {
+        for (int i = threadIdx.x; i < pow2 / 2; i += 256) {
+          const int lo = 2 * i - (i & (stride - 1)), hi = lo + stride;
+          if (hi < len) { const int a = data[lo], b = data[hi]; if (a > b) { data[lo] = b; data[hi] = a; } }
+        }
+        __syncthreads();
+      }
+    }
+    if (in_smem) for (int i = threadIdx.x; i < len; i += 256) perm[s + i] = buf[i];
+  }
+}
+
+// col_t[q] = the column of CSC entry perm[q]: the last j with col_ptr[j] <= perm[q].
+__global__ void __launch_bounds__(256) csc_cols_kernel(long long nnz, int n, const int* __restrict__ col_ptr, const int* __restrict__ perm,
+                                                       int* __restrict__ col_t) {
+  for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < nnz; q += (long long)gridDim.x * blockDim.x) {
+    const int p = perm[q];
+    int lo = 0, hi = n;                             // first j with col_ptr[j] > p, minus one
+    while (lo < hi) { const int mid = (lo + hi) >> 1; if (col_ptr[mid + 1] <= p) lo = mid + 1; else hi = mid; }
+    col_t[q] = lo;
+  }
 }
 
 // CSC front end, per call: values permuted into the row-major order that the transpose plan computed.

@@ -46,16 +46,20 @@ static int coo_row_ptr(const int32_t** out, int64_t m, int64_t n, int64_t nnz, c
   return B200SP_OK;
 }
 
-// ---- CSC front end: a transpose plan (built on the host, stable in column order), then the CSR path ----
-struct CscEntry { int32_t* row_ptr = nullptr; int32_t* col = nullptr; int32_t* perm = nullptr; void* vals_t = nullptr; };
+// ---- CSC front end: a transpose plan built on the device (see format_kernels.cuh), then the CSR path ----
+// One pool block per pattern: row offsets, columns and CSC positions in row-major order, and room for the permuted values.
+struct CscEntry { void* block = nullptr; int32_t* row_ptr = nullptr; int32_t* col = nullptr; int32_t* perm = nullptr; void* vals_t = nullptr; };
 static std::map<std::tuple<int, const void*, const void*, int64_t, int64_t, int64_t>, CscEntry> g_csc_cache;
 
 static void csc_free(CscEntry& e) {
-  for (void* q : {(void*)e.row_ptr, (void*)e.col, (void*)e.perm, e.vals_t}) if (q) cudaFree(q);
+  if (e.block) cudaFree(e.block);
   e = CscEntry();
 }
 
 static int csc_plan(CscEntry* out, int64_t m, int64_t n, int64_t nnz, const int32_t* col_ptr, const int32_t* row_idx, cudaStream_t stream) {
+  DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
   int d = 0;
   CU(cudaGetDevice(&d));
   const auto key = std::make_tuple(d, (const void*)col_ptr, (const void*)row_idx, m, n, nnz);
@@ -64,45 +68,55 @@ static int csc_plan(CscEntry* out, int64_t m, int64_t n, int64_t nnz, const int3
     auto it = g_csc_cache.find(key);
     if (it != g_csc_cache.end()) { *out = it->second; return B200SP_OK; }
   }
-  // pattern to the host, stable counting sort by row (entries of a row end up in ascending column order), back to the device
-  std::vector<int32_t> h_cp((size_t)n + 1), h_ri((size_t)nnz), h_rp((size_t)m + 1, 0), h_col((size_t)nnz), h_perm((size_t)nnz);
-  CU(cudaMemcpyAsync(h_cp.data(), col_ptr, ((size_t)n + 1) * 4, cudaMemcpyDeviceToHost, stream));
-  if (nnz > 0) CU(cudaMemcpyAsync(h_ri.data(), row_idx, (size_t)nnz * 4, cudaMemcpyDeviceToHost, stream));
-  CU(cudaStreamSynchronize(stream));
-  if (h_cp[0] != 0 || h_cp[(size_t)n] != nnz) return B200SP_ERR_BAD_CSR;
-  for (int64_t p = 0; p < nnz; ++p) {
-    if (h_ri[(size_t)p] < 0 || h_ri[(size_t)p] >= m) return B200SP_ERR_BAD_CSR;
-    h_rp[(size_t)h_ri[(size_t)p] + 1]++;
-  }
-  for (int64_t i = 0; i < m; ++i) h_rp[(size_t)i + 1] += h_rp[(size_t)i];
-  {
-    std::vector<int32_t> next(h_rp.begin(), h_rp.end() - 1);
-    for (int64_t j = 0; j < n; ++j) {
-      if (h_cp[(size_t)j + 1] < h_cp[(size_t)j]) return B200SP_ERR_BAD_CSR;
-      for (int32_t p = h_cp[(size_t)j]; p < h_cp[(size_t)j + 1]; ++p) {
-        const int32_t q = next[(size_t)h_ri[(size_t)p]]++;
-        h_col[(size_t)q] = (int32_t)j;
-        h_perm[(size_t)q] = p;
-      }
-    }
-  }
-  CscEntry e;
-  auto fail = [&](cudaError_t err, const char* what) { csc_free(e); return cuda_fail(err, what); };
-  cudaError_t err;
-  if ((err = cudaMalloc(&e.row_ptr, ((size_t)m + 1) * 4)) != cudaSuccess) return fail(err, "cudaMalloc");
+  auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
   const size_t nz = nnz > 0 ? (size_t)nnz : 1;
-  if ((err = cudaMalloc(&e.col, nz * 4)) != cudaSuccess) return fail(err, "cudaMalloc");
-  if ((err = cudaMalloc(&e.perm, nz * 4)) != cudaSuccess) return fail(err, "cudaMalloc");
-  if ((err = cudaMalloc(&e.vals_t, nz * 4)) != cudaSuccess) return fail(err, "cudaMalloc");
-  if ((err = cudaMemcpyAsync(e.row_ptr, h_rp.data(), ((size_t)m + 1) * 4, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return fail(err, "cudaMemcpyAsync");
+  const size_t blocks = (size_t)((m + 1 + kScanBlock - 1) / kScanBlock);
+  const size_t o_rp = 0, o_col = o_rp + up(((size_t)m + 2) * 4), o_perm = o_col + up(nz * 4), o_vals = o_perm + up(nz * 4),
+               o_fill = o_vals + up(nz * 4), o_bs = o_fill + up(((size_t)m + 2) * 4), o_bad = o_bs + up((blocks + 1) * 4), total = o_bad + 256;
+  CscEntry e;
+  rc = pool_alloc(dev, &e.block, total, stream);
+  if (rc != B200SP_OK) return rc;
+  char* base = (char*)e.block;
+  e.row_ptr = (int32_t*)(base + o_rp);
+  e.col = (int32_t*)(base + o_col);
+  e.perm = (int32_t*)(base + o_perm);
+  e.vals_t = base + o_vals;
+  int* fill = (int*)(base + o_fill);
+  int* bsum = (int*)(base + o_bs);
+  int* d_bad = (int*)(base + o_bad);
+  int h_bad = 0;
+  auto fail = [&](int code) { cudaFreeAsync(e.block, stream); cudaStreamSynchronize(stream); return code; };
+#define CUF(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail(cuda_fail(e_, #call)); } while (0)
+  const unsigned wide = (unsigned)(dev->sms * 16);
+  auto grid_for = [&](int64_t work) { long long b = (work + 255) / 256; if (b < 1) b = 1; return (unsigned)(b > (long long)wide ? wide : b); };
+  CUF(cudaMemsetAsync(d_bad, 0, sizeof(int), stream));
+  CUF(cudaMemsetAsync(fill, 0, ((size_t)m + 2) * 4, stream));
+  csc_check_kernel<<<grid_for(nnz > n ? nnz : n), 256, 0, stream>>>(col_ptr, row_idx, (int)m, (int)n, (int)nnz, d_bad);
+  g_launches++;
+  CUF(cudaGetLastError());
+  CUF(cudaMemcpyAsync(&h_bad, d_bad, sizeof(int), cudaMemcpyDeviceToHost, stream));
+  CUF(cudaStreamSynchronize(stream));                          // nothing below may index with an unchecked row number
+  if (h_bad) return fail(B200SP_ERR_BAD_CSR);
+  if (nnz > 0) csc_count_rows_kernel<<<grid_for(nnz), 256, 0, stream>>>(row_idx, (long long)nnz, fill);
+  // exclusive scan of the m + 1 counts (the last one is zero) -> row offsets, row_ptr[m] = nnz
+  scan_block_sums_kernel<<<(unsigned)blocks, 256, 0, stream>>>(fill, (long long)m + 1, bsum);
+  plan_compact_scan_kernel<<<1, 1024, 0, stream>>>(bsum, (int)blocks);
+  scan_apply_kernel<<<(unsigned)blocks, 256, 0, stream>>>(fill, (long long)m + 1, bsum, e.row_ptr);
+  g_launches += 4;
+  CUF(cudaGetLastError());
+  CUF(cudaMemsetAsync(fill, 0, ((size_t)m + 2) * 4, stream));
   if (nnz > 0) {
-    if ((err = cudaMemcpyAsync(e.col, h_col.data(), (size_t)nnz * 4, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return fail(err, "cudaMemcpyAsync");
-    if ((err = cudaMemcpyAsync(e.perm, h_perm.data(), (size_t)nnz * 4, cudaMemcpyHostToDevice, stream)) != cudaSuccess) return fail(err, "cudaMemcpyAsync");
+    csc_place_kernel<<<grid_for(nnz), 256, 0, stream>>>(row_idx, (long long)nnz, e.row_ptr, fill, e.perm);
+    csc_sort_rows_kernel<<<(unsigned)((m + 255) / 256), 256, 0, stream>>>((int)m, e.row_ptr, e.perm);
+    csc_cols_kernel<<<grid_for(nnz), 256, 0, stream>>>((long long)nnz, (int)n, col_ptr, e.perm, e.col);
+    g_launches += 3;
+    CUF(cudaGetLastError());
   }
-  if ((err = cudaStreamSynchronize(stream)) != cudaSuccess) return fail(err, "cudaStreamSynchronize");
+  CUF(cudaStreamSynchronize(stream));
+#undef CUF
   std::lock_guard<std::mutex> lock(g_mutex);
   auto ins = g_csc_cache.emplace(key, e);
-  if (!ins.second) { csc_free(e); e = ins.first->second; }
+  if (!ins.second) { cudaFreeAsync(e.block, stream); e = ins.first->second; }
   *out = e;
   return B200SP_OK;
 }

@@ -19,7 +19,7 @@ using namespace b200sp;
 
 namespace {
 
-constexpr int kVersion = 100;  // 0.1.0
+constexpr int kVersion = 200;  // 0.2.0
 
 // SpMV merge-tile configuration
 constexpr int kItems = 4096;

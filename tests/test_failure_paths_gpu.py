@@ -237,3 +237,61 @@ print("ok")
 ''' % root
     out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=600)
     assert out.returncode == 0 and "ok" in out.stdout, out.stdout + out.stderr
+
+
+def test_checked_build_refuses_an_inconsistent_matrix_before_touching_it():
+    """libb200sp_check.so (built with -DB200SP_BOUNDS_CHECK) validates row_ptr and col_idx on the device before every compute
+    call: a column index equal to n, or a decreasing row_ptr, comes back as B200SP_ERR_BAD_CSR with y untouched, and a
+    consistent matrix gives the same result as the ordinary build.  It stands in for a memory checker: nothing traps.
+    Run in a process of its own because the library file is chosen when the binding is imported."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    lib = os.path.join(root, "paper_2603_07169_b200", "libb200sp_check.so")
+    if not os.path.exists(lib):
+        from paper_2603_07169_b200 import build
+        build.build(checked=True)
+    code = r'''
+import numpy as np, torch, sys
+sys.path.insert(0, %r)
+import gen, oracle, paper_2603_07169_b200 as b
+assert b.b200sp_checked_build() == 1
+dev = "cuda:0"
+A = gen.random_csr(3000, 700, np.random.default_rng(1).integers(0, 30, 3000), 5)
+x = np.random.default_rng(2).standard_normal(700).astype(np.float32)
+up = lambda a: torch.from_numpy(a).to(dev)
+d_rp, d_ci, d_va, d_x = up(A.row_ptr), up(A.col_idx), up(A.vals), up(x)
+y = torch.full((A.m,), 7.0, device=dev)
+b.spmv_csr(A.m, A.n, A.nnz, d_rp, d_ci, d_va, d_x, y, 1.0, 0.0, "f32")
+torch.cuda.synchronize()
+y_ref, S = oracle.spmv_csr(A.m, A.n, A.row_ptr, A.col_idx, A.vals, x, None, 1.0, 0.0, "f32")
+assert oracle.tolerance_ratio(y.cpu().numpy(), y_ref, S, "f32")[0] <= 1.0
+b.b200sp_cache_clear()
+for what in ("col", "row"):
+    ci, rp = A.col_idx.copy(), A.row_ptr.copy()
+    if what == "col": ci[1234] = A.n
+    else: rp[100] = rp[101] + 3
+    y = torch.full((A.m,), 7.0, device=dev)
+    n0 = b.b200sp_launch_count()
+    try:
+        b.spmv_csr(A.m, A.n, A.nnz, up(rp), up(ci), d_va, d_x, y, 1.0, 0.0, "f32")
+        raise SystemExit("accepted a bad " + what)
+    except b.B200spError as e:
+        assert e.status == 6, e.status
+    torch.cuda.synchronize()
+    assert torch.all(y == 7.0)                     # no compute kernel ran
+    b.b200sp_cache_clear()
+Y = torch.full((A.m * 8,), 7.0, device=dev)
+ci = A.col_idx.copy(); ci[5] = -1
+try:
+    b.spmm_csr(A.m, A.n, A.nnz, 8, d_rp, up(ci), d_va, up(np.ones(700 * 8, np.float32)), Y, 1.0, 0.0, "f32")
+    raise SystemExit("accepted a negative column")
+except b.B200spError as e:
+    assert e.status == 6
+assert torch.all(Y == 7.0)
+print("ok")
+''' % root
+    env = dict(os.environ, B200SP_LIBRARY="libb200sp_check.so")
+    out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=600, env=env)
+    assert out.returncode == 0 and "ok" in out.stdout, out.stdout + out.stderr

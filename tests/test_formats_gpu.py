@@ -20,6 +20,8 @@ def matrices():
         "stencil": gen.stencil27(12, 5),
         "short_ragged": gen.random_csr(4001, 333, rng.integers(0, 10, 4001), 2),
         "one_column": gen.random_csr(500, 1, rng.integers(0, 2, 500), 4, allow_dup=True),
+        # rows of every size class of the CSC transpose plan: <= 32 (a thread sorts), 33-4096 (a CTA in shared memory), more (a CTA in global memory)
+        "long_rows": gen.random_csr(700, 12000, np.concatenate([rng.integers(0, 40, 690), [33, 4096, 4097, 9000, 5000, 0, 64, 1, 100, 11000]]), 6),
     }
 
 
@@ -51,7 +53,7 @@ def test_coo_spmv_and_spmm(name, dtype):
 
 
 @pytest.mark.parametrize("dtype", DTYPES)
-@pytest.mark.parametrize("name", ["power_law", "uniform16", "stencil", "short_ragged"])
+@pytest.mark.parametrize("name", ["power_law", "uniform16", "stencil", "short_ragged", "long_rows", "one_column"])
 def test_csc_spmv_and_spmm(name, dtype):
     A = matrices()[name]
     rng = np.random.default_rng(3)
@@ -75,6 +77,31 @@ def test_csc_spmv_and_spmm(name, dtype):
     torch.cuda.synchronize()
     Y_ref, S = oracle.spmm_csc(A.m, A.n, k, cp, ri, v_s, B_s, None, 1.0, 0.0, dtype)
     assert_within(to_host(Y, dtype).reshape(A.m, k), Y_ref, S, dtype, what="csc spmm " + name)
+    b200sp.b200sp_cache_clear()
+
+
+def test_csc_transpose_plan_is_built_on_the_device_and_reproducible():
+    """The same CSC pattern planned twice (the cache dropped in between) gives bit-identical results: the order of a row's
+    entries is fixed by their CSC positions, not by the order in which the placement kernel's atomics happened to run."""
+    A = matrices()["long_rows"]
+    cp, ri, va = gen.csr_to_csc(A)
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal(A.n).astype(np.float32)
+    d_cp, d_ri, d_v, d_x = to_dev(cp), to_dev(ri), to_dev(va), to_dev(x)
+    outs = []
+    for _ in range(3):
+        y = empty_out(A.m, "f32")
+        b200sp.spmv_csc(A.m, A.n, A.nnz, d_cp, d_ri, d_v, d_x, y, 1.0, 0.0, "f32")
+        torch.cuda.synchronize()
+        outs.append(y.cpu().numpy().copy())
+        b200sp.b200sp_cache_drop(d_cp)
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+    # and equal, bit for bit, to the CSR path on the same matrix with columns in ascending order (the order the plan produces)
+    order = np.lexsort((A.col_idx, np.repeat(np.arange(A.m), np.diff(A.row_ptr))))
+    y = empty_out(A.m, "f32")
+    b200sp.spmv_csr(A.m, A.n, A.nnz, to_dev(A.row_ptr), to_dev(A.col_idx[order]), to_dev(A.vals[order]), d_x, y, 1.0, 0.0, "f32")
+    torch.cuda.synchronize()
+    assert np.array_equal(outs[0], y.cpu().numpy())
     b200sp.b200sp_cache_clear()
 
 
