@@ -421,8 +421,8 @@ def request_bound(rec, w, dtype, gather_rate):
     """A bound from MEASURED L1-to-L2 traffic instead of one miss per nonzero: the ncu capture of this workload counts the
     sectors the L1s asked L2 for; the CSR stream's share of them arrives four sectors to a request (128-bit coalesced loads of
     whole lines), every other sector is a request of its own, and the SMs issue requests at the probe's rate."""
-    if not rec or "l2_sectors_read_by_l1" not in rec:
-        return {}
+    if not rec or "l2_sectors_read_by_l1" not in rec or rec.get("l1_hit_pct", 0.0) > 50.0:
+        return {}       # no capture, or a kernel whose gathers mostly hit L1 (and whose CSR stream arrives by bulk copies): not request-bound
     A = w.A
     e = 4 if dtype == "f32" else 2
     stream_sectors = (A.nnz * (4 + e) + (A.m + 1) * 4) / 32.0

@@ -136,13 +136,25 @@ def _dev(t, elems: int, esize: int, what: str) -> Optional[int]:
     against the sizes)."""
     if t is None:
         return None
-    import torch
-    ok = isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous() and t.device.index == torch.cuda.current_device() \
-        and t.element_size() == esize and (elems < 0 or t.numel() >= elems)
+    try:        # attribute checks only (this sits on the launch path of microsecond kernels); anything without them is not a tensor
+        ok = t.is_cuda and t.element_size() == esize and t.numel() >= elems and t.is_contiguous() and t.device.index == _current_device()
+    except AttributeError:
+        ok = False
     if not ok:
         raise B200spError(1, "%s: expected a contiguous CUDA tensor on the current device with >= %d elements of %d bytes, got %s"
                           % (what, elems, esize, _describe(t)))
     return t.data_ptr()
+
+
+_torch = None
+
+
+def _current_device() -> int:
+    global _torch
+    if _torch is None:
+        import torch
+        _torch = torch
+    return _torch.cuda.current_device()
 
 
 def _host(t, elems: int, esize: int, what: str) -> Optional[int]:
