@@ -128,7 +128,7 @@ def _esize(dtype) -> int:
     return 4 if _dt(dtype) == F32 else 2
 
 
-def _dev(t, elems: int, esize: int, what: str) -> Optional[int]:
+def _dev(t, elems: int, esize: int, what: str, cur: Optional[int] = None) -> Optional[int]:
     """Address of a DEVICE operand.  The kernels dereference it on the GPU, and the library cannot tell a host address from
     a device address or see how long an array is, so this is the only place where a wrong tensor can be stopped: it must be
     a contiguous CUDA tensor on the current device with elements of `esize` bytes and at least `elems` of them.  Anything
@@ -136,8 +136,9 @@ def _dev(t, elems: int, esize: int, what: str) -> Optional[int]:
     against the sizes)."""
     if t is None:
         return None
-    try:        # attribute checks only (this sits on the launch path of microsecond kernels); anything without them is not a tensor
-        ok = t.is_cuda and t.element_size() == esize and t.numel() >= elems and t.is_contiguous() and t.device.index == _current_device()
+    try:        # a few method calls only (this sits on the launch path of microsecond kernels); get_device() is -1 for a CPU tensor,
+        #             and anything without these methods (a numpy array) is not a tensor
+        ok = t.get_device() == (_current_device() if cur is None else cur) and t.element_size() == esize and t.numel() >= elems and t.is_contiguous()
     except AttributeError:
         ok = False
     if not ok:
@@ -150,11 +151,15 @@ _torch = None
 
 
 def _current_device() -> int:
+    """Index of the current CUDA device; -2 (which no tensor's device matches) on a machine without one."""
     global _torch
     if _torch is None:
         import torch
         _torch = torch
-    return _torch.cuda.current_device()
+    try:
+        return _torch.cuda.current_device()
+    except (RuntimeError, AssertionError):
+        return -2
 
 
 def _host(t, elems: int, esize: int, what: str) -> Optional[int]:
@@ -203,6 +208,10 @@ def _ck(status: int, where: str):
 def _csr_args(m, n, nnz, k, row_ptr, col_idx, vals, dense_in, dense_out, dtype, what, conv=_dev):
     e = _esize(dtype)
     kk = max(k, 1)
+    if conv is _dev:
+        cur = _current_device()          # once per call, not once per operand
+        return (_dev(row_ptr, m + 1 if m > 0 else 0, 4, what, cur), _dev(col_idx, nnz, 4, what, cur), _dev(vals, nnz, e, what, cur),
+                _dev(dense_in, n * kk if nnz > 0 else 0, e, what, cur), _dev(dense_out, m * kk, e, what, cur))
     return (conv(row_ptr, m + 1 if m > 0 else 0, 4, what + " row_ptr"), conv(col_idx, nnz, 4, what + " col_idx"), conv(vals, nnz, e, what + " vals"),
             conv(dense_in, n * kk if nnz > 0 else 0, e, what + " x/B"), conv(dense_out, m * kk, e, what + " y/Y"))
 
