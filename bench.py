@@ -409,10 +409,12 @@ def run_probes(dev, l2_bytes):
     reads = 1 << 25
     for lines, label in ((1 << 19, "64 MB of lines (one k-slice of B of the SpMM workload)"), (1 << 17, "16 MB of lines (L2-resident)")):
         buf = torch.zeros(lines * 32, dtype=torch.int32, device=dev)
-        for inflight, to_smem in ((4, 0), (8, 0), (16, 0), (4, 1), (8, 1), (16, 1)):
-            t = timed(lambda: b200sp.b200sp_probe_lines(buf, lines, reads, sink, inflight, to_smem, stream))
-            row("random 128-byte line reads by groups of 8 lanes, %d in flight per group %s, %s" % (inflight, "to shared memory (cp.async)" if to_smem else "to registers", label),
-                reads * 128 / t * 1e-12, "TB/s", "%.1f bytes per clock per SM" % (reads * 128 / t / sms / clock_hz))
+        for inflight, to_smem, gl in ((4, 0, 8), (8, 0, 8), (16, 0, 8), (4, 1, 8), (8, 1, 8), (16, 1, 8), (4, 0, 16), (4, 0, 32), (8, 0, 32)):
+            nreads = reads * 8 // gl                       # the same number of bytes for every group width
+            t = timed(lambda: b200sp.b200sp_probe_lines(buf, lines, nreads, sink, inflight, to_smem, stream, gl))
+            row("random %d-byte reads (%d consecutive line%s) by groups of %d lanes, %d in flight per group %s, %s"
+                % (gl * 16, gl // 8, "s" if gl > 8 else "", gl, inflight, "to shared memory (cp.async)" if to_smem else "to registers", label),
+                nreads * gl * 16 / t * 1e-12, "TB/s", "%.1f bytes per clock per SM" % (nreads * gl * 16 / t / sms / clock_hz))
         del buf
     return out
 

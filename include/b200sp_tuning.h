@@ -82,15 +82,17 @@ int b200sp_set_option(const char* name, int value);
  *   the table (at most 224 KB) first copied into each CTA's shared memory and gathered from there.
  * b200sp_probe_stream: reads `bytes` (a multiple of 16; buf 16-byte aligned) once with coalesced 128-bit loads: what
  *   a pure stream of the CSR arrays reaches at that size.
- * b200sp_probe_lines: `reads` random 128-byte lines out of `lines` (a power of two), each by a group of eight lanes
- *   with 16 bytes per lane and in_flight = 4, 8 or 16 lines in flight per group, into registers or, with
- *   to_shared_memory = 1, into shared memory with cp.async: the L2-to-SM rate of SpMM's reads of B (the k-sliced kernel
- *   keeps four lines per group in registers). */
+ * b200sp_probe_lines: `reads` random chunks of one, two or four consecutive 128-byte lines out of a buffer of `lines`
+ *   lines (a power of two), each chunk by a group of group_lanes = 8, 16 or 32 lanes with 16 bytes per lane and
+ *   in_flight = 4, 8 or 16 chunks in flight per group, into registers or, with to_shared_memory = 1 (group_lanes = 8
+ *   only), into shared memory with cp.async: the L2-to-SM rate of SpMM's reads of B (the k-sliced kernel keeps four
+ *   lines per group of eight lanes in registers). */
 int b200sp_probe_gather(const float* table, int64_t table_elems, int64_t gathers, float* sink, void* stream);
 int b200sp_probe_gather_ex(const void* table, int64_t table_elems, int64_t gathers, int elem_bytes, int in_shared_memory, float* sink,
                            void* stream);
 int b200sp_probe_stream(const void* buf, int64_t bytes, float* sink, void* stream);
-int b200sp_probe_lines(const void* buf, int64_t lines, int64_t reads, int in_flight, int to_shared_memory, float* sink, void* stream);
+int b200sp_probe_lines(const void* buf, int64_t lines, int64_t reads, int in_flight, int to_shared_memory, int group_lanes, float* sink,
+                       void* stream);
 
 #ifdef __cplusplus
 }

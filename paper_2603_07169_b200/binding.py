@@ -86,7 +86,7 @@ def lib() -> ctypes.CDLL:
         L.b200sp_probe_gather_ex.restype = i32
         L.b200sp_probe_stream.argtypes = [p, i64, p, p]
         L.b200sp_probe_stream.restype = i32
-        L.b200sp_probe_lines.argtypes = [p, i64, i64, i32, i32, p, p]
+        L.b200sp_probe_lines.argtypes = [p, i64, i64, i32, i32, i32, p, p]
         L.b200sp_probe_lines.restype = i32
         L.spmm_csr_host.argtypes = L.spmm_csr.argtypes
         L.b200sp_plan_create.argtypes = [ctypes.POINTER(p), i64, i64, i64, p, p]
@@ -303,9 +303,9 @@ def b200sp_probe_stream(buf, nbytes, sink, stream=None):
                                   _dev(sink, 1, 4, "probe sink"), _stream(stream)), "b200sp_probe_stream")
 
 
-def b200sp_probe_lines(buf, lines, reads, sink, in_flight=4, to_shared_memory=0, stream=None):
+def b200sp_probe_lines(buf, lines, reads, sink, in_flight=4, to_shared_memory=0, stream=None, group_lanes=8):
     _ck(lib().b200sp_probe_lines(_dev(buf, lines * 128 // max(buf.element_size(), 1), buf.element_size(), "probe buffer"), lines, reads,
-                                 in_flight, to_shared_memory, _dev(sink, 1, 4, "probe sink"), _stream(stream)), "b200sp_probe_lines")
+                                 in_flight, to_shared_memory, group_lanes, _dev(sink, 1, 4, "probe sink"), _stream(stream)), "b200sp_probe_lines")
 
 
 def b200sp_noalloc_max_items() -> int:

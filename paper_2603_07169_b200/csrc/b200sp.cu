@@ -251,27 +251,31 @@ int b200sp_probe_stream(const void* buf, int64_t bytes, float* sink, void* strea
                 (long long)(bytes / 16), sink);
 }
 
-int b200sp_probe_lines(const void* buf, int64_t lines, int64_t reads, int in_flight, int to_shared_memory, float* sink, void* stream) {
+int b200sp_probe_lines(const void* buf, int64_t lines, int64_t reads, int in_flight, int to_shared_memory, int group_lanes, float* sink,
+                       void* stream) {
   if (!buf || !sink || lines <= 0 || (lines & (lines - 1)) != 0 || lines > ((int64_t)1 << 31) || reads < 0 || !aligned16(buf) ||
-      (in_flight != 4 && in_flight != 8 && in_flight != 16))
+      (in_flight != 4 && in_flight != 8 && in_flight != 16) || (group_lanes != 8 && group_lanes != 16 && group_lanes != 32) ||
+      lines < group_lanes / 8 || (to_shared_memory && group_lanes != 8))
     return B200SP_ERR_INVALID_ARG;
   DeviceInfo* dev = nullptr;
   int rc = device_info(&dev);
   if (rc != B200SP_OK) return rc;
   cudaStream_t st = (cudaStream_t)stream;
   const dim3 grid((unsigned)(dev->sms * 8)), block(256);
-  const unsigned mask = (unsigned)(lines - 1);
+  const unsigned mask = (unsigned)(lines / (group_lanes / 8) - 1);      // chunks of group_lanes / 8 lines
   const size_t smem = to_shared_memory ? (size_t)256 * in_flight * 16 : 0;
-#define B200SP_PROBE_LINES(U, A) return launch_smem(probe_lines_kernel<U, A>, grid, block, smem, st, nullptr, 0, dev, (const int4*)buf, mask, (long long)reads, sink)
+#define B200SP_PROBE_LINES(U, A, GL) return launch_smem(probe_lines_kernel<U, A, GL>, grid, block, smem, st, nullptr, 0, dev, (const int4*)buf, mask, (long long)reads, sink)
   if (to_shared_memory) {
-    if (in_flight == 4) B200SP_PROBE_LINES(4, true);
-    if (in_flight == 8) B200SP_PROBE_LINES(8, true);
-    CU(cudaFuncSetAttribute(probe_lines_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    B200SP_PROBE_LINES(16, true);
+    if (in_flight == 4) B200SP_PROBE_LINES(4, true, 8);
+    if (in_flight == 8) B200SP_PROBE_LINES(8, true, 8);
+    CU(cudaFuncSetAttribute(probe_lines_kernel<16, true, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    B200SP_PROBE_LINES(16, true, 8);
   }
-  if (in_flight == 4) B200SP_PROBE_LINES(4, false);
-  if (in_flight == 8) B200SP_PROBE_LINES(8, false);
-  B200SP_PROBE_LINES(16, false);
+  if (group_lanes == 16) { if (in_flight == 4) B200SP_PROBE_LINES(4, false, 16); if (in_flight == 8) B200SP_PROBE_LINES(8, false, 16); B200SP_PROBE_LINES(16, false, 16); }
+  if (group_lanes == 32) { if (in_flight == 4) B200SP_PROBE_LINES(4, false, 32); if (in_flight == 8) B200SP_PROBE_LINES(8, false, 32); B200SP_PROBE_LINES(16, false, 32); }
+  if (in_flight == 4) B200SP_PROBE_LINES(4, false, 8);
+  if (in_flight == 8) B200SP_PROBE_LINES(8, false, 8);
+  B200SP_PROBE_LINES(16, false, 8);
 #undef B200SP_PROBE_LINES
 }
 

@@ -4,7 +4,8 @@
 //   probe_gather_kernel   random reads of a table: the rate at which an SM takes L1 misses (table >> L1), L1 hits (table fits L1)
 //                         or shared-memory reads (table staged in shared memory) -- the bound on gathering x
 //   probe_stream_kernel   coalesced 128-bit reads of a buffer: what a pure stream of the CSR arrays can reach at a given size
-//   probe_lines_kernel    random reads of whole 128-byte lines by groups of eight lanes: the L2-to-SM path that SpMM's reads of B use
+//   probe_lines_kernel    random reads of whole 128-byte lines (or two / four consecutive ones) by groups of 8 (16 / 32) lanes: the L2-to-SM path
+//                         that SpMM's reads of B use
 #pragma once
 #include "common.cuh"
 
@@ -60,26 +61,27 @@ __global__ void __launch_bounds__(256) probe_stream_kernel(const int4* __restric
   if (acc == 0x5A5A1234) *sink = (float)acc;
 }
 
-// `reads` random 128-byte lines of a buffer of `lines` lines (a power of two): every group of eight lanes reads one line, 16 bytes
-// per lane, U lines in flight per group -- the access pattern of the k-sliced SpMM kernel's reads of B (which keeps U = 4 in
-// registers).  ASYNC: the lines go to shared memory with cp.async (16 bytes per lane) instead of registers, so the bytes in
-// flight are bounded by shared memory rather than by the register file.
-template <int U, bool ASYNC>
-__global__ void __launch_bounds__(256) probe_lines_kernel(const int4* __restrict__ buf, unsigned line_mask, long long reads,
+// `reads` random chunks of GL * 16 bytes (GL = 8, 16 or 32 lanes: one, two or four consecutive 128-byte lines) out of a buffer of
+// `chunks` such chunks (a power of two): every group of GL lanes reads one chunk, 16 bytes per lane, U chunks in flight per group
+// -- the access pattern of the k-sliced SpMM kernel's reads of B (GL = 8, U = 4 in registers).  ASYNC: the chunks go to shared
+// memory with cp.async (16 bytes per lane) instead of registers, so the bytes in flight are bounded by shared memory rather than
+// by the register file.
+template <int U, bool ASYNC, int GL>
+__global__ void __launch_bounds__(256) probe_lines_kernel(const int4* __restrict__ buf, unsigned chunk_mask, long long reads,
                                                           float* __restrict__ sink) {
   extern __shared__ __align__(16) unsigned char probe_smem[];
-  const long long groups = ((long long)gridDim.x * blockDim.x) >> 3;
-  const long long g = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
-  const int l8 = threadIdx.x & 7;
+  const long long groups = ((long long)gridDim.x * blockDim.x) / GL;
+  const long long g = ((long long)blockIdx.x * blockDim.x + threadIdx.x) / GL;
+  const int l = threadIdx.x % GL;
   int acc = 0;
   int4* mine = reinterpret_cast<int4*>(probe_smem) + (size_t)threadIdx.x * U;
   for (long long i = g; i < reads; i += groups * U) {
     if (ASYNC) {
 #pragma unroll
       for (int u = 0; u < U; ++u) {
-        const unsigned line = probe_hash((unsigned long long)(i + u * groups)) & line_mask;
+        const unsigned chunk = probe_hash((unsigned long long)(i + u * groups)) & chunk_mask;
         const unsigned dst = (unsigned)__cvta_generic_to_shared(mine + u);
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(buf + (size_t)line * 8 + l8) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(buf + (size_t)chunk * GL + l) : "memory");
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
       asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -89,8 +91,8 @@ __global__ void __launch_bounds__(256) probe_lines_kernel(const int4* __restrict
       int4 v[U];
 #pragma unroll
       for (int u = 0; u < U; ++u) {
-        const unsigned line = probe_hash((unsigned long long)(i + u * groups)) & line_mask;
-        v[u] = (i + u * groups < reads) ? __ldg(buf + (size_t)line * 8 + l8) : make_int4(0, 0, 0, 0);
+        const unsigned chunk = probe_hash((unsigned long long)(i + u * groups)) & chunk_mask;
+        v[u] = (i + u * groups < reads) ? __ldg(buf + (size_t)chunk * GL + l) : make_int4(0, 0, 0, 0);
       }
 #pragma unroll
       for (int u = 0; u < U; ++u) acc ^= v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
