@@ -834,6 +834,8 @@ def main():
                     "algorithmic_bytes": r["algorithmic_bytes"], "nnz": r["nnz"], "copies": r["copies"],
                     "plan_ms_first_call": round(r["plan_ms_first_call"], 3),
                     "cusparse_ms": round(r["cusparse_ms"], 5) if isinstance(r["cusparse_ms"], float) else r["cusparse_ms"]}
+                ck = sampler.summary(r["t0"], r["t1"])      # SM clock and throttle reasons while THIS workload was timed (long SpMM kernels reach the power cap)
+                extras["%s_%s" % (name, dt)]["clocks"] = {"sm_mhz": ck.get("sm_mhz"), "reasons": ck.get("reasons"), "samples": ck.get("samples")}
                 if name == "c1":   # launch-latency regime: per-call device time from a CUDA graph, and the floors on the same box
                     extras["c1_f32"].update(latency_floor(r["_call"], r["_sets"], dev, r["algorithmic_bytes"]))
                 if not ww.k:   # SpMV: time at the measured L1-miss gather rate for this x
