@@ -392,3 +392,46 @@ def test_dependent_calls_back_to_back(name, scale, dtype):
     assert_within(y1, y_ref, S, dtype, what="first link %s %s" % (name, dtype))
     for links in (2, 7):
         assert np.array_equal(chain(1, links), chain(0, links)), "chain of %d differs between launch modes" % links
+
+
+def test_sizes_next_to_the_int32_limit():
+    """nnz = 2^31 - 16, the largest the 32-bit CSR arrays allow with 16 nonzeros per row (m = 2^27 - 1): every product of an
+    index and a size inside the kernels must be taken in 64 bits or stay below 2^31.  The matrix is made on the device (17 GB of
+    col_idx and vals), the uniform-row, merge-tile and row-direct kernels each run it, and 4096 sampled rows plus the first and
+    the last rows are compared with the oracle, which gets those rows as a small CSR matrix of their own."""
+    dev = "cuda:0"
+    if torch.cuda.mem_get_info()[0] < (40 << 30):
+        pytest.skip("needs 40 GB of free device memory")
+    m, n, per_row = (1 << 27) - 1, 1 << 20, 16
+    nnz = m * per_row
+    assert nnz == (1 << 31) - 16
+    g = torch.Generator(device=dev); g.manual_seed(7)
+    col = torch.randint(0, n, (nnz,), dtype=torch.int32, device=dev, generator=g)
+    val = torch.empty(nnz, dtype=torch.float32, device=dev).normal_(generator=g)
+    row_ptr = (torch.arange(m + 1, dtype=torch.int64, device=dev) * per_row).to(torch.int32)
+    assert int(row_ptr[-1]) == nnz
+    x_h = np.random.default_rng(3).standard_normal(n).astype(np.float32)
+    x = torch.from_numpy(x_h).to(dev)
+    rows = np.unique(np.concatenate([np.arange(0, 64), np.arange(m - 64, m), np.random.default_rng(4).integers(0, m, 4096)])).astype(np.int64)
+    idx = (torch.from_numpy(rows).to(dev)[:, None] * per_row + torch.arange(per_row, device=dev)[None, :]).reshape(-1)
+    sub_col = col[idx].cpu().numpy()
+    sub_val = val[idx].cpu().numpy()
+    sub_rp = (np.arange(len(rows) + 1) * per_row).astype(np.int32)
+    y_ref, S = oracle.spmv_csr(len(rows), n, sub_rp, sub_col, sub_val, x_h, None, 1.0, 0.0, "f32")
+    d_rows = torch.from_numpy(rows).to(dev)
+    try:
+        for kernel in (2, 0, 1):
+            b200sp.b200sp_set_option("spmv_kernel", kernel)
+            y = torch.full((m,), float("nan"), dtype=torch.float32, device=dev)
+            b200sp.spmv_csr(m, n, nnz, row_ptr, col, val, x, y, 1.0, 0.0, "f32")
+            torch.cuda.synchronize()
+            assert not bool(torch.isnan(y).any()), "kernel %d left rows unwritten" % kernel
+            assert_within(y[d_rows].cpu().numpy(), y_ref, S, "f32", what="nnz = 2^31 - 16, kernel %d" % kernel)
+            b200sp.b200sp_cache_clear()
+            del y
+        b200sp.b200sp_check()
+    finally:
+        b200sp.b200sp_set_option("spmv_kernel", -1)
+        b200sp.b200sp_cache_clear()
+        del col, val, row_ptr
+        torch.cuda.empty_cache()
