@@ -60,6 +60,9 @@ extern "C" {
  *  memory
  *   "pool_keep_mb"   MiB of freed memory the library's pool keeps across synchronisation points, default 1024
  *                    (read when a device's pool is created, i.e. before the first call that allocates on it)
+ *  logging
+ *   "log"            1 = every plan that is built prints one line on stderr: row statistics, the SpMV kernel chosen, tiles and
+ *                    scratch; 0 = silent (default).  B200SP_LOG=1 in the environment sets it when the library is loaded.
  *  test switches (they make a failure path run; none of them can fault or hang the device)
  *   "spin_limit"       polls after which a kernel's bounded wait on a shared-memory barrier gives up, default 1048576
  *   "debug_no_copies"  1 = the kernels that stage data through shared memory (row-direct SpMV, ELL row-direct SpMV, SpMM with
@@ -69,6 +72,10 @@ extern "C" {
  *                      B200SP_ERR_ALLOC (the switch then clears itself); 0 = off (default)
  * "spmv_kernel", "merge_items" and "merge_empty" apply to plans created afterwards, the others to the next call. */
 int b200sp_set_option(const char* name, int value);
+/* Reads a switch back into *value (a host pointer).  Unknown names return B200SP_ERR_INVALID_ARG. */
+int b200sp_get_option(const char* name, int* value);
+/* Environment, read once when the library is loaded: B200SP_OPTIONS="name=value,name=value" sets switches as
+ * b200sp_set_option would (an entry that is not accepted is reported on stderr and skipped); B200SP_LOG=1 sets "log". */
 
 /* ---- measurement probes (no counterpart in the paper's operations) ----------------------------------------------
  * Each enqueues one kernel that does nothing but the access pattern named, so that the caller, timing it with events,

@@ -20,7 +20,7 @@ F32, BF16 = 0, 1
 EXPORTS = (
     "spmv_csr", "spmm_csr", "b200sp_plan_create", "b200sp_plan_destroy", "b200sp_plan_info", "b200sp_spmv",
     "b200sp_spmm", "spmv_csr_host", "spmm_csr_host", "b200sp_validate_csr", "b200sp_cache_clear",
-    "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_checked_build", "b200sp_launch_count", "b200sp_set_option",
+    "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_checked_build", "b200sp_launch_count", "b200sp_set_option", "b200sp_get_option",
     "b200sp_check", "b200sp_cache_drop", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_probe_gather_ex", "b200sp_probe_stream", "b200sp_probe_lines", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell", "spmv_csc", "spmm_csc", "spmv_csr_vec_host",
 )
 
@@ -106,6 +106,8 @@ def lib() -> ctypes.CDLL:
         L.b200sp_checked_build.restype = i32
         L.b200sp_launch_count.restype = i64
         L.b200sp_set_option.argtypes = [ctypes.c_char_p, i32]
+        L.b200sp_get_option.argtypes = [ctypes.c_char_p, ctypes.POINTER(ctypes.c_int)]
+        L.b200sp_get_option.restype = i32
         L.b200sp_check.argtypes = [p]
         L.b200sp_check.restype = i32
         for name in ("spmv_csr", "spmm_csr", "spmv_csr_host", "spmm_csr_host", "b200sp_plan_create", "b200sp_plan_destroy",
@@ -399,3 +401,9 @@ def b200sp_launch_count() -> int:
 
 def b200sp_set_option(name: str, value: int):
     _ck(lib().b200sp_set_option(name.encode(), value), "b200sp_set_option(%s)" % name)
+
+
+def b200sp_get_option(name: str) -> int:
+    out = ctypes.c_int(0)
+    _ck(lib().b200sp_get_option(name.encode(), ctypes.byref(out)), "b200sp_get_option(%s)" % name)
+    return out.value

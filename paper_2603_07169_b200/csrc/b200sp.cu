@@ -559,10 +559,9 @@ int b200sp_checked_build(void) {
 }
 int64_t b200sp_launch_count(void) { return g_launches.load(); }
 
-int b200sp_set_option(const char* name, int value) {
-  if (!name) return B200SP_ERR_INVALID_ARG;
-  std::lock_guard<std::mutex> lock(g_mutex);
-  // each switch accepts exactly the values listed for it in b200sp_tuning.h; the test suite runs every one of them
+// One row per switch: where it lives and which values it accepts (exactly those listed in b200sp_tuning.h; the test suite
+// runs every one of them).  Called with g_mutex held.
+static int option_access(const char* name, int* get, const int* set) {
   struct Entry { const char* name; int* slot; bool boolean; std::initializer_list<int> values; int lo, hi; };
   const Entry table[] = {
       {"spmv_kernel", &g_opt.spmv_kernel, false, {-1, 0, 1, 2, 3}, 0, 0},
@@ -589,12 +588,15 @@ int b200sp_set_option(const char* name, int value) {
       {"x_l2_window", &g_opt.x_l2_window, true, {}, 0, 0},
       {"pdl", &g_opt.pdl, true, {}, 0, 0},
       {"debug_no_copies", &g_opt.debug_no_copies, true, {}, 0, 0},
+      {"log", &g_opt.log, true, {}, 0, 0},
       {"pool_keep_mb", &g_opt.pool_keep_mb, false, {}, 0, 1 << 20},
       {"spin_limit", &g_opt.spin_limit, false, {}, 1, 1 << 30},
       {"fail_alloc_after", &g_opt.fail_alloc_after, false, {}, 0, 1 << 30},
   };
   for (const Entry& e : table) {
     if (strcmp(name, e.name)) continue;
+    if (get) { *get = *e.slot; return B200SP_OK; }
+    const int value = *set;
     if (e.boolean) { *e.slot = value ? 1 : 0; return B200SP_OK; }
     if (e.values.size()) {
       for (int v : e.values) if (v == value) { *e.slot = value; return B200SP_OK; }
@@ -607,4 +609,39 @@ int b200sp_set_option(const char* name, int value) {
   return B200SP_ERR_INVALID_ARG;
 }
 
+int b200sp_set_option(const char* name, int value) {
+  if (!name) return B200SP_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  return option_access(name, nullptr, &value);
+}
+
+int b200sp_get_option(const char* name, int* value) {
+  if (!name || !value) return B200SP_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  return option_access(name, value, nullptr);
+}
+
 }  // extern "C"
+
+// Environment at load time: B200SP_OPTIONS="name=value,name=value" sets switches as b200sp_set_option would (entries that
+// are not accepted are reported on stderr and skipped); B200SP_LOG=1 is short for the switch "log" = 1.
+namespace {
+struct EnvironmentAtLoad {
+  EnvironmentAtLoad() {
+    if (const char* lg = getenv("B200SP_LOG")) b200sp_set_option("log", atoi(lg));
+    const char* opts = getenv("B200SP_OPTIONS");
+    if (!opts) return;
+    std::string all(opts);
+    size_t pos = 0;
+    while (pos < all.size()) {
+      size_t end = all.find(',', pos);
+      if (end == std::string::npos) end = all.size();
+      const std::string item = all.substr(pos, end - pos);
+      const size_t eq = item.find('=');
+      if (eq == std::string::npos || b200sp_set_option(item.substr(0, eq).c_str(), atoi(item.c_str() + eq + 1)) != B200SP_OK)
+        fprintf(stderr, "b200sp: B200SP_OPTIONS entry '%s' not accepted\n", item.c_str());
+      pos = end + 1;
+    }
+  }
+} g_environment_at_load;
+}  // namespace

@@ -159,6 +159,14 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   if (g_opt.spmv_kernel == 1) choice = row_direct_possible ? 1 : 0;
   if (g_opt.spmv_kernel == 2) choice = uniform_ok ? 2 : (row_direct_ok ? 1 : 0);
   I.spmv_kernel = choice;
+  if (g_opt.log) {
+    static const char* const kname[4] = {"merge-tile", "row-direct", "uniform-row", "sub-warp"};
+    fprintf(stderr, "b200sp plan: m=%lld n=%lld nnz=%lld rows by length 0|1-4|5-32|33-128|129-1024|>1024 = %lld|%lld|%lld|%lld|%lld|%lld min=%d max=%d "
+                    "spmv kernel=%s tiles=%d x %d items%s scratch=%lld bytes\n",
+            (long long)m, (long long)n, (long long)nnz, (long long)I.bin_rows[0], (long long)I.bin_rows[1], (long long)I.bin_rows[2], (long long)I.bin_rows[3],
+            (long long)I.bin_rows[4], (long long)I.bin_rows[5], I.min_row_len, I.max_row_len, kname[choice & 3], I.spmv_tiles, I.spmv_tile_items,
+            p->compact_rows > 0 ? " (non-empty rows only)" : "", (long long)I.scratch_bytes);
+  }
   *out = p;
   return B200SP_OK;
 }

@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -66,6 +67,7 @@ struct Options {
   int pdl = 1;             // 1 = launch the kernels that begin with griddepcontrol.wait with programmatic stream serialisation
   int pool_keep_mb = 1024; // freed memory the library's pool keeps across synchronisation points, MiB (read when the pool is created)
   int merge_carve = 45;    // shared-memory carveout (percent) requested for it, -1 = leave to the driver
+  int log = 0;                // 1 = one line on stderr per plan built: row statistics and the kernel chosen (also set by B200SP_LOG=1 in the environment)
   // test switches (failure paths that must be reachable without faulting a GPU)
   int spin_limit = 1 << 20;   // polls before a bounded barrier wait gives up
   int debug_no_copies = 0;    // 1 = the kernels that stage through shared memory issue no copy and arm no barrier: their waits run out

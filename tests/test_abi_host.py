@@ -78,6 +78,28 @@ def test_invalid_arguments_are_rejected_on_the_host():
     assert L.b200sp_set_option(b"row_unroll", 3) == BAD
 
 
+def test_switches_read_back_and_environment_at_load():
+    """b200sp_get_option returns what b200sp_set_option stored; B200SP_OPTIONS / B200SP_LOG in the environment set switches when
+    the library is loaded (checked in a process of its own), and an entry that is not accepted is reported and skipped."""
+    import subprocess
+    import sys
+    assert b200sp.b200sp_get_option("merge_items") == 2048
+    b200sp.b200sp_set_option("merge_items", 4096)
+    try:
+        assert b200sp.b200sp_get_option("merge_items") == 4096
+    finally:
+        b200sp.b200sp_set_option("merge_items", 2048)
+    with pytest.raises(b200sp.B200spError):
+        b200sp.b200sp_get_option("no_such_option")
+    code = ("import sys; sys.path.insert(0, %r); import paper_2603_07169_b200 as b; "
+            "print(b.b200sp_get_option('spmv_kernel'), b.b200sp_get_option('merge_short'), b.b200sp_get_option('log'), b.b200sp_get_option('row_unroll'))" % ROOT)
+    env = dict(os.environ, B200SP_OPTIONS="spmv_kernel=0,merge_short=16,row_unroll=5,nonsense", B200SP_LOG="1")
+    out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, env=env, timeout=120)
+    assert out.returncode == 0, out.stderr
+    assert out.stdout.split() == ["0", "16", "1", "8"]
+    assert "row_unroll=5" in out.stderr and "nonsense" in out.stderr
+
+
 def test_empty_problem_is_a_no_op_without_a_device():
     L = b200sp.lib()
     assert L.spmv_csr(0, 0, 0, None, None, None, None, None, 1.0, 0.0, 0, None) == 0

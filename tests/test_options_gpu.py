@@ -108,13 +108,13 @@ def test_spmm_switch_value_against_oracle(switch, value, dtype):
 
 def test_every_switch_of_the_header_is_covered_here():
     """The list of switches in include/b200sp_tuning.h and the tables above must name the same switches (the test switches
-    spin_limit / debug_no_copies / fail_alloc_after and pool_keep_mb have tests of their own)."""
+    spin_limit / debug_no_copies / fail_alloc_after, pool_keep_mb and log have tests of their own)."""
     import os
     import re
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     text = open(os.path.join(root, "include", "b200sp_tuning.h")).read()
     declared = set(re.findall(r'^ \*\s+"([a-z_0-9]+)"', text, flags=re.M))
-    elsewhere = {"spin_limit", "debug_no_copies", "fail_alloc_after", "pool_keep_mb"}
+    elsewhere = {"spin_limit", "debug_no_copies", "fail_alloc_after", "pool_keep_mb", "log"}
     here = {s[0] for s in SPMV_SWITCHES} | {s[0] for s in SPMM_SWITCHES}
     assert declared == here | elsewhere, (sorted(declared - here - elsewhere), sorted((here | elsewhere) - declared))
     assert set(DEFAULTS) == here

@@ -435,3 +435,20 @@ def test_sizes_next_to_the_int32_limit():
         b200sp.b200sp_cache_clear()
         del col, val, row_ptr
         torch.cuda.empty_cache()
+
+
+def test_plan_log_line(capfd):
+    """With the switch "log" (B200SP_LOG=1 in the environment) every plan that is built reports its row statistics and the kernel chosen."""
+    w = gen.workload("c3", scale_down=3)
+    A = w.A
+    b200sp.b200sp_set_option("log", 1)
+    try:
+        plan = b200sp.b200sp_plan_create(A.m, A.n, A.nnz, to_dev(A.row_ptr))
+        b200sp.b200sp_plan_destroy(plan)
+    finally:
+        b200sp.b200sp_set_option("log", 0)
+    err = capfd.readouterr().err
+    L = np.diff(A.row_ptr)
+    assert "b200sp plan: m=%d n=%d nnz=%d" % (A.m, A.n, A.nnz) in err, err
+    assert "max=%d" % L.max() in err and "= %d|" % int((L == 0).sum()) in err, err
+    assert any("spmv kernel=" + k in err for k in ("merge-tile", "row-direct", "uniform-row", "sub-warp")), err
