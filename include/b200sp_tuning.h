@@ -23,6 +23,9 @@ extern "C" {
  *                    3 = sub-warp per row; a kernel the matrix is not eligible for falls back to an eligible one
  *   "spmm_bstage"    1 = SpMM keeps a slice of B in shared memory when A has few columns (default), 0 = never
  *   "spmm_sliced"    1 = SpMM walks k in 128-byte slices so that a slice of B can stay in L2 (default), 0 = one pass
+ *   "spmm_flat"      SpMM by chunks of 32 nonzeros per lane group instead of by rows (nnz-balanced, with carries between chunks and
+ *                    tiles): 1 = always, 0 = never, 2 = when the rows are uneven (default: 5 % or more of the nonzeros in rows
+ *                    longer than 128, a quarter or more of the rows empty, or a longest row far above the mean)
  *   "spmm_stage_a"   the k-sliced SpMM kernel's warps first copy their rows' (col, val) pairs into shared memory: 1 = yes, 0 = no,
  *                    2 = for BF16 storage only (default: measured 5-6 % faster there and 2-3 % slower for FP32)
  *   "spmm_ranges"    k-sliced SpMM on rows with ascending columns, one launch per column range so that the rows of B a

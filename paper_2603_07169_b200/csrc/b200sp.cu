@@ -568,6 +568,7 @@ static int option_access(const char* name, int* get, const int* set) {
       {"spmm_bstage", &g_opt.spmm_bstage, true, {}, 0, 0},
       {"spmm_sliced", &g_opt.spmm_sliced, true, {}, 0, 0},
       {"spmm_stage_a", &g_opt.spmm_stage_a, false, {0, 1, 2}, 0, 0},
+      {"spmm_flat", &g_opt.spmm_flat, false, {0, 1, 2}, 0, 0},
       {"spmm_ranges", &g_opt.spmm_ranges, false, {0, 1, 2, 3, 4, 8}, 0, 0},
       {"merge_items", &g_opt.merge_items, false, {1024, 2048, 4096}, 0, 0},
       {"merge_threads", &g_opt.merge_threads, false, {64, 128, 256}, 0, 0},

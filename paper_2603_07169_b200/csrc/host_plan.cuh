@@ -20,12 +20,13 @@ constexpr size_t kCacheCap = 1024;
 int plan_free(b200sp_plan* p, bool stream_ordered = false, cudaStream_t stream = nullptr) {
   if (!p) return B200SP_OK;
   int rc = B200SP_OK;
-  if (p->block || p->cuts_block || p->compact_block) {
+  if (p->block || p->cuts_block || p->compact_block || p->flat_tile_row) {
     cudaError_t e = cudaSuccess;
     if (stream_ordered) {
       if (p->block) e = cudaFreeAsync(p->block, stream);
       if (p->cuts_block && e == cudaSuccess) e = cudaFreeAsync(p->cuts_block, stream);
       if (p->compact_block && e == cudaSuccess) e = cudaFreeAsync(p->compact_block, stream);
+      if (p->flat_tile_row && e == cudaSuccess) e = cudaFreeAsync(p->flat_tile_row, stream);
     } else {
       int cur = 0;
       e = cudaGetDevice(&cur);
@@ -34,12 +35,44 @@ int plan_free(b200sp_plan* p, bool stream_ordered = false, cudaStream_t stream =
       if (e == cudaSuccess && p->block) e = cudaFree(p->block);
       if (e == cudaSuccess && p->cuts_block) e = cudaFree(p->cuts_block);
       if (e == cudaSuccess && p->compact_block) e = cudaFree(p->compact_block);
+      if (e == cudaSuccess && p->flat_tile_row) e = cudaFree(p->flat_tile_row);
       if (cur != p->device) cudaSetDevice(cur);
     }
     if (e != cudaSuccess) rc = cuda_fail(e, "freeing a plan");
   }
   delete p;
   return rc;
+}
+
+// The list of the rows that have nonzeros (their numbers and their offsets), built on the device in stream order and kept with
+// the plan: used by the merge-tile SpMV kernel under the switch "merge_empty" and by the nnz-balanced SpMM kernel.  Needs
+// info.bin_rows[0] (the number of empty rows).  No synchronisation.
+int plan_compact_rows(b200sp_plan* p, cudaStream_t stream, DeviceInfo* dev) {
+  if (p->compact_block) return B200SP_OK;
+  b200sp_plan_info_t& I = p->info;
+  const int64_t m = I.m, mc = m - I.bin_rows[0];
+  auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+  const int blocks = (int)((m + kCompactBlock - 1) / kCompactBlock);
+  const size_t o_id = 0, o_rp = o_id + up((size_t)(mc + 1) * 4), o_bc = o_rp + up((size_t)(mc + 1) * 4), total = o_bc + up((size_t)(blocks + 1) * 4);
+  void* blk = nullptr;
+  int rc = pool_alloc(dev, &blk, total, stream);
+  if (rc != B200SP_OK) return rc;
+  char* b2 = (char*)blk;
+  int32_t* row_id = (int32_t*)(b2 + o_id);
+  int32_t* row_ptr_c = (int32_t*)(b2 + o_rp);
+  int* d_bc = (int*)(b2 + o_bc);
+  plan_compact_count_kernel<<<blocks, 256, 0, stream>>>(p->row_ptr, (int)m, d_bc);
+  plan_compact_scan_kernel<<<1, 1024, 0, stream>>>(d_bc, blocks);
+  plan_compact_write_kernel<<<blocks, 256, 0, stream>>>(p->row_ptr, (int)m, (int)I.nnz, d_bc, row_id, row_ptr_c);
+  g_launches += 3;
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { cudaFreeAsync(blk, stream); return cuda_fail(e, "list of non-empty rows"); }
+  p->compact_block = blk;
+  p->compact_row_id = row_id;
+  p->compact_row_ptr = row_ptr_c;
+  p->compact_rows = (int)mc;
+  I.scratch_bytes += (int64_t)total;
+  return B200SP_OK;
 }
 
 int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32_t* row_ptr, cudaStream_t stream) {
@@ -117,26 +150,17 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
   // Many rows without nonzeros (a quarter or more): the merge list is built over the rows that have nonzeros only, and the
   // split points are searched again over that list.
   if (!h.bad && g_opt.merge_empty && nnz > 0 && (int64_t)h.bin_rows[0] * 4 >= m) {
-    const int64_t mc = m - (int64_t)h.bin_rows[0];
-    const int blocks = (int)((m + kCompactBlock - 1) / kCompactBlock);
-    const size_t o_id = 0, o_rp = o_id + up((size_t)mc * 4), o_bc = o_rp + up((size_t)(mc + 1) * 4), tot2 = o_bc + up((size_t)(blocks + 1) * 4);
-    rc = pool_alloc(dev, &p->compact_block, tot2, stream);
+    for (int j = 0; j < B200SP_NUM_BINS; ++j) I.bin_rows[j] = (int64_t)h.bin_rows[j];
+    rc = plan_compact_rows(p, stream, dev);
     if (rc != B200SP_OK) return fail(rc);
-    char* b2 = (char*)p->compact_block;
-    p->compact_row_id = (int32_t*)(b2 + o_id);
-    p->compact_row_ptr = (int32_t*)(b2 + o_rp);
-    int* d_bc = (int*)(b2 + o_bc);
-    plan_compact_count_kernel<<<blocks, 256, 0, stream>>>(row_ptr, (int)m, d_bc);
-    plan_compact_scan_kernel<<<1, 1024, 0, stream>>>(d_bc, blocks);
-    plan_compact_write_kernel<<<blocks, 256, 0, stream>>>(row_ptr, (int)m, (int)nnz, d_bc, p->compact_row_id, p->compact_row_ptr);
+    const int64_t mc = p->compact_rows;
     const size_t ntc = (size_t)((mc + nnz + items - 1) / items);     // fewer items, fewer tiles: the arrays sized above suffice
     plan_merge_split_kernel<<<(unsigned)((ntc + 1 + 255) / 256), 256, 0, stream>>>(p->compact_row_ptr, (int)mc, (int)nnz, items, (int)ntc, p->split_row);
-    g_launches += 4;
+    g_launches++;
     CUP(cudaGetLastError());
     CUP(cudaStreamSynchronize(stream));
-    p->compact_rows = (int)mc;
+    p->merge_compact = true;
     I.spmv_tiles = (int32_t)ntc;
-    I.scratch_bytes += (int64_t)tot2;
   }
 #undef CUP
   if (h.bad) { plan_free(p, true, stream); cudaStreamSynchronize(stream); return B200SP_ERR_BAD_CSR; }
@@ -165,7 +189,7 @@ int plan_build(b200sp_plan** out, int64_t m, int64_t n, int64_t nnz, const int32
                     "spmv kernel=%s tiles=%d x %d items%s scratch=%lld bytes\n",
             (long long)m, (long long)n, (long long)nnz, (long long)I.bin_rows[0], (long long)I.bin_rows[1], (long long)I.bin_rows[2], (long long)I.bin_rows[3],
             (long long)I.bin_rows[4], (long long)I.bin_rows[5], I.min_row_len, I.max_row_len, kname[choice & 3], I.spmv_tiles, I.spmv_tile_items,
-            p->compact_rows > 0 ? " (non-empty rows only)" : "", (long long)I.scratch_bytes);
+            p->merge_compact ? " (non-empty rows only)" : "", (long long)I.scratch_bytes);
   }
   *out = p;
   return B200SP_OK;

@@ -62,6 +62,7 @@ struct Options {
   int sub_lanes = 0;       // lanes per row of the sub-warp kernel (0 = from the mean row length)
   int merge_empty = 0;     // 1 = when a quarter or more of the rows have no nonzeros the merge list holds only the others, 0 = every row is a merge item (default: measured 3 % slower on the power-law workload, where the extra pass over y costs more than the skipped items save)
   int spmm_stage_a = 2;    // the k-sliced SpMM kernel's warps stage their rows' (col, val) pairs in shared memory: 1 = yes, 0 = no (broadcast loads from global memory), 2 = for BF16 storage only (default)
+  int spmm_flat = 2;       // nnz-balanced SpMM kernel (a chunk of nonzeros per lane group instead of a row): 1 = always, 0 = never, 2 = when the rows are uneven (default)
   int spmm_ranges = 1;     // column ranges per slice of the k-sliced SpMM kernel with sorted columns: 1 = none (default), 0 = as many as make a range of B fit L2, 2, 3, 4, 8 = forced
   int merge_short = 32;    // rows up to this many products are added by one thread (8, 16, 32, 64)
   int pdl = 1;             // 1 = launch the kernels that begin with griddepcontrol.wait with programmatic stream serialisation
@@ -246,9 +247,11 @@ struct b200sp_plan {
   unsigned long long* probe_out = nullptr;  // two counters for the column-locality probe
   int num_medium = 0, num_long = 0;
   const void* probed_col_idx = nullptr;   // col_idx the column-locality probe last ran on
+  int32_t* flat_tile_row = nullptr;       // tile starts of the nnz-balanced SpMM kernel (a pool block of its own, built on first use)
   // merge list over the rows that have nonzeros (matrices with many empty rows)
   void* compact_block = nullptr;          // one pool block: row ids, their offsets, block counts
-  int compact_rows = 0;                   // 0 = the merge list is the matrix's own row list
+  int compact_rows = 0;                   // number of rows that have nonzeros (0 = the list has not been built)
+  bool merge_compact = false;             // the SpMV merge list (split_row) was built over that list
   int32_t* compact_row_id = nullptr;      // compact_rows matrix row numbers, ascending
   int32_t* compact_row_ptr = nullptr;     // compact_rows + 1 offsets
   // column ranges of the k-sliced SpMM kernel (rows with ascending columns): built on the first SpMM call with a given col_idx

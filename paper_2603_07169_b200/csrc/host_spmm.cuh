@@ -134,6 +134,70 @@ int spmm_column_ranges(b200sp_plan* p, const int32_t* col_idx, int slice_bytes, 
   return B200SP_OK;
 }
 
+// nnz-balanced SpMM (spmm_flat_kernel) for matrices whose rows are too uneven for one lane group per row.
+constexpr int kFlatChunk = 32;                          // nonzeros per lane group
+constexpr int kFlatTile = (kSpmmThreads / 8) * kFlatChunk;   // nonzeros per CTA
+
+bool spmm_rows_are_uneven(const b200sp_plan_info_t& I) {
+  if (I.nnz <= 0 || I.m <= 0) return false;
+  const int64_t nonempty = I.m - I.bin_rows[0];
+  const double mean = (double)I.nnz / (double)(nonempty > 0 ? nonempty : 1);
+  return (I.bin_nnz[4] + I.bin_nnz[5]) * 20 >= I.nnz      // 5 % or more of the nonzeros sit in rows longer than 128
+         || I.bin_rows[0] * 4 >= I.m                        // a quarter or more of the rows are empty
+         || (double)I.max_row_len > 4.0 * mean + 8.0;       // or the longest row is far above the mean
+}
+
+template <typename T, int VEC>
+int run_spmm_flat(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const T* B, T* Y, float alpha, float beta,
+                  cudaStream_t stream, DeviceInfo* dev) {
+  const b200sp_plan_info_t& I = p->info;
+  constexpr int KS = 8 * VEC;
+  const int tiles = (int)((I.nnz + kFlatTile - 1) / kFlatTile);
+  const int slices = (k + KS - 1) / KS;
+  if ((long long)slices * tiles >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+  int rc;
+  if (I.bin_rows[0] > 0) {   // the rows that have nonzeros, listed once per plan (stream order, no synchronisation)
+    rc = plan_compact_rows(p, stream, dev);
+    if (rc != B200SP_OK) return rc;
+  }
+  const int rows = I.bin_rows[0] > 0 ? p->compact_rows : (int)I.m;
+  const int* rp = I.bin_rows[0] > 0 ? p->compact_row_ptr : p->row_ptr;
+  const int* rid = I.bin_rows[0] > 0 ? p->compact_row_id : nullptr;
+  if (!p->flat_tile_row) {   // tile starts: once per plan, a small kernel in stream order
+    rc = pool_alloc(dev, (void**)&p->flat_tile_row, (size_t)(tiles + 1) * sizeof(int32_t), stream);
+    if (rc != B200SP_OK) return rc;
+    rc = launch(plan_nnz_tile_rows_kernel, dim3((unsigned)((tiles + 1 + 255) / 256)), dim3(256), stream, nullptr, 0, dev, rp, rows,
+                (int)I.nnz, kFlatTile, tiles, (int*)p->flat_tile_row);
+    if (rc != B200SP_OK) return rc;
+  }
+  // per-call scratch: what each tile leaves unfinished and what it finishes for an earlier tile, KS floats per (slice, tile)
+  float* scratch = nullptr;
+  const size_t per = (size_t)slices * tiles * KS;
+  rc = pool_alloc(dev, (void**)&scratch, 2 * per * sizeof(float), stream);
+  if (rc != B200SP_OK) return rc;
+  if (I.bin_rows[0] > 0) {
+    long long blocks = ((long long)I.m * (k / VEC) + 255) / 256;
+    if (blocks > (long long)dev->sms * 16) blocks = (long long)dev->sms * 16;
+    rc = launch(spmm_empty_rows_kernel<T, VEC>, dim3((unsigned)blocks), dim3(256), stream, nullptr, 0, dev, (int)I.m, k, p->row_ptr, Y, beta);
+  }
+  if (rc == B200SP_OK) {
+    tl_pdl_kernel = true;
+    rc = launch(spmm_flat_kernel<T, VEC, kSpmmThreads, kFlatChunk>, dim3((unsigned)(slices * tiles)), dim3(kSpmmThreads), stream, B,
+                (size_t)I.n * k * sizeof(T), dev, rows, (int)I.nnz, k, tiles, rp, rid, (const int*)p->flat_tile_row, col_idx, vals, B, Y,
+                scratch, scratch + per, alpha, beta);
+  }
+  if (rc == B200SP_OK && tiles > 1) {
+    const long long groups = (long long)slices * tiles;
+    tl_pdl_kernel = true;
+    rc = launch(spmm_flat_fixup_kernel<T, VEC, kSpmmThreads, kFlatTile>, dim3((unsigned)((groups * 8 + kSpmmThreads - 1) / kSpmmThreads)),
+                dim3(kSpmmThreads), stream, nullptr, 0, dev, rows, (int)I.nnz, k, tiles, slices, rp, rid, (const int*)p->flat_tile_row,
+                (const float*)scratch, (const float*)(scratch + per), Y, alpha, beta);
+  }
+  const cudaError_t e = cudaFreeAsync(scratch, stream);
+  if (e != cudaSuccess && rc == B200SP_OK) rc = cuda_fail(e, "cudaFreeAsync");
+  return rc;
+}
+
 template <typename T, int VEC>
 int run_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const T* B, T* Y, float alpha, float beta,
              cudaStream_t stream, DeviceInfo* dev) {
@@ -172,6 +236,8 @@ int run_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const
     const int slices = (k + KS - 1) / KS;
     const int row_blocks = (int)((I.m + GROUPS - 1) / GROUPS);
     if ((long long)slices * row_blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+    if (lanes == 8 && (g_opt.spmm_flat == 1 || (g_opt.spmm_flat == 2 && spmm_rows_are_uneven(I))))
+      return run_spmm_flat<T, VEC>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev);
     int rc;
     const int mid_blocks = (p->num_medium + GROUPS - 1) / GROUPS;
     int ranges = 1;

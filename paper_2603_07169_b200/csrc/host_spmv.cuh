@@ -173,9 +173,9 @@ int run_spmv_merge(b200sp_plan* p, const int32_t* col_idx, const T* vals, const 
                    cudaStream_t stream, DeviceInfo* dev) {
   const b200sp_plan_info_t& I = p->info;
   const int tiles = I.spmv_tiles;
-  const int rows = p->compact_rows > 0 ? p->compact_rows : (int)I.m;
-  const int* rp = p->compact_rows > 0 ? p->compact_row_ptr : p->row_ptr;
-  const int* rid = p->compact_rows > 0 ? p->compact_row_id : nullptr;
+  const int rows = p->merge_compact ? p->compact_rows : (int)I.m;
+  const int* rp = p->merge_compact ? p->compact_row_ptr : p->row_ptr;
+  const int* rid = p->merge_compact ? p->compact_row_id : nullptr;
   int rc = B200SP_OK;
   if (rid) {
     rc = run_empty_rows<T>(p, y, beta, stream, dev);

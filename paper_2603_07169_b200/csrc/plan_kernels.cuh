@@ -144,6 +144,22 @@ __global__ void __launch_bounds__(256) plan_compact_write_kernel(const int* __re
   if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) row_ptr_c[out] = nnz;
 }
 
+// Tile starts of the nnz-balanced SpMM kernel: tile_row[t] = the row that holds nonzero t * tile_nnz, i.e. the first r with
+// row_ptr[r + 1] > t * tile_nnz (rows without nonzeros are skipped over); m when t * tile_nnz >= nnz.
+__global__ void __launch_bounds__(256) plan_nnz_tile_rows_kernel(const int* __restrict__ row_ptr, int m, int nnz, int tile_nnz, int tiles,
+                                                                 int* __restrict__ tile_row) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t > tiles) return;
+  const long long p = (long long)t * tile_nnz;
+  if (p >= nnz) { tile_row[t] = m; return; }
+  int lo = 0, hi = m - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if ((long long)row_ptr[mid + 1] <= p) lo = mid + 1; else hi = mid;
+  }
+  tile_row[t] = lo;
+}
+
 // Rows of mid_thresh + 1 .. long_thresh nonzeros and rows longer than long_thresh, each appended to a list of its own
 // (count[0], count[1]; the host sorts the lists, and their order only affects scheduling, never a value).
 __global__ void __launch_bounds__(256) plan_row_lists_kernel(const int* __restrict__ row_ptr, int m, int mid_thresh, int long_thresh,

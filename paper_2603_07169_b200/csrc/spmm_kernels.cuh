@@ -497,6 +497,193 @@ spmm_medium_row_kernel(int num_rows, const int* __restrict__ rows, int k, int ro
   slice_store<T, VEC>(Y + row * k + col0, tot, alpha, beta);
 }
 
+// ---- nnz-balanced SpMM for irregular rows -------------------------------------------------------------------------------
+// The k-sliced kernels above give every row to one group of eight lanes, so a row of a thousand nonzeros keeps its group busy
+// long after its neighbours' rows of three are done, and empty rows idle the groups they were dealt.  Here the unit of work is
+// a CHUNK of C consecutive nonzeros per lane group, whatever rows they belong to; a CTA owns a tile of GROUPS chunks.  A group
+// walks its chunk row segment by row segment (the same vectorised inner loop), stores the rows that begin and end inside the
+// chunk, and leaves two partial sums in shared memory: `head` for a first row that began before the chunk, `carry` for a last
+// row that goes on after it.  After one barrier the group that holds a row's end adds the carries of the groups before it (in
+// group order: reproducible) and stores the row; what crosses the tile's own ends goes to tile_tail / tile_carry in global
+// memory and is finished by spmm_flat_fixup_kernel.  The rows are those that have nonzeros (m of them; row_ptr their m + 1
+// offsets; row_id[r] the matrix row of list row r, or nullptr when every row of the matrix has nonzeros), so a tile holds at most
+// TILE rows and all their bounds fit in shared memory; Y of the rows without nonzeros is written by spmm_empty_rows_kernel.
+// No chain is longer than C products plus one term per group or tile that a row spans.
+//   tile_row[t]  the list row that holds nonzero t * TILE, m for t * TILE >= nnz
+template <typename T, int VEC, int THREADS, int C>
+__global__ void __launch_bounds__(THREADS)
+spmm_flat_kernel(int m, int nnz, int k, int tiles, const int* __restrict__ row_ptr, const int* __restrict__ row_id,
+                 const int* __restrict__ tile_row, const int* __restrict__ col_idx, const T* __restrict__ vals, const T* __restrict__ B,
+                 T* __restrict__ Y, float* __restrict__ tile_carry, float* __restrict__ tile_tail, float alpha, float beta) {
+  constexpr int LANES = 8, GROUPS = THREADS / LANES, KS = LANES * VEC, TILE = GROUPS * C, RB = TILE + 32;
+  __shared__ int rp_s[RB];                       // row_ptr[r_lo .. r_lo + RB): the bounds of the tile's rows (what does not fit is read from global memory)
+  __shared__ float head_s[GROUPS][KS], carry_s[GROUPS][KS];
+  grid_dependency_wait();
+  const int slice = blockIdx.x / tiles, t = blockIdx.x - slice * tiles;
+  const int p_lo = t * TILE, p_hi = min(nnz, p_lo + TILE);
+  const int r_lo = __ldg(tile_row + t);
+  const int r_hi = min(__ldg(tile_row + t + 1), m - 1);
+  for (int j = threadIdx.x; j < RB && r_lo + j <= m; j += THREADS) rp_s[j] = __ldg(row_ptr + r_lo + j);
+  __syncthreads();
+  auto bound = [&](int r) { const int j = r - r_lo; return j < RB ? rp_s[j] : __ldg(row_ptr + r); };
+  const int g = threadIdx.x / LANES, l8 = threadIdx.x % LANES;
+  const int col0 = slice * KS + l8 * VEC;
+  const bool active = col0 < k;
+  const T* Bc = B + col0;
+  const int c0 = p_lo + g * C, c1 = min(p_hi, c0 + C);
+  typedef typename RawVec<T, VEC>::type raw_t;
+  int head_row = -1, carry_rs = -1;              // the row whose end this chunk holds but whose start it does not; the start of the row it leaves unfinished
+  bool has_carry = false;
+  float acc[VEC];
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
+  if (c0 < c1) {
+    int lo = r_lo, hi = r_hi;                    // the row that holds nonzero c0: the first r with row_ptr[r + 1] > c0
+    while (lo < hi) { const int mid = (lo + hi) >> 1; if (bound(mid + 1) <= c0) lo = mid + 1; else hi = mid; }
+    int r = lo, rs = bound(r), re = bound(r + 1);
+    // a row that has been added up to its last nonzero: stored if it began in this chunk, else left as the chunk's head
+    auto finish_row = [&]() {
+      if (rs >= c0) { if (active) slice_store<T, VEC>(Y + (long long)(row_id ? __ldg(row_id + r) : r) * k + col0, acc, alpha, beta); }
+      else {
+        head_row = r;
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) head_s[g][l8 * VEC + j] = acc[j];
+      }
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
+    };
+    const int nnz4 = nnz & ~3;
+    // the chunk is walked four nonzeros at a time whatever rows they belong to (c0 is a multiple of four): the loads stay
+    // vectorised and four reads of B are in flight even where the rows are one or two nonzeros long
+    for (int q = c0; q < c1; q += 4) {
+      int c[4]; float v[4];
+      if (q + 4 <= nnz4) ld_a4(col_idx, vals, q, c, v);
+      else {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { const bool in = q + u < c1; c[u] = in ? __ldg(col_idx + q + u) : 0; v[u] = in ? to_f32(__ldg(vals + q + u)) : 0.0f; }
+      }
+      raw_t bv[4];
+      if (active) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) bv[u] = RawVec<T, VEC>::ld(Bc + (long long)c[u] * k);   // past c1 the column is one of the chunk's own or 0: a valid row of B
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int p = q + u;
+        if (p < c1) {
+          if (p == re) {                         // row r ended just before p: finish it and move to the row that holds p
+            finish_row();
+            do { ++r; rs = re; re = bound(r + 1); } while (re == rs);
+          }
+          if (active) RawVec<T, VEC>::fma(bv[u], v[u], acc);
+        }
+      }
+    }
+    if (re <= c1) finish_row();                  // the last row ends with the chunk
+    else {                                       // or goes on after it
+      has_carry = true;
+      carry_rs = rs;
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) carry_s[g][l8 * VEC + j] = acc[j];
+    }
+  }
+  if (!has_carry) {
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) carry_s[g][l8 * VEC + j] = 0.0f;
+  }
+  __syncthreads();
+  const long long slot = ((long long)slice * tiles + t) * KS + l8 * VEC;
+  if (head_row >= 0) {                           // complete the row that ends here: carries of the groups it passed through, in order, then the head
+    const int rs = bound(head_row);
+    const int j0 = rs >= p_lo ? (rs - p_lo) / C : 0;
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
+    for (int u = j0; u < g; ++u) {
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) acc[j] += carry_s[u][l8 * VEC + j];
+    }
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) acc[j] += head_s[g][l8 * VEC + j];
+    if (rs >= p_lo) { if (active) slice_store<T, VEC>(Y + (long long)(row_id ? __ldg(row_id + head_row) : head_row) * k + col0, acc, alpha, beta); }
+    else {
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) tile_tail[slot + j] = acc[j];   // began in an earlier tile: finished by the fix-up kernel
+    }
+  }
+  if (c0 < c1 && c1 == p_hi) {                   // the tile's last chunk: what the tile leaves unfinished
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
+    if (has_carry) {
+      const int j1 = carry_rs >= p_lo ? (carry_rs - p_lo) / C : 0;
+      for (int u = j1; u <= g; ++u) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) acc[j] += carry_s[u][l8 * VEC + j];
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) tile_carry[slot + j] = acc[j];
+  }
+}
+
+// Finishes the rows that a tile boundary of spmm_flat_kernel cut: tile t holds the end of such a row when its first row began
+// before the tile's first nonzero and ends inside the tile.  The row's value is tile_carry[first .. t-1] + tile_tail[t], the
+// carries added in blocks of 16 whose sums form a second chain; one lane group per (slice, tile), fixed order.
+template <typename T, int VEC, int THREADS, int TILE>
+__global__ void __launch_bounds__(THREADS)
+spmm_flat_fixup_kernel(int m, int nnz, int k, int tiles, int slices, const int* __restrict__ row_ptr, const int* __restrict__ row_id,
+                       const int* __restrict__ tile_row, const float* __restrict__ tile_carry, const float* __restrict__ tile_tail,
+                       T* __restrict__ Y, float alpha, float beta) {
+  constexpr int LANES = 8, KS = LANES * VEC;
+  grid_dependency_wait();
+  const long long id = ((long long)blockIdx.x * THREADS + threadIdx.x) / LANES;
+  const int l8 = threadIdx.x % LANES;
+  if (id >= (long long)slices * tiles) return;
+  const int slice = (int)(id / tiles), t = (int)(id - (long long)slice * tiles);
+  if (t < 1) return;
+  const int p_lo = t * TILE, p_hi = min(nnz, p_lo + TILE);
+  const int r = tile_row[t];
+  if (r >= m) return;
+  const int rs = row_ptr[r], re = row_ptr[r + 1];
+  if (rs >= p_lo || re > p_hi) return;           // the tile's first row begins inside it, or does not end in it
+  const int col0 = slice * KS + l8 * VEC;
+  if (col0 >= k) return;
+  const int tf = rs / TILE;
+  float acc[VEC], blk[VEC];
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
+  for (int u = tf; u < t; u += 16) {
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) blk[j] = 0.0f;
+    const int ue = min(u + 16, t);
+    for (int v = u; v < ue; ++v) {
+      const float* c = tile_carry + ((long long)slice * tiles + v) * KS + l8 * VEC;
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) blk[j] += c[j];
+    }
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) acc[j] += blk[j];
+  }
+  const float* tl = tile_tail + ((long long)slice * tiles + t) * KS + l8 * VEC;
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) acc[j] += tl[j];
+  slice_store<T, VEC>(Y + (long long)(row_id ? row_id[r] : r) * k + col0, acc, alpha, beta);
+}
+
+// Y[i, :] = beta * Y[i, :] (zero when beta == 0) for the rows without nonzeros: the pass that goes with spmm_flat_kernel.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(256) spmm_empty_rows_kernel(int m, int k, const int* __restrict__ row_ptr, T* __restrict__ Y, float beta) {
+  const int vecs = k / VEC;
+  const long long total = (long long)m * vecs;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long row = i / vecs;
+    if (__ldg(row_ptr + row) != __ldg(row_ptr + row + 1)) continue;
+    float z[VEC];
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) z[j] = 0.0f;
+    slice_store<T, VEC>(Y + row * k + (i - row * vecs) * VEC, z, 0.0f, beta);
+  }
+}
+
 // One CTA per (long row, slice): the CTA's groups of eight lanes stride over the row's nonzeros (sums in blocks of
 // kChainBlock / 2 products, block sums in a second chain), then the per-group partial sums are combined pairwise through
 // shared memory in a fixed tree (reproducible; five levels instead of a chain of 32).

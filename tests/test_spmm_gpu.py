@@ -183,3 +183,75 @@ def test_output_larger_than_2_31_elements():
             b200sp.b200sp_set_option("spmm_bstage", 1)
             b200sp.b200sp_cache_clear()
     b200sp.b200sp_check()
+
+
+def flat_row_cases():
+    rng = np.random.default_rng(0)
+    return {
+        "every_length_0_to_130": np.arange(131),
+        "all_empty_but_one": np.concatenate([np.zeros(3000, np.int64), [5], np.zeros(3000, np.int64)]),
+        "one_huge_row": np.array([3, 0, 100000, 5, 0, 0, 1]),
+        "huge_first_and_last": np.array([20000, 1, 0, 2, 30000]),
+        "single_row": np.array([9000]),
+        "single_entry": np.array([1]),
+        "rows_of_32": np.full(700, 32),                      # chunks and rows coincide
+        "rows_of_31_33": np.tile([31, 33], 400),             # every chunk boundary cuts a row
+        "tile_exact": np.full(64, 1024),                     # rows and tiles coincide
+        "power_law": (rng.pareto(1.2, 3000) * 3).astype(np.int64).clip(0, 40000),
+        "long_run_of_empty_rows_inside_a_tile": np.concatenate([[7], np.zeros(5000, np.int64), [9], np.zeros(2000, np.int64), [2000]]),
+    }
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("case", sorted(flat_row_cases()))
+def test_nnz_balanced_kernel_adversarial_rows(case, dtype):
+    """The nnz-balanced SpMM kernel (a chunk of 32 nonzeros per lane group, carries between chunks and tiles) forced on row-length
+    patterns that hit every branch: rows inside a chunk, rows cut by chunk and by tile boundaries, rows spanning many tiles,
+    runs of empty rows longer than the tile's staged row bounds, k that is and is not a multiple of a slice, beta != 0."""
+    lens = flat_row_cases()[case]
+    m, n = len(lens), 777
+    A = gen.random_csr(m, n, lens, seed=len(case), sort_cols=False, allow_dup=True)
+    rng = np.random.default_rng(2)
+    b200sp.b200sp_set_option("spmm_flat", 1)
+    b200sp.b200sp_set_option("spmm_bstage", 0)
+    try:
+        for k in (64, 72):
+            B = rng.standard_normal(n * k).astype(np.float32)
+            Y0 = rng.standard_normal(m * k).astype(np.float32)
+            Y, Y_ref, S = run_spmm(A, B, k, None, 1.0, 0.0, dtype)
+            assert_within(Y, Y_ref, S, dtype, what="flat %s k=%d" % (case, k))
+            Y, Y_ref, S = run_spmm(A, B, k, Y0, -0.5, 1.25, dtype)
+            y0f = Y0 if dtype == "f32" else gen.bf16_to_f32(gen.to_bf16(Y0))
+            assert_within(Y, Y_ref, S, dtype, 1.0, np.abs(1.25 * y0f.astype(np.float64)).reshape(m, k), what="flat %s k=%d ab" % (case, k))
+    finally:
+        b200sp.b200sp_set_option("spmm_flat", 2)
+        b200sp.b200sp_set_option("spmm_bstage", 1)
+
+
+def test_nnz_balanced_kernel_is_reproducible_and_keeps_chains_short():
+    """Bit-identical results from run to run (the carries are added in a fixed order), and all-positive data on rows of up to
+    60,000 nonzeros stays far below the literal FP32 bound."""
+    import torch
+    from gpu_util import empty_out, store, to_dev
+    rng = np.random.default_rng(9)
+    lens = (rng.pareto(1.1, 20000) * 2).astype(np.int64).clip(0, 60000)
+    n, k = 50000, 64
+    A = gen.random_csr(len(lens), n, lens, seed=4)
+    A.vals[:] = rng.random(A.nnz).astype(np.float32) + 0.01
+    B = rng.random(n * k).astype(np.float32) + 0.01
+    b200sp.b200sp_set_option("spmm_flat", 1)
+    try:
+        Y, Y_ref, S = run_spmm(A, B, k, None, 1.0, 0.0, "f32")
+        assert assert_within(Y, Y_ref, S, "f32", what="flat, positive data") < 0.5
+        d = [to_dev(a) for a in (A.row_ptr, A.col_idx, A.vals, B)]
+        outs = []
+        for _ in range(3):
+            Yd = empty_out(A.m * k, "f32")
+            b200sp.spmm_csr(A.m, A.n, A.nnz, k, d[0], d[1], d[2], d[3], Yd, 1.0, 0.0, "f32")
+            torch.cuda.synchronize()
+            outs.append(Yd.cpu().numpy().copy())
+        assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+        assert np.array_equal(outs[0].reshape(A.m, k), Y)
+    finally:
+        b200sp.b200sp_set_option("spmm_flat", 2)
+        b200sp.b200sp_cache_clear()
