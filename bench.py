@@ -865,6 +865,25 @@ def main():
                     b200sp.b200sp_set_option("x_l2_window", 0)
                     b200sp.b200sp_cache_clear()
                     torch.cuda.empty_cache()
+        # SpMM on the power-law matrix (not one of the five configurations): the nnz-balanced kernel that the plan picks for uneven rows
+        try:
+            cache = {}
+            wpl = gen.workload("c3k64")
+            lr = probe_lines_rate(dev)
+            for dt in ("f32", "bf16"):
+                r = measure(wpl, dt, min(steps, 20), 3, dev, l2, cusparse=cusp)
+                extras["c3k64_%s" % dt] = {
+                    "ms_per_step": round(r["ms_per_step"], 5), "gbs": round(r["gbs"], 1), "frac_of_hbm": round(r["gbs"] / peak, 4),
+                    "algorithmic_bytes": r["algorithmic_bytes"], "nnz": r["nnz"], "copies": r["copies"],
+                    "cusparse_ms": round(r["cusparse_ms"], 5) if isinstance(r["cusparse_ms"], float) else r["cusparse_ms"],
+                    "line_read_bound_ms": round(wpl.A.nnz * 64 * (4 if dt == "f32" else 2) / lr * 1e3, 5),
+                    "note": "R-MAT scale 22 pattern (61 % empty rows, rows up to 57 k) times a dense 2^22 x 64 B: spmm_flat_kernel"}
+                del r
+                b200sp.b200sp_cache_clear()
+                torch.cuda.empty_cache()
+            del wpl
+        except Exception as ex:  # pragma: no cover
+            extras["c3k64"] = {"error": repr(ex)}
         extras["x_l2_window_ab"] = dict(window_ab, note="per-launch access-policy window (persisting hits) over x, or over B for SpMM; default off")
         # the COO and ELL front ends on the same matrices (paper tasks 8 and 14)
         for name, dt in (("c2", "f32"), ("c4", "bf16")):

@@ -259,6 +259,7 @@ def workload(name: str, scale_down: int = 0) -> Workload:
     c2  m = n = 2^20, exactly 16 nnz/row, vals N(0,1), x and y0 U[-1,1), alpha 1.5, beta 0.5 (FP32, BF16)
     c3  R-MAT scale 22, 34.14 M generated edges, vals and x U(0,1], alpha 1, beta 0    (FP32)
     c3p the edges of c3 with every vertex renamed by one pseudo-random bijection (secondary measurement) (FP32)
+    c3k64  the matrix of c3 times a dense B N(0,1) of n x 64: SpMM on uneven rows (secondary measurement) (FP32, BF16)
     c4  27-point stencil 160^3, diag 26, off -1 + N(0, 0.01^2), x N(0,1)               (BF16)
     c5k64 / c5k256  m = n = 2^19, 32 nnz/row, vals N(0,1), B N(0,1) n x k              (FP32, BF16)
     paper12_E / paper13_E  the paper's own SpMV / SpMM inputs: 2^E rows x 2048 columns at density 0.01 (K = 4096)
@@ -283,6 +284,11 @@ def workload(name: str, scale_down: int = 0) -> Workload:
         e_gen = 34_140_000 >> (2 * s)
         A = rmat(scale, e_gen, 1003, relabel=True)
         return Workload("c3p", A, x=uniform_open_low(A.n, 1003, 10), dtypes=("f32",))
+    if name == "c3k64":
+        scale = 22 - 2 * s
+        e_gen = 34_140_000 >> (2 * s)
+        A = rmat(scale, e_gen, 1003)
+        return Workload("c3k64", A, B=normal(A.n * 64, 1003, 12), k=64, dtypes=("f32", "bf16"))
     if name == "c4":
         N = 160 >> s
         A = stencil27(N, 1004)

@@ -511,18 +511,32 @@ spmm_medium_row_kernel(int num_rows, const int* __restrict__ rows, int k, int ro
 // No chain is longer than C products plus one term per group or tile that a row spans.
 //   tile_row[t]  the list row that holds nonzero t * TILE, m for t * TILE >= nnz
 template <typename T, int VEC, int THREADS, int C>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 1536 / THREADS)
 spmm_flat_kernel(int m, int nnz, int k, int tiles, const int* __restrict__ row_ptr, const int* __restrict__ row_id,
                  const int* __restrict__ tile_row, const int* __restrict__ col_idx, const T* __restrict__ vals, const T* __restrict__ B,
                  T* __restrict__ Y, float* __restrict__ tile_carry, float* __restrict__ tile_tail, float alpha, float beta) {
   constexpr int LANES = 8, GROUPS = THREADS / LANES, KS = LANES * VEC, TILE = GROUPS * C, RB = TILE + 32;
   __shared__ int rp_s[RB];                       // row_ptr[r_lo .. r_lo + RB): the bounds of the tile's rows (what does not fit is read from global memory)
   __shared__ float head_s[GROUPS][KS], carry_s[GROUPS][KS];
+  __shared__ __align__(16) int col_s[TILE];      // the tile's (col, val) pairs, fetched once with coalesced 128-bit loads
+  __shared__ __align__(16) T val_s[TILE];
   grid_dependency_wait();
   const int slice = blockIdx.x / tiles, t = blockIdx.x - slice * tiles;
   const int p_lo = t * TILE, p_hi = min(nnz, p_lo + TILE);
   const int r_lo = __ldg(tile_row + t);
   const int r_hi = min(__ldg(tile_row + t + 1), m - 1);
+  {
+    const int nnz4 = nnz & ~3;
+    for (int i = threadIdx.x * 4; i < p_hi - p_lo; i += THREADS * 4) {
+      const int p = p_lo + i;
+      if (p + 4 <= nnz4) {
+        *(int4*)(col_s + i) = ld_stream_i4(col_idx + p);
+        sts_vals4(val_s, i, vals, p);
+      } else {
+        for (int u = 0; u < 4 && p + u < p_hi; ++u) { col_s[i + u] = __ldg(col_idx + p + u); val_s[i + u] = __ldg(vals + p + u); }
+      }
+    }
+  }
   for (int j = threadIdx.x; j < RB && r_lo + j <= m; j += THREADS) rp_s[j] = __ldg(row_ptr + r_lo + j);
   __syncthreads();
   auto bound = [&](int r) { const int j = r - r_lo; return j < RB ? rp_s[j] : __ldg(row_ptr + r); };
@@ -552,20 +566,15 @@ spmm_flat_kernel(int m, int nnz, int k, int tiles, const int* __restrict__ row_p
 #pragma unroll
       for (int j = 0; j < VEC; ++j) acc[j] = 0.0f;
     };
-    const int nnz4 = nnz & ~3;
-    // the chunk is walked four nonzeros at a time whatever rows they belong to (c0 is a multiple of four): the loads stay
-    // vectorised and four reads of B are in flight even where the rows are one or two nonzeros long
+    // the chunk is walked four nonzeros at a time whatever rows they belong to (c0 is a multiple of four): the pairs come from
+    // shared memory and four reads of B are in flight even where the rows are one or two nonzeros long
     for (int q = c0; q < c1; q += 4) {
       int c[4]; float v[4];
-      if (q + 4 <= nnz4) ld_a4(col_idx, vals, q, c, v);
-      else {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) { const bool in = q + u < c1; c[u] = in ? __ldg(col_idx + q + u) : 0; v[u] = in ? to_f32(__ldg(vals + q + u)) : 0.0f; }
-      }
+      lds_a4(col_s, val_s, q - p_lo, c, v);
       raw_t bv[4];
       if (active) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) bv[u] = RawVec<T, VEC>::ld(Bc + (long long)c[u] * k);   // past c1 the column is one of the chunk's own or 0: a valid row of B
+        for (int u = 0; u < 4; ++u) bv[u] = RawVec<T, VEC>::ld(Bc + (long long)(q + u < c1 ? c[u] : c[0]) * k);   // past the chunk's end: any valid row of B
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {

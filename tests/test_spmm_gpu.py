@@ -116,7 +116,7 @@ def test_spmm_column_equals_spmv(dtype):
     assert_within(Y, Y_ref, S, dtype)
 
 
-@pytest.mark.parametrize("name", ["c5k64", "c5k256"])
+@pytest.mark.parametrize("name", ["c5k64", "c5k256", "c3k64"])
 def test_workload_scaled(name):
     w = gen.workload(name, scale_down=3)
     for dtype in w.dtypes:
@@ -131,6 +131,20 @@ def test_workload_full_size_every_entry_k64():
         Y, Y_ref, S = run_spmm(w.A, w.B, w.k, None, w.alpha, w.beta, dtype)
         assert_within(Y, Y_ref, S, dtype, what="c5k64 %s full, all rows" % dtype)
         del Y, Y_ref, S
+
+
+def test_power_law_spmm_full_size_sampled_rows():
+    """The R-MAT matrix of the power-law workload times a dense n x 64 B at full size (the nnz-balanced kernel): 8192 sampled
+    rows plus the 64 longest rows, the first and the last row, and a run of rows around the longest one."""
+    w = gen.workload("c3k64")
+    L = np.diff(w.A.row_ptr)
+    rng = np.random.default_rng(13)
+    longest = np.argsort(L)[-64:]
+    rows = np.unique(np.concatenate([[0, w.A.m - 1], longest, np.arange(max(0, longest[-1] - 8), min(w.A.m, longest[-1] + 8)),
+                                     rng.integers(0, w.A.m, 8192)])).astype(np.int64)
+    for dtype in w.dtypes:
+        Y, Y_ref, S = run_spmm(w.A, w.B, w.k, None, w.alpha, w.beta, dtype, rows=rows)
+        assert_within(Y, Y_ref, S, dtype, what="c3k64 %s full" % dtype)
 
 
 def test_workload_full_size_sampled_rows_k256():
