@@ -39,8 +39,9 @@
  *    nothing; a device that is not compute capability 10.x returns B200SP_ERR_ARCH; a failing CUDA
  *    call returns B200SP_ERR_CUDA and its message is kept for b200sp_last_cuda_error().
  *  - Device memory the library needs (plan scratch, the staging buffers of the "host" entry
- *    points) comes from a stream-ordered memory pool of its own, one per device, created at first
- *    use.  The pool keeps up to 1 GiB of freed memory for the next call (option "pool_keep_mb",
+ *    points, and for SpMM on matrices with very uneven rows a few bytes per 1024 nonzeros and dense
+ *    column of per-call scratch, taken and returned in the order of `stream`) comes from a
+ *    stream-ordered memory pool of its own, one per device, created at first use.  The pool keeps up to 1 GiB of freed memory for the next call (option "pool_keep_mb",
  *    read when the pool is created); b200sp_cache_clear hands all unused pool memory back.
  *  - There is no CPU fallback: without a B200 the compute entry points fail.
  */
@@ -109,7 +110,10 @@ int spmm_csr(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_pt
  * The plan pass depends on the sparsity pattern's row structure only (row_ptr): it computes the
  * row-length statistics and bins, chooses the kernels, and computes the nnz-balanced split points
  * (a merge-path search over rows + nonzeros) and the lists of rows of 129-1024 and of more than 1024 nonzeros that
- * SpMM treats separately, all on the device.
+ * SpMM treats separately, all on the device.  From the same statistics it decides whether SpMM gives every row to a
+ * group of eight lanes (even rows) or cuts the nonzeros into equal chunks whatever rows they belong to (uneven rows:
+ * many empty rows, or a share of the nonzeros in rows of more than 128); the list of non-empty rows that the second
+ * form needs is built on the first SpMM call, in stream order.
  * When the row statistics select the row-direct SpMV kernel, the first b200sp_spmv / spmv_csr call with a given
  * col_idx additionally samples how local the columns are (one small kernel and one synchronisation of the stream)
  * and falls back to the merge-tile kernel for matrices with scattered columns.
