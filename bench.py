@@ -63,7 +63,7 @@ def measured_peaks():
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML (read-only) from a background thread."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.004):
         self.samples = []
         self.period = period_s
         self._stop = threading.Event()
@@ -106,7 +106,12 @@ class ClockSampler:
     def summary(self, t0: float, t1: float):
         if not self.ok:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml unavailable"]}
-        sel = [s for s in self.samples if t0 <= s[0] <= t1] or self.samples
+        sel = [s for s in self.samples if t0 <= s[0] <= t1]
+        inside = len(sel)
+        if not sel:                      # a region shorter than the sampling period: the two samples that bracket it, and say so
+            before = [s for s in self.samples if s[0] < t0][-1:]
+            after = [s for s in self.samples if s[0] > t1][:1]
+            sel = before + after
         names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
                  0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
         seen = 0
@@ -115,7 +120,7 @@ class ClockSampler:
         reasons = [n for bit, n in names.items() if seen & bit]
         clk = sorted(s[1] for s in sel)
         return {"sm_mhz": clk[len(clk) // 2] if clk else None, "sm_max_mhz": self.max_sm, "reasons": reasons,
-                "samples": len(sel)}
+                "samples": inside, "bracketing_samples": len(sel) - inside if not inside else 0}
 
 
 # ------------------------------------------------------------------------------------------ helpers
@@ -834,7 +839,7 @@ def main():
                     "algorithmic_bytes": r["algorithmic_bytes"], "nnz": r["nnz"], "copies": r["copies"],
                     "plan_ms_first_call": round(r["plan_ms_first_call"], 3),
                     "cusparse_ms": round(r["cusparse_ms"], 5) if isinstance(r["cusparse_ms"], float) else r["cusparse_ms"]}
-                ck = sampler.summary(r["t0"], r["t1"])      # SM clock and throttle reasons while THIS workload was timed (long SpMM kernels reach the power cap)
+                ck = sampler.summary(r["t0"], r["t1"])      # SM clock and throttle reasons sampled while THIS workload was timed
                 extras["%s_%s" % (name, dt)]["clocks"] = {"sm_mhz": ck.get("sm_mhz"), "reasons": ck.get("reasons"), "samples": ck.get("samples")}
                 if name == "c1":   # launch-latency regime: per-call device time from a CUDA graph, and the floors on the same box
                     extras["c1_f32"].update(latency_floor(r["_call"], r["_sets"], dev, r["algorithmic_bytes"]))
