@@ -324,6 +324,9 @@ def latency_floor(call, sets, dev, nbytes):
         out["graph_replay_us_per_call"] = round(graph_us(lambda i: call(sets[i % len(sets)], torch.cuda.current_stream())), 3)
         out["empty_kernel_us"] = round(graph_us(lambda i: b200sp.b200sp_probe_gather(tab, 1024, 0, sink, torch.cuda.current_stream())), 3)
         out["copy_same_bytes_us"] = round(graph_us(lambda i: dst.copy_(src)), 3)
+        # the same copy over as many independent buffers as the SpMV calls rotate over, so that it too reads cold lines
+        srcs = [torch.zeros(nbytes // 8, dtype=torch.float32, device=dev) for _ in range(len(sets))]
+        out["copy_same_bytes_cold_us"] = round(graph_us(lambda i: dst.copy_(srcs[i % len(srcs)])), 3)
     except Exception as ex:  # pragma: no cover
         out["latency_floor_error"] = repr(ex)
     return out

@@ -54,6 +54,11 @@ extern "C" {
  *   "bstage_nnz"     nonzeros of A per CTA that kernel aims for: 16384, 65536, 131072 (default) or 524288
  *   "bstage_stage_a" 1 = its warps first copy their rows' (col, val) pairs into shared-memory buffers of their own (default),
  *                    0 = the pairs are read from global memory inside the row loop
+ *   "bstage_quads"   1 = that kernel runs on a copy of A made once per call (default): every row padded to whole groups of
+ *                    four (byte offset, FP32 value) pairs and ordered so that neighbouring rows read different halves of a
+ *                    shared-memory bank line; a warp fetches its rows' groups with one bulk copy per array.  The copy takes
+ *                    8 * (nnz + 3 m + 8) bytes from the library's pool for the duration of the call.
+ *                    0 = the kernel walks the caller's col_idx / vals
  *   "x_l2_window"    1 = pin the gathered operand (x, or B for SpMM) in L2 with a per-launch access-policy window, 0 = off
  *                    (default; the measured effect is recorded with the benchmarks)
  *  launch

@@ -586,6 +586,7 @@ static int option_access(const char* name, int* get, const int* set) {
       {"bstage_threads", &g_opt.bstage_threads, false, {256, 512, 1024}, 0, 0},
       {"bstage_nnz", &g_opt.bstage_nnz, false, {16384, 65536, 131072, 524288}, 0, 0},
       {"bstage_stage_a", &g_opt.bstage_stage_a, true, {}, 0, 0},
+      {"bstage_quads", &g_opt.bstage_quads, true, {}, 0, 0},
       {"x_l2_window", &g_opt.x_l2_window, true, {}, 0, 0},
       {"pdl", &g_opt.pdl, true, {}, 0, 0},
       {"debug_no_copies", &g_opt.debug_no_copies, true, {}, 0, 0},

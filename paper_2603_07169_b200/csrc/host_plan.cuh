@@ -20,13 +20,14 @@ constexpr size_t kCacheCap = 1024;
 int plan_free(b200sp_plan* p, bool stream_ordered = false, cudaStream_t stream = nullptr) {
   if (!p) return B200SP_OK;
   int rc = B200SP_OK;
-  if (p->block || p->cuts_block || p->compact_block || p->flat_tile_row) {
+  if (p->block || p->cuts_block || p->compact_block || p->flat_tile_row || p->quad_block) {
     cudaError_t e = cudaSuccess;
     if (stream_ordered) {
       if (p->block) e = cudaFreeAsync(p->block, stream);
       if (p->cuts_block && e == cudaSuccess) e = cudaFreeAsync(p->cuts_block, stream);
       if (p->compact_block && e == cudaSuccess) e = cudaFreeAsync(p->compact_block, stream);
       if (p->flat_tile_row && e == cudaSuccess) e = cudaFreeAsync(p->flat_tile_row, stream);
+      if (p->quad_block && e == cudaSuccess) e = cudaFreeAsync(p->quad_block, stream);
     } else {
       int cur = 0;
       e = cudaGetDevice(&cur);
@@ -36,6 +37,7 @@ int plan_free(b200sp_plan* p, bool stream_ordered = false, cudaStream_t stream =
       if (e == cudaSuccess && p->cuts_block) e = cudaFree(p->cuts_block);
       if (e == cudaSuccess && p->compact_block) e = cudaFree(p->compact_block);
       if (e == cudaSuccess && p->flat_tile_row) e = cudaFree(p->flat_tile_row);
+      if (e == cudaSuccess && p->quad_block) e = cudaFree(p->quad_block);
       if (cur != p->device) cudaSetDevice(cur);
     }
     if (e != cudaSuccess) rc = cuda_fail(e, "freeing a plan");

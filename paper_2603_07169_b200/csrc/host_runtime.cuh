@@ -57,6 +57,7 @@ struct Options {
   int bstage_threads = 1024; // threads per CTA of that kernel (256, 512 or 1024)
   int bstage_nnz = 131072;   // nonzeros per CTA it aims for
   int bstage_stage_a = 1;  // 1 = that kernel's warps copy their rows' (col, val) pairs into shared-memory buffers of their own (default), 0 = read them from global memory
+  int bstage_quads = 1;    // 1 = that kernel runs on a copy of A re-laid once per call into padded quads ordered against bank conflicts (default), 0 = on the caller's CSR arrays
   int spmm_bstage = 1;     // 1 = hold the slice of B in shared memory when A has few columns (default), 0 = never
   int spmm_sliced = 1;     // 1 = k-sliced SpMM kernel (default), 0 = one pass over all of k
   int sub_lanes = 0;       // lanes per row of the sub-warp kernel (0 = from the mean row length)
@@ -259,6 +260,12 @@ struct b200sp_plan {
   const void* cuts_col_idx = nullptr;     // col_idx they were computed from
   int cuts_ranges = 0;                    // number of ranges they describe (0 = none computed)
   bool cols_sorted = false;               // every row's columns ascend
+  // processing order of the SpMM kernel with B in shared memory: rows of at most kLongRow nonzeros sorted by length, in blocks of quad_gpw
+  void* quad_block = nullptr;             // one pool block: row numbers, row lengths, block offsets (built on first use)
+  int32_t* quad_row = nullptr;            // quad_blocks * quad_gpw row numbers (-1 = unused slot)
+  int32_t* quad_len = nullptr;            // their lengths
+  int32_t* quad_pos = nullptr;            // quad_blocks + 1: where each block's quads start in the per-call copy of A
+  int quad_gpw = 0, quad_blocks = 0;
   const void* probed_key = nullptr;       // host entry points: the HOST col_idx that verdict belongs to
   bool cols_local = true;                 // its verdict: adjacent rows share most of their lines of x
 };

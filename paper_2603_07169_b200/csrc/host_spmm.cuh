@@ -4,6 +4,7 @@
 #include "host_spmv.cuh"
 #include "spmm_kernels.cuh"
 #include "spmm_bstage_kernels.cuh"
+#include "format_kernels.cuh"
 
 namespace {
 
@@ -92,6 +93,150 @@ int launch_spmm_bstage(b200sp_plan* p, int k, const int32_t* col_idx, const T* v
   return launch_smem(kernel, dim3((unsigned)(slices * row_chunks)), dim3(THREADS), smem, stream, nullptr, 0, dev, map, (int)I.m, (int)I.n,
                      k, row_chunks, rows_per_chunk, box_rows, (int)bslice, capw, p->row_ptr, col_idx, vals, Y, alpha, beta, dev->err_flag,
                      g_opt.spin_limit, g_opt.debug_no_copies);
+}
+
+// Exclusive scan of `count` ints in place; bsum: (count + kScanBlock - 1) / kScanBlock + 1 ints of scratch.  Three launches.
+int device_scan_in_place(int* data, long long count, int* bsum, cudaStream_t stream) {
+  const long long blocks = (count + kScanBlock - 1) / kScanBlock;
+  if (blocks < 1 || blocks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+  scan_block_sums_kernel<<<(unsigned)blocks, 256, 0, stream>>>(data, count, bsum);
+  plan_compact_scan_kernel<<<1, 1024, 0, stream>>>(bsum, (int)blocks);
+  scan_apply_kernel<<<(unsigned)blocks, 256, 0, stream>>>(data, count, bsum, data);
+  g_launches += 3;
+  CU(cudaGetLastError());
+  return B200SP_OK;
+}
+
+// The processing order of spmm_bstage_quads_kernel (see plan_kernels.cuh), built once per plan and lane-group width, on the
+// device and in stream order: no synchronisation.  B200SP_ERR_UNSUPPORTED when the positions would not fit 32 bits.
+int plan_quad_order(b200sp_plan* p, int gpw, cudaStream_t stream, DeviceInfo* dev) {
+  static_assert(kLongRow == 1024, "quad_key() assumes rows of at most 1024 nonzeros");
+  if (p->quad_block && p->quad_gpw == gpw) return B200SP_OK;
+  const b200sp_plan_info_t& I = p->info;
+  const long long listed = I.m - p->num_long;
+  const long long blocks = (listed + gpw - 1) / gpw;
+  if ((I.nnz + 3 * I.m) / 4 + (long long)(kLongRow / 4 + 2) * gpw >= (1LL << 31) - 64 || blocks < 1) return B200SP_ERR_UNSUPPORTED;
+  if (p->quad_block) { CU(cudaFreeAsync(p->quad_block, stream)); p->quad_block = nullptr; p->quad_gpw = 0; }
+  long long rows_per_blk = (I.m + 65535) / 65536;
+  if (rows_per_blk < 256) rows_per_blk = 256;
+  rows_per_blk = (rows_per_blk + 31) / 32 * 32;
+  const long long nblk = (I.m + rows_per_blk - 1) / rows_per_blk;
+  const long long slots = blocks * gpw, table = (long long)kQuadKeys * nblk;
+  const long long scan_len = table > blocks + 1 ? table : blocks + 1;
+  auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+  const size_t o_row = 0, o_len = up((size_t)slots * 4), o_pos = o_len + up((size_t)slots * 4), keep = o_pos + up((size_t)(blocks + 1) * 4);
+  void* blk = nullptr;
+  void* tmp = nullptr;      // the histogram table and the scan's block sums: only needed while the order is built
+  int rc = pool_alloc(dev, &blk, keep, stream);
+  if (rc != B200SP_OK) return rc;
+  rc = pool_alloc(dev, &tmp, up((size_t)table * 4) + up((size_t)(scan_len / kScanBlock + 2) * 4), stream);
+  if (rc != B200SP_OK) { cudaFreeAsync(blk, stream); return rc; }
+  int* row_of = (int*)((char*)blk + o_row);
+  int* len_of = (int*)((char*)blk + o_len);
+  int* pos = (int*)((char*)blk + o_pos);
+  int* hist = (int*)tmp;
+  int* bsum = (int*)((char*)tmp + up((size_t)table * 4));
+  auto fail = [&](int code) { cudaFreeAsync(tmp, stream); cudaFreeAsync(blk, stream); return code; };
+#define CUQ(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail(cuda_fail(e_, #call)); } while (0)
+  CUQ(cudaMemsetAsync(row_of, 0xFF, (size_t)slots * 4, stream));      // unused slots: row -1, length 0
+  CUQ(cudaMemsetAsync(len_of, 0, (size_t)slots * 4, stream));
+  const unsigned grid = (unsigned)((nblk + 3) / 4);
+  quad_order_hist_kernel<<<grid, 128, 0, stream>>>(p->row_ptr, (int)I.m, (int)rows_per_blk, (int)nblk, hist);
+  g_launches++;
+  CUQ(cudaGetLastError());
+  rc = device_scan_in_place(hist, table, bsum, stream);
+  if (rc != B200SP_OK) return fail(rc);
+  quad_order_scatter_kernel<<<grid, 128, 0, stream>>>(p->row_ptr, (int)I.m, (int)rows_per_blk, (int)nblk, hist, row_of, len_of);
+  quad_order_block_quads_kernel<<<(unsigned)((blocks + 1 + 255) / 256), 256, 0, stream>>>(len_of, (int)blocks, gpw, pos);
+  g_launches += 2;
+  CUQ(cudaGetLastError());
+  rc = device_scan_in_place(pos, blocks + 1, bsum, stream);
+  if (rc != B200SP_OK) return fail(rc);
+  CUQ(cudaFreeAsync(tmp, stream));
+#undef CUQ
+  p->quad_block = blk;
+  p->quad_row = row_of;
+  p->quad_len = len_of;
+  p->quad_pos = pos;
+  p->quad_gpw = gpw;
+  p->quad_blocks = (int)blocks;
+  return B200SP_OK;
+}
+
+// The same with the rows in the plan's sorted order and A re-laid once per call into padded quads (spmm_bstage_prep_kernel),
+// which the main kernel's warps fetch with bulk copies; rows longer than kLongRow by spmm_long_row_kernel.
+template <typename T, int VEC, int LANES, int THREADS = 1024>
+int launch_spmm_bstage_quads(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const T* B, T* Y, float alpha, float beta,
+                             cudaStream_t stream, DeviceInfo* dev, EncodeTiledFn encode) {
+  const b200sp_plan_info_t& I = p->info;
+  constexpr int KS = LANES * VEC, ROW_BYTES = LANES * 16, GPW = 32 / LANES, WARPS = THREADS / 32;
+  const int box_rows = I.n < 256 ? (int)I.n : 256;
+  const int boxes = (int)((I.n + box_rows - 1) / box_rows);
+  const size_t bslice = (((size_t)boxes * box_rows * ROW_BYTES) + 127) & ~(size_t)127;
+  // what the slice of B leaves of the SM's shared memory is split among the warps as buffers for their blocks' quads (32 bytes each)
+  const size_t limit = (size_t)kSmemPerSm - 2048 - 32 * WARPS;
+  int capq = 0;
+  if (g_opt.bstage_stage_a && bslice < limit) {
+    const size_t quads = (limit - bslice) / WARPS / 32;
+    capq = (int)(quads > 2048 ? 2048 : quads) & ~1;
+    if (capq < 2 * GPW) capq = 0;
+  }
+  const size_t smem = bslice + (size_t)WARPS * capq * 32;
+  CUtensorMap map;
+  const cuuint64_t gdim[2] = {(cuuint64_t)k, (cuuint64_t)I.n};
+  const cuuint64_t gstride[1] = {(cuuint64_t)k * sizeof(T)};
+  const cuuint32_t box[2] = {(cuuint32_t)KS, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult cr = encode(&map, sizeof(T) == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<T*>(B), gdim,
+                             gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (cr != CUDA_SUCCESS) return B200SP_ERR_UNSUPPORTED;
+  int rc = plan_quad_order(p, GPW, stream, dev);
+  if (rc != B200SP_OK) return rc;
+  auto kernel = spmm_bstage_quads_kernel<T, VEC, LANES, THREADS>;
+  static bool configured[64] = {};
+  if (!configured[p->device]) {
+    CU(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerSm - 2048));
+    configured[p->device] = true;
+  }
+  const int slices = (k + KS - 1) / KS;
+  const int blocks = p->quad_blocks;
+  long long chunks = (I.nnz + g_opt.bstage_nnz - 1) / g_opt.bstage_nnz;   // a given number of nonzeros per CTA ...
+  const long long fill = (2LL * dev->sms + slices - 1) / slices;   // ... but at least two CTAs per SM over the grid
+  if (chunks < fill) chunks = fill;
+  if (chunks > (blocks + WARPS - 1) / WARPS) chunks = (blocks + WARPS - 1) / WARPS;   // a block per warp at least
+  if (chunks < 1) chunks = 1;
+  const int row_chunks = (int)chunks;
+  if ((long long)slices * row_chunks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+  rc = ensure_err_flag(dev);
+  if (rc != B200SP_OK) return rc;
+  // the per-call copy of A: at most the rows' quads plus (kLongRow / 4 + 2) * GPW of padding where the length changes along the list
+  const size_t entries = ((size_t)((I.nnz + 3 * I.m) / 4) + (size_t)(kLongRow / 4 + 2) * GPW) * 4 + 8;
+  void* scratch = nullptr;
+  rc = pool_alloc(dev, &scratch, entries * 8, stream);
+  if (rc != B200SP_OK) return rc;
+  int* qoff = (int*)scratch;
+  float* qval = (float*)scratch + entries;
+  const long long slots = (long long)blocks * GPW;
+  tl_pdl_kernel = true;
+  rc = launch(spmm_bstage_prep_kernel<T, ROW_BYTES>, dim3((unsigned)((slots * 8 + 255) / 256)), dim3(256), stream, nullptr, 0, dev, (int)slots, GPW,
+              (const int*)p->quad_row, (const int*)p->quad_pos, p->row_ptr, col_idx, vals, qoff, qval);
+  if (rc == B200SP_OK) {
+    tl_pdl_kernel = true;
+    rc = launch_smem(kernel, dim3((unsigned)(slices * row_chunks)), dim3(THREADS), smem, stream, nullptr, 0, dev, map, (int)I.n, k, row_chunks,
+                     blocks, box_rows, (int)bslice, capq, (const int*)p->quad_row, (const int*)p->quad_len, (const int*)p->quad_pos,
+                     (const int*)qoff, (const float*)qval, Y, alpha, beta, dev->err_flag, g_opt.spin_limit, g_opt.debug_no_copies);
+  }
+  const cudaError_t e = cudaFreeAsync(scratch, stream);
+  if (e != cudaSuccess && rc == B200SP_OK) rc = cuda_fail(e, "cudaFreeAsync");
+  if (rc == B200SP_OK && p->num_long > 0) {
+    const long long ctas = (long long)((k + 8 * VEC - 1) / (8 * VEC)) * p->num_long;
+    if (ctas >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
+    tl_pdl_kernel = true;
+    rc = launch(spmm_long_row_kernel<T, VEC, kSpmmThreads>, dim3((unsigned)ctas), dim3(kSpmmThreads), stream, nullptr, 0, dev, k, p->num_long,
+                (const int*)p->long_rows, p->row_ptr, col_idx, vals, B, Y, alpha, beta);
+  }
+  return rc;
 }
 
 // Column ranges for the k-sliced kernel: how many, and the per-row cut positions (computed once per col_idx; one small
@@ -212,19 +357,25 @@ int run_spmm(b200sp_plan* p, int k, const int32_t* col_idx, const T* vals, const
     EncodeTiledFn encode = tensor_map_encoder();
     if (encode && n_pad * 32 <= budget) {
       int rc;
-      if (g_opt.bstage_threads == 256) {
-        if (n_pad * 128 <= budget) rc = launch_spmm_bstage<T, VEC, 8, 256>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
-        else if (n_pad * 64 <= budget) rc = launch_spmm_bstage<T, VEC, 4, 256>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
-        else rc = launch_spmm_bstage<T, VEC, 2, 256>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
-      } else if (g_opt.bstage_threads == 512) {
-        if (n_pad * 128 <= budget) rc = launch_spmm_bstage<T, VEC, 8, 512>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
-        else if (n_pad * 64 <= budget) rc = launch_spmm_bstage<T, VEC, 4, 512>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
-        else rc = launch_spmm_bstage<T, VEC, 2, 512>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
-      } else {
-        if (n_pad * 128 <= budget) rc = launch_spmm_bstage<T, VEC, 8>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
-        else if (n_pad * 64 <= budget) rc = launch_spmm_bstage<T, VEC, 4>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
-        else rc = launch_spmm_bstage<T, VEC, 2>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);
-      }
+#define B200SP_BSTAGE(FN)                                                                                                                  \
+  do {                                                                                                                                     \
+    if (g_opt.bstage_threads == 256) {                                                                                                     \
+      if (n_pad * 128 <= budget) rc = FN<T, VEC, 8, 256>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);                     \
+      else if (n_pad * 64 <= budget) rc = FN<T, VEC, 4, 256>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);                 \
+      else rc = FN<T, VEC, 2, 256>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);                                           \
+    } else if (g_opt.bstage_threads == 512) {                                                                                              \
+      if (n_pad * 128 <= budget) rc = FN<T, VEC, 8, 512>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);                     \
+      else if (n_pad * 64 <= budget) rc = FN<T, VEC, 4, 512>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);                 \
+      else rc = FN<T, VEC, 2, 512>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);                                           \
+    } else {                                                                                                                               \
+      if (n_pad * 128 <= budget) rc = FN<T, VEC, 8, 1024>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);                    \
+      else if (n_pad * 64 <= budget) rc = FN<T, VEC, 4, 1024>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);                \
+      else rc = FN<T, VEC, 2, 1024>(p, k, col_idx, vals, B, Y, alpha, beta, stream, dev, encode);                                          \
+    }                                                                                                                                      \
+  } while (0)
+      if (g_opt.bstage_quads) B200SP_BSTAGE(launch_spmm_bstage_quads);
+      else B200SP_BSTAGE(launch_spmm_bstage);
+#undef B200SP_BSTAGE
       if (rc != B200SP_ERR_UNSUPPORTED) return rc;   // unsupported shape for the tensor map: fall through to the sliced kernel
     }
   }

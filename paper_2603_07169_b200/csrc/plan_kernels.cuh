@@ -177,6 +177,78 @@ __global__ void __launch_bounds__(256) plan_row_lists_kernel(const int* __restri
   }
 }
 
+// ---- processing order of the SpMM kernel that keeps a slice of B in shared memory --------------------------------
+// That kernel gives a lane group one row at a time and a warp `gpw` rows per step, so a step lasts as long as its
+// longest row, and lane groups whose rows differ in length by less than four still part ways in the last, partly filled
+// group of four nonzeros.  The rows of at most kLongRow nonzeros are therefore sorted by their length (0 .. kLongRow),
+// longest first, with a stable counting sort in three passes: per-block histograms
+// (one warp per block of `rows_per_blk` consecutive rows), an exclusive scan of the (key, block) table, and a
+// scatter in which a warp walks its rows in order, so that equal keys keep their row order.  Integer work only.
+constexpr int kQuadKeys = 1024 + 1;   // kLongRow + 1
+
+__device__ __forceinline__ int quad_key(int len) { return len > 1024 ? -1 : kQuadKeys - 1 - len; }
+
+__global__ void __launch_bounds__(128) quad_order_hist_kernel(const int* __restrict__ row_ptr, int m, int rows_per_blk, int nblk,
+                                                              int* __restrict__ hist) {
+  __shared__ int s_hist[4][kQuadKeys];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int blk = blockIdx.x * 4 + warp;
+  for (int j = lane; j < kQuadKeys; j += 32) s_hist[warp][j] = 0;
+  __syncwarp();
+  if (blk < nblk) {
+    const long long r0 = (long long)blk * rows_per_blk;
+    const long long r1 = min((long long)m, r0 + rows_per_blk);
+    for (long long r = r0 + lane; r < r1; r += 32) {
+      const int key = quad_key(__ldg(row_ptr + r + 1) - __ldg(row_ptr + r));
+      if (key >= 0) atomicAdd(&s_hist[warp][key], 1);
+    }
+    __syncwarp();
+    for (int j = lane; j < kQuadKeys; j += 32) hist[(long long)j * nblk + blk] = s_hist[warp][j];
+  }
+}
+
+// offset: the scanned table.  row_of / len_of: the sorted list (slots past its end are preset by the caller).
+__global__ void __launch_bounds__(128) quad_order_scatter_kernel(const int* __restrict__ row_ptr, int m, int rows_per_blk, int nblk,
+                                                                 const int* __restrict__ offset, int* __restrict__ row_of,
+                                                                 int* __restrict__ len_of) {
+  __shared__ int s_next[4][kQuadKeys];
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int blk = blockIdx.x * 4 + warp;
+  if (blk >= nblk) return;
+  for (int j = lane; j < kQuadKeys; j += 32) s_next[warp][j] = offset[(long long)j * nblk + blk];
+  __syncwarp();
+  const long long r0 = (long long)blk * rows_per_blk;
+  const long long r1 = min((long long)m, r0 + rows_per_blk);
+  for (long long rb = r0; rb < r1; rb += 32) {
+    const long long r = rb + lane;
+    int len = 0, key = -1 - lane;            // lanes without a row get keys of their own
+    if (r < r1) {
+      len = __ldg(row_ptr + r + 1) - __ldg(row_ptr + r);
+      const int kq = quad_key(len);
+      if (kq >= 0) key = kq;
+    }
+    const unsigned peers = __match_any_sync(FULL, key);
+    const int rank = __popc(peers & ((1u << lane) - 1u));
+    int base = 0;
+    if (key >= 0) base = s_next[warp][key];
+    __syncwarp();
+    if (key >= 0 && rank == 0) s_next[warp][key] = base + __popc(peers);
+    __syncwarp();
+    if (key >= 0) {
+      row_of[base + rank] = (int)r;
+      len_of[base + rank] = len;
+    }
+  }
+}
+
+// quads[b] = quads of block b of `gpw` list slots: gpw times those of its first (longest) row; quads[blocks] = 0.
+__global__ void __launch_bounds__(256) quad_order_block_quads_kernel(const int* __restrict__ len_of, int blocks, int gpw, int* __restrict__ quads) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b > blocks) return;
+  quads[b] = b < blocks ? ((len_of[(long long)b * gpw] + 3) >> 2) * gpw : 0;
+}
+
 // Column-locality probe for matrices with short rows: for `samples` evenly spaced pairs of adjacent rows (r, r + 1),
 // counts the entries of row r + 1 whose 128-byte line of x (32 four-byte entries) is also touched by row r.
 // Banded / stencil / mesh matrices score near 1, matrices with random columns near 0.  out[0] += hits, out[1] += entries.

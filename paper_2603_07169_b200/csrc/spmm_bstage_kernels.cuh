@@ -32,6 +32,23 @@ template <typename T> struct RawFromSmem;
 template <> struct RawFromSmem<float> { typedef float4 type; };
 template <> struct RawFromSmem<bf16_t> { typedef uint4 type; };
 
+// 128-bit loads from a 32-bit shared-memory address (no generic-address arithmetic in the row loops)
+__device__ __forceinline__ float4 lds128(unsigned addr, const float4*) {
+  float4 r;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "r"(addr));
+  return r;
+}
+__device__ __forceinline__ uint4 lds128(unsigned addr, const uint4*) {
+  uint4 r;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+  return r;
+}
+__device__ __forceinline__ int4 lds128(unsigned addr, const int4*) {
+  int4 r;
+  asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+  return r;
+}
+
 // Dynamic shared memory: [ slice of B: bslice_bytes | per warp: (capw + 4) ints, (capw + 4) values ]; capw + 4 is a multiple of 8.
 template <typename T, int VEC, int LANES, int THREADS>
 __global__ void __launch_bounds__(THREADS)
@@ -158,6 +175,250 @@ spmm_bstage_kernel(const __grid_constant__ CUtensorMap tmapB, int m, int n, int 
       }
       VecLoad<T, VEC>::st(yp, out);
     }
+  }
+}
+
+// ---- the same product with A re-laid once per call ------------------------------------------------------------
+//
+// In spmm_bstage_kernel above every (row, slice) pair walks the row's (col, val) pairs again, and the L1 data pipe
+// that kernel is bound by spends 40 % of its wavefronts on things other than the reads of B: single steps up to the
+// first multiple of four, the copies of the pairs into the per-warp buffers, and bank conflicts between the two
+// (four) lane groups of a quarter warp whose rows of the slice fall into the same half (quarter) of a 128-byte bank
+// line; a quarter of its lanes idle because the rows of a warp's step differ in length.  All of this depends only
+// on A, so it is dealt with once per plan and once per call instead of once per slice:
+//
+// * per plan (quad_order_* kernels): the rows of at most kLongRow nonzeros sorted by length, longest first, in blocks
+//   of GPW = 32 / LANES list slots: the rows of a block -- one step of a warp -- are equally long, except where the
+//   length changes along the list; a quad is a group of four nonzeros;
+// * per call (spmm_bstage_prep_kernel): A copied into two arrays of quads (four byte offsets col * ROW_BYTES; four
+//   FP32 values).  Quad i of the row in slot g of block b sits at quad position pos[b] + i * GPW + g, so the GPW
+//   groups of a warp read GPW consecutive quads at every step: one wavefront.  The last quad of a row is padded with
+//   (0, 0.0f), which is never multiplied.  Inside a row the entries are ordered by (col - g) mod G, G = 128 / ROW_BYTES
+//   rows of the slice per bank line: the groups of a quarter warp own neighbouring slots, so while the classes of
+//   their rows are equally long they read different parts of the bank line.  (The order of a row's products
+//   changes; each lane still adds them in one fixed order.)
+//
+// spmm_bstage_quads_kernel then needs no alignment steps and gets a block's quads with ONE bulk copy per array (TMA,
+// on a barrier of the warp's own, outside the LSU pipe).
+// Rows longer than kLongRow are left to spmm_long_row_kernel.
+template <typename T, int ROW_BYTES>
+__global__ void __launch_bounds__(256)
+spmm_bstage_prep_kernel(int slots, int gpw, const int* __restrict__ quad_row, const int* __restrict__ quad_pos,
+                        const int* __restrict__ row_ptr, const int* __restrict__ col_idx, const T* __restrict__ vals,
+                        int* __restrict__ qoff, float* __restrict__ qval) {
+  constexpr int G = 128 / ROW_BYTES;
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  grid_dependency_wait();
+  const int lane = threadIdx.x & 31, sub = lane & 7, first = lane & ~7;   // eight lanes per row, four rows per warp
+  const long long slot = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
+  int rs = 0, re = 0, g = 0;
+  long long base = 0;       // entry index of quad 0 of this row
+  if (slot < slots) {
+    const int row = __ldg(quad_row + slot);
+    const int b = (int)(slot / gpw);
+    g = (int)(slot - (long long)b * gpw);
+    if (row >= 0) { rs = __ldg(row_ptr + row); re = __ldg(row_ptr + row + 1); }
+    base = ((long long)__ldg(quad_pos + b) + g) * 4;
+  }
+  const int len = re - rs;
+  const int stride = gpw * 4;                 // entries from one quad of the row to the next
+  const int gc = g & (G - 1);
+  int start[G];    // where class j begins inside the row
+  {
+    int cnt[G];
+#pragma unroll
+    for (int j = 0; j < G; ++j) cnt[j] = 0;
+    if (G > 1) {
+      for (int p = rs + sub; p < re; p += 8) {
+        const int cls = (__ldg(col_idx + p) - gc) & (G - 1);
+#pragma unroll
+        for (int j = 0; j < G; ++j) cnt[j] += (cls == j);
+      }
+#pragma unroll
+      for (int j = 0; j < G; ++j) {
+        cnt[j] += __shfl_xor_sync(FULL, cnt[j], 1);
+        cnt[j] += __shfl_xor_sync(FULL, cnt[j], 2);
+        cnt[j] += __shfl_xor_sync(FULL, cnt[j], 4);
+      }
+    }
+    int run = 0;
+#pragma unroll
+    for (int j = 0; j < G; ++j) { start[j] = run; run += cnt[j]; }
+  }
+  int longest = len;    // the ballots below need every lane of the warp: all four rows walk as far as the longest
+  longest = max(longest, __shfl_xor_sync(FULL, longest, 8));
+  longest = max(longest, __shfl_xor_sync(FULL, longest, 16));
+  for (int p0 = 0; p0 < longest; p0 += 8) {
+    const bool valid = p0 + sub < len;
+    int c = 0, cls = -1;
+    float v = 0.0f;
+    if (valid) {
+      c = __ldg(col_idx + rs + p0 + sub);
+      v = to_f32(__ldg(vals + rs + p0 + sub));
+      cls = (c - gc) & (G - 1);
+    }
+    int dest = 0;
+#pragma unroll
+    for (int j = 0; j < G; ++j) {
+      const unsigned bits = (__ballot_sync(FULL, cls == j) >> first) & 0xFFu;
+      if (cls == j) dest = start[j] + __popc(bits & ((1u << sub) - 1u));
+      start[j] += __popc(bits);
+    }
+    if (valid) {
+      const long long e = base + (long long)(dest >> 2) * stride + (dest & 3);
+      qoff[e] = c * ROW_BYTES;
+      qval[e] = v;
+    }
+  }
+  for (int d = len + sub; d < ((len + 3) & ~3); d += 8) {
+    const long long e = base + (long long)(d >> 2) * stride + (d & 3);
+    qoff[e] = 0;
+    qval[e] = 0.0f;
+  }
+}
+
+// acc += the products of one row's quads 0 .. (len + 3) / 4 - 1 with this lane's columns of the slice (at shared address bs).
+// SHARED: the quads sit in shared memory at addresses so / sv, else in global memory at qo / qv; consecutive quads of the
+// row are qstride quads apart.
+template <typename T, int VEC, bool SHARED>
+__device__ __forceinline__ void bstage_row_quads(const int4* __restrict__ qo, const float4* __restrict__ qv, unsigned so, unsigned sv, int qstride,
+                                                 int len, unsigned bs, float (&acc)[VEC], float (&tot)[VEC]) {
+  typedef typename RawVec<T, VEC>::type raw_t;
+  const int full = len >> 2, rem = len & 3;
+  int fold = 0;
+  for (int i = 0; i < full; ++i) {
+    if (++fold > kChainBlock / 4) {
+      fold = 1;
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) { tot[j] += acc[j]; acc[j] = 0.0f; }
+    }
+    const int4 o = SHARED ? lds128(so, (const int4*)nullptr) : __ldg(qo);
+    const float4 v = SHARED ? lds128(sv, (const float4*)nullptr) : __ldg(qv);
+    so += 16u * qstride; sv += 16u * qstride; qo += qstride; qv += qstride;
+    raw_t b[4];
+    b[0] = lds128(bs + o.x, (const raw_t*)nullptr); b[1] = lds128(bs + o.y, (const raw_t*)nullptr);
+    b[2] = lds128(bs + o.z, (const raw_t*)nullptr); b[3] = lds128(bs + o.w, (const raw_t*)nullptr);
+    RawVec<T, VEC>::fma_mixed(b[0], v.x, acc); RawVec<T, VEC>::fma_mixed(b[1], v.y, acc);
+    RawVec<T, VEC>::fma_mixed(b[2], v.z, acc); RawVec<T, VEC>::fma_mixed(b[3], v.w, acc);
+  }
+  if (rem) {   // the padded last quad: its padding is never multiplied (0 * inf would be NaN)
+    const int4 o = SHARED ? lds128(so, (const int4*)nullptr) : __ldg(qo);
+    const float4 v = SHARED ? lds128(sv, (const float4*)nullptr) : __ldg(qv);
+    RawVec<T, VEC>::fma_mixed(lds128(bs + o.x, (const raw_t*)nullptr), v.x, acc);
+    if (rem > 1) RawVec<T, VEC>::fma_mixed(lds128(bs + o.y, (const raw_t*)nullptr), v.y, acc);
+    if (rem > 2) RawVec<T, VEC>::fma_mixed(lds128(bs + o.z, (const raw_t*)nullptr), v.z, acc);
+  }
+}
+
+// Dynamic shared memory: [ slice of B: bslice_bytes | per warp: capq offset quads (16 B each), capq value quads ].
+// CTA `chunk` of a slice takes the blocks chunk, chunk + row_chunks, ... of the sorted list, its warps in turn, so that
+// every CTA gets the same mix of long and short rows.  A block of more than capq quads is read from global memory.
+// (Fetching the next block's quads a step ahead into a second half of the buffer was measured: no gain.)
+template <typename T, int VEC, int LANES, int THREADS>
+__global__ void __launch_bounds__(THREADS)
+spmm_bstage_quads_kernel(const __grid_constant__ CUtensorMap tmapB, int n, int k, int row_chunks, int blocks, int box_rows, int bslice_bytes,
+                         int capq, const int* __restrict__ quad_row, const int* __restrict__ quad_len, const int* __restrict__ quad_pos,
+                         const int* __restrict__ qoff, const float* __restrict__ qval, T* __restrict__ Y, float alpha, float beta,
+                         int* __restrict__ err, int spin_limit, int no_copies) {
+  constexpr int KS = LANES * VEC, ROW_BYTES = LANES * 16, GPW = 32 / LANES, WARPS = THREADS / 32;
+  constexpr unsigned FULL = 0xFFFFFFFFu;
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ __align__(8) unsigned long long wbar[WARPS];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int slice = blockIdx.x / row_chunks, chunk = blockIdx.x - slice * row_chunks;
+  const int col_base = slice * KS;
+  if (tid == 0) mbar_init(smem_addr(&bar), 1);
+  if (lane == 0) mbar_init(smem_addr(&wbar[warp]), 1);
+  mbar_init_fence();
+  __syncthreads();
+  grid_dependency_wait();   // nothing above touches global memory
+  if (tid == 0 && !no_copies) {   // no_copies (a test switch): nothing is issued, the wait below runs out with nothing in flight
+    const int boxes = (n + box_rows - 1) / box_rows;
+    mbar_arrive_expect_tx(smem_addr(&bar), (unsigned)boxes * (unsigned)box_rows * ROW_BYTES);   // rows past n are zero-filled and still counted
+    for (int b = 0; b < boxes; ++b)
+      tma_load_2d(smem_addr(smem + (size_t)b * box_rows * ROW_BYTES), &tmapB, col_base, b * box_rows, smem_addr(&bar));
+  }
+  const int gl = lane / LANES, l = lane % LANES;     // group inside the warp, lane inside the group
+  const int col0 = col_base + l * VEC;
+  const bool active = col0 < k;
+  const unsigned bs = smem_addr(smem) + l * 16;
+  const unsigned woff = smem_addr(smem) + bslice_bytes + warp * capq * 32;   // the warp's buffer: capq quads of offsets, then of values
+  const unsigned wval = woff + capq * 16;
+  const unsigned my_bar = smem_addr(&wbar[warp]);
+  const long long step_blocks = (long long)WARPS * row_chunks;
+  // one step's description, a value per lane: lanes < GPW the row number (m_row) and length (m_len) of their slot,
+  // lanes 30 / 31 the block's last / first quad position (m_len)
+  auto load_meta = [&](long long b, int& m_row, int& m_len) {
+    m_row = -1; m_len = 0;
+    if (b < blocks) {
+      if (lane < GPW) { m_row = __ldg(quad_row + b * GPW + lane); m_len = __ldg(quad_len + b * GPW + lane); }
+      else if (lane >= 30) m_len = __ldg(quad_pos + b + (31 - lane));
+    }
+  };
+  // the bulk copies that fetch a block's quads (lane 0 issues; the buffer must be free)
+  auto issue = [&](int q0, int nq) {
+    if (nq > 0 && nq <= capq && lane == 0) {
+      mbar_arrive_expect_tx(my_bar, (unsigned)nq * 32u);
+      bulk_copy_g2s(woff, qoff + (long long)q0 * 4, (unsigned)nq * 16u, my_bar);
+      bulk_copy_g2s(wval, qval + (long long)q0 * 4, (unsigned)nq * 16u, my_bar);
+    }
+  };
+  long long b = chunk + (long long)warp * row_chunks;
+  int row_cur, len_cur, row_next, len_next;
+  load_meta(b, row_cur, len_cur);
+  load_meta(b + step_blocks, row_next, len_next);
+  int q0_cur = __shfl_sync(FULL, len_cur, 31), nq_cur = __shfl_sync(FULL, len_cur, 30) - q0_cur;
+  issue(q0_cur, nq_cur);        // the copies of the first step overlap the fetch of the slice of B (no block: nq_cur is 0)
+  unsigned phase = 0;
+  const bool arrived = mbar_wait_bounded(smem_addr(&bar), 0, spin_limit);
+  if (!__syncthreads_and(arrived)) {
+    if (tid == 0) atomicExch(err, 1);
+    (void)mbar_wait_bounded(smem_addr(&bar), 0, spin_limit);   // bounded second chance for the copies in flight
+    if (nq_cur > 0 && nq_cur <= capq) (void)mbar_wait_bounded(my_bar, 0, spin_limit);
+    return;
+  }
+  for (; b < blocks; b += step_blocks) {
+    const int q0_next = __shfl_sync(FULL, len_next, 31), nq_next = __shfl_sync(FULL, len_next, 30) - q0_next;
+    const bool staged = nq_cur > 0 && nq_cur <= capq;
+    if (staged) {
+      const bool ok = mbar_wait_bounded(my_bar, phase, spin_limit);
+      if (!__all_sync(FULL, ok)) {
+        if (lane == 0) atomicExch(err, 1);
+        (void)mbar_wait_bounded(my_bar, phase, spin_limit);
+        return;
+      }
+      phase ^= 1u;
+    }
+    const int row = __shfl_sync(FULL, row_cur, gl), len = __shfl_sync(FULL, len_cur, gl);
+    float acc[VEC], tot[VEC];   // acc: the current block of at most kChainBlock products; tot: the sum of the completed blocks
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) { acc[j] = 0.0f; tot[j] = 0.0f; }
+    if (staged) {
+      bstage_row_quads<T, VEC, true>(nullptr, nullptr, woff + 16u * gl, wval + 16u * gl, GPW, len, bs, acc, tot);
+    } else {
+      bstage_row_quads<T, VEC, false>((const int4*)qoff + q0_cur + gl, (const float4*)qval + q0_cur + gl, 0u, 0u, GPW, len, bs, acc, tot);
+    }
+    __syncwarp();                       // every lane is done with the buffer: the next block's quads may land in it
+    issue(q0_next, nq_next);            // (past the last block nq_next is 0)
+    if (active && row >= 0) {
+      T* yp = Y + (long long)row * k + col0;
+      float out[VEC];
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) acc[j] += tot[j];
+      if (beta != 0.0f) {
+        float old[VEC];
+        VecLoad<T, VEC>::ld_plain(yp, old);
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) out[j] = alpha * acc[j] + beta * old[j];
+      } else {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) out[j] = alpha * acc[j];
+      }
+      VecLoad<T, VEC>::st(yp, out);
+    }
+    row_cur = row_next; len_cur = len_next; q0_cur = q0_next; nq_cur = nq_next;
+    load_meta(b + 2 * step_blocks, row_next, len_next);
   }
 }
 
