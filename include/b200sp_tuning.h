@@ -51,13 +51,15 @@ extern "C" {
  *   "sub_lanes"      least number of lanes per row of the sub-warp kernel (1..32, power of two), 0 = from the mean row
  *                    length (default); more lanes are used where a lane would otherwise add more than 128 products
  *   "bstage_threads" threads per CTA of the SpMM kernel with B in shared memory: 256, 512 or 1024 (default)
- *   "bstage_nnz"     nonzeros of A per CTA that kernel aims for: 16384, 65536, 131072 (default) or 524288
+ *   "bstage_nnz"     nonzeros of A per CTA that kernel aims for: 16384, 65536, 131072 or 524288; 0 (default) = chosen per
+ *                    call so that the grid fills whole rounds of one CTA per SM ("bstage_quads" = 0: 131072)
  *   "bstage_stage_a" 1 = its warps first copy their rows' (col, val) pairs into shared-memory buffers of their own (default),
  *                    0 = the pairs are read from global memory inside the row loop
  *   "bstage_quads"   1 = that kernel runs on a copy of A made once per call (default): every row padded to whole groups of
- *                    four (byte offset, FP32 value) pairs and ordered so that neighbouring rows read different halves of a
- *                    shared-memory bank line; a warp fetches its rows' groups with one bulk copy per array.  The copy takes
- *                    8 * (nnz + 3 m + 8) bytes from the library's pool for the duration of the call.
+ *                    four (16-bit offset, value) pairs and ordered so that neighbouring rows read different halves of a
+ *                    shared-memory bank line, the rows taken in order of length (an order built once per plan, 8 m bytes);
+ *                    a warp fetches its rows' groups with one bulk copy per array.  The copy takes about
+ *                    (2 + bytes per value) * (nnz + 3 m) bytes from the library's pool for the duration of the call.
  *                    0 = the kernel walks the caller's col_idx / vals
  *   "x_l2_window"    1 = pin the gathered operand (x, or B for SpMM) in L2 with a per-launch access-policy window, 0 = off
  *                    (default; the measured effect is recorded with the benchmarks)

@@ -584,7 +584,7 @@ static int option_access(const char* name, int* get, const int* set) {
       {"uni_ctas", &g_opt.uni_ctas, false, {0, 1, 2, 4, 8}, 0, 0},
       {"sub_lanes", &g_opt.sub_lanes, false, {0, 1, 2, 4, 8, 16, 32}, 0, 0},
       {"bstage_threads", &g_opt.bstage_threads, false, {256, 512, 1024}, 0, 0},
-      {"bstage_nnz", &g_opt.bstage_nnz, false, {16384, 65536, 131072, 524288}, 0, 0},
+      {"bstage_nnz", &g_opt.bstage_nnz, false, {0, 16384, 65536, 131072, 524288}, 0, 0},
       {"bstage_stage_a", &g_opt.bstage_stage_a, true, {}, 0, 0},
       {"bstage_quads", &g_opt.bstage_quads, true, {}, 0, 0},
       {"x_l2_window", &g_opt.x_l2_window, true, {}, 0, 0},

@@ -55,7 +55,7 @@ struct Options {
   int merge_items = 2048; // merge items per tile (1024, 2048 or 4096)
   int merge_threads = 128; // threads per CTA of the one-tile-per-CTA merge kernel (128 or 256)
   int bstage_threads = 1024; // threads per CTA of that kernel (256, 512 or 1024)
-  int bstage_nnz = 131072;   // nonzeros per CTA it aims for
+  int bstage_nnz = 0;        // nonzeros per CTA it aims for; 0 = chosen so that the grid fills whole rounds of one CTA per SM (the kernel on the caller's CSR arrays: 131072)
   int bstage_stage_a = 1;  // 1 = that kernel's warps copy their rows' (col, val) pairs into shared-memory buffers of their own (default), 0 = read them from global memory
   int bstage_quads = 1;    // 1 = that kernel runs on a copy of A re-laid once per call into padded quads ordered against bank conflicts (default), 0 = on the caller's CSR arrays
   int spmm_bstage = 1;     // 1 = hold the slice of B in shared memory when A has few columns (default), 0 = never

@@ -79,7 +79,8 @@ int launch_spmm_bstage(b200sp_plan* p, int k, const int32_t* col_idx, const T* v
     configured[p->device] = true;
   }
   const int slices = (k + KS - 1) / KS;
-  long long chunks = (I.nnz + g_opt.bstage_nnz - 1) / g_opt.bstage_nnz;   // a given number of nonzeros per CTA ...
+  const int per_cta = g_opt.bstage_nnz > 0 ? g_opt.bstage_nnz : 131072;
+  long long chunks = (I.nnz + per_cta - 1) / per_cta;   // a given number of nonzeros per CTA ...
   const long long fill = (2LL * dev->sms + slices - 1) / slices;   // ... but at least two CTAs per SM over the grid
   if (chunks < fill) chunks = fill;
   if (chunks > I.m) chunks = I.m;
@@ -173,15 +174,17 @@ int launch_spmm_bstage_quads(b200sp_plan* p, int k, const int32_t* col_idx, cons
   const int box_rows = I.n < 256 ? (int)I.n : 256;
   const int boxes = (int)((I.n + box_rows - 1) / box_rows);
   const size_t bslice = (((size_t)boxes * box_rows * ROW_BYTES) + 127) & ~(size_t)127;
-  // what the slice of B leaves of the SM's shared memory is split among the warps as buffers for their blocks' quads (32 bytes each)
+  // what the slice of B leaves of the SM's shared memory is split among the warps as buffers for their blocks' quads
+  // (four 16-bit offsets and four values each)
+  constexpr size_t QUAD_BYTES = 8 + 4 * sizeof(T);
   const size_t limit = (size_t)kSmemPerSm - 2048 - 32 * WARPS;
   int capq = 0;
   if (g_opt.bstage_stage_a && bslice < limit) {
-    const size_t quads = (limit - bslice) / WARPS / 32;
+    const size_t quads = (limit - bslice) / WARPS / QUAD_BYTES;
     capq = (int)(quads > 2048 ? 2048 : quads) & ~1;
     if (capq < 2 * GPW) capq = 0;
   }
-  const size_t smem = bslice + (size_t)WARPS * capq * 32;
+  const size_t smem = bslice + (((size_t)WARPS * capq * QUAD_BYTES + 15) & ~(size_t)15);
   CUtensorMap map;
   const cuuint64_t gdim[2] = {(cuuint64_t)k, (cuuint64_t)I.n};
   const cuuint64_t gstride[1] = {(cuuint64_t)k * sizeof(T)};
@@ -201,22 +204,37 @@ int launch_spmm_bstage_quads(b200sp_plan* p, int k, const int32_t* col_idx, cons
   }
   const int slices = (k + KS - 1) / KS;
   const int blocks = p->quad_blocks;
-  long long chunks = (I.nnz + g_opt.bstage_nnz - 1) / g_opt.bstage_nnz;   // a given number of nonzeros per CTA ...
-  const long long fill = (2LL * dev->sms + slices - 1) / slices;   // ... but at least two CTAs per SM over the grid
-  if (chunks < fill) chunks = fill;
-  if (chunks > (blocks + WARPS - 1) / WARPS) chunks = (blocks + WARPS - 1) / WARPS;   // a block per warp at least
+  const long long most = (blocks + WARPS - 1) / WARPS;   // a block per warp at least
+  long long chunks;
+  if (g_opt.bstage_nnz > 0) {
+    chunks = (I.nnz + g_opt.bstage_nnz - 1) / g_opt.bstage_nnz;   // a given number of nonzeros per CTA ...
+    const long long fill = (2LL * dev->sms + slices - 1) / slices;   // ... but at least two CTAs per SM over the grid
+    if (chunks < fill) chunks = fill;
+  } else {
+    // One CTA per SM is resident and all CTAs take the same time (each gets the same mix of rows), so the kernel lasts
+    // ceil(CTAs / SMs) rounds of (nonzeros per CTA + the fetch of the slice of B, about 4096 nonzeros' worth): the chunk
+    // count with the smallest product, among those that leave a CTA at least 8192 nonzeros (or one chunk).
+    chunks = 1;
+    double best = 0.0;
+    for (long long c = 1; c <= 4096 && c <= most && (c == 1 || I.nnz / c >= 8192); ++c) {
+      const double rounds = (double)((slices * c + dev->sms - 1) / dev->sms);
+      const double cost = rounds * ((double)I.nnz / (double)c + 4096.0);
+      if (c == 1 || cost < best) { best = cost; chunks = c; }
+    }
+  }
+  if (chunks > most) chunks = most;
   if (chunks < 1) chunks = 1;
   const int row_chunks = (int)chunks;
   if ((long long)slices * row_chunks >= (1LL << 31)) return B200SP_ERR_UNSUPPORTED;
   rc = ensure_err_flag(dev);
   if (rc != B200SP_OK) return rc;
   // the per-call copy of A: at most the rows' quads plus (kLongRow / 4 + 2) * GPW of padding where the length changes along the list
-  const size_t entries = ((size_t)((I.nnz + 3 * I.m) / 4) + (size_t)(kLongRow / 4 + 2) * GPW) * 4 + 8;
+  const size_t entries = (((size_t)((I.nnz + 3 * I.m) / 4) + (size_t)(kLongRow / 4 + 2) * GPW) * 4 + 15) & ~(size_t)7;
   void* scratch = nullptr;
-  rc = pool_alloc(dev, &scratch, entries * 8, stream);
+  rc = pool_alloc(dev, &scratch, entries * (2 + sizeof(T)), stream);
   if (rc != B200SP_OK) return rc;
-  int* qoff = (int*)scratch;
-  float* qval = (float*)scratch + entries;
+  unsigned short* qoff = (unsigned short*)scratch;       // entries 16-bit offsets, then entries values (16-byte aligned: entries is a multiple of 8)
+  T* qval = (T*)((char*)scratch + entries * 2);
   const long long slots = (long long)blocks * GPW;
   tl_pdl_kernel = true;
   rc = launch(spmm_bstage_prep_kernel<T, ROW_BYTES>, dim3((unsigned)((slots * 8 + 255) / 256)), dim3(256), stream, nullptr, 0, dev, (int)slots, GPW,
@@ -225,7 +243,7 @@ int launch_spmm_bstage_quads(b200sp_plan* p, int k, const int32_t* col_idx, cons
     tl_pdl_kernel = true;
     rc = launch_smem(kernel, dim3((unsigned)(slices * row_chunks)), dim3(THREADS), smem, stream, nullptr, 0, dev, map, (int)I.n, k, row_chunks,
                      blocks, box_rows, (int)bslice, capq, (const int*)p->quad_row, (const int*)p->quad_len, (const int*)p->quad_pos,
-                     (const int*)qoff, (const float*)qval, Y, alpha, beta, dev->err_flag, g_opt.spin_limit, g_opt.debug_no_copies);
+                     (const unsigned short*)qoff, (const T*)qval, Y, alpha, beta, dev->err_flag, g_opt.spin_limit, g_opt.debug_no_copies);
   }
   const cudaError_t e = cudaFreeAsync(scratch, stream);
   if (e != cudaSuccess && rc == B200SP_OK) rc = cuda_fail(e, "cudaFreeAsync");

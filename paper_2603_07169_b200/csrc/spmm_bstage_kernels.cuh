@@ -43,6 +43,11 @@ __device__ __forceinline__ uint4 lds128(unsigned addr, const uint4*) {
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
   return r;
 }
+__device__ __forceinline__ uint2 lds64(unsigned addr) {
+  uint2 r;
+  asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(r.x), "=r"(r.y) : "r"(addr));
+  return r;
+}
 __device__ __forceinline__ int4 lds128(unsigned addr, const int4*) {
   int4 r;
   asm volatile("ld.shared.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
@@ -190,10 +195,10 @@ spmm_bstage_kernel(const __grid_constant__ CUtensorMap tmapB, int m, int n, int 
 // * per plan (quad_order_* kernels): the rows of at most kLongRow nonzeros sorted by length, longest first, in blocks
 //   of GPW = 32 / LANES list slots: the rows of a block -- one step of a warp -- are equally long, except where the
 //   length changes along the list; a quad is a group of four nonzeros;
-// * per call (spmm_bstage_prep_kernel): A copied into two arrays of quads (four byte offsets col * ROW_BYTES; four
-//   FP32 values).  Quad i of the row in slot g of block b sits at quad position pos[b] + i * GPW + g, so the GPW
-//   groups of a warp read GPW consecutive quads at every step: one wavefront.  The last quad of a row is padded with
-//   (0, 0.0f), which is never multiplied.  Inside a row the entries are ordered by (col - g) mod G, G = 128 / ROW_BYTES
+// * per call (spmm_bstage_prep_kernel): A copied into two arrays of quads: four 16-bit offsets col * ROW_BYTES / 16 (the
+//   slice has fewer than 2^16 sixteen-byte pieces), and the four values as stored (FP32 or BF16).  Quad i of the row in
+//   slot g of block b sits at quad position pos[b] + i * GPW + g, so the GPW groups of a warp read GPW consecutive
+//   quads at every step.  The last quad of a row is padded with (0, 0), which is never multiplied.  Inside a row the entries are ordered by (col - g) mod G, G = 128 / ROW_BYTES
 //   rows of the slice per bank line: the groups of a quarter warp own neighbouring slots, so while the classes of
 //   their rows are equally long they read different parts of the bank line.  (The order of a row's products
 //   changes; each lane still adds them in one fixed order.)
@@ -205,7 +210,7 @@ template <typename T, int ROW_BYTES>
 __global__ void __launch_bounds__(256)
 spmm_bstage_prep_kernel(int slots, int gpw, const int* __restrict__ quad_row, const int* __restrict__ quad_pos,
                         const int* __restrict__ row_ptr, const int* __restrict__ col_idx, const T* __restrict__ vals,
-                        int* __restrict__ qoff, float* __restrict__ qval) {
+                        unsigned short* __restrict__ qoff, T* __restrict__ qval) {
   constexpr int G = 128 / ROW_BYTES;
   constexpr unsigned FULL = 0xFFFFFFFFu;
   grid_dependency_wait();
@@ -251,10 +256,10 @@ spmm_bstage_prep_kernel(int slots, int gpw, const int* __restrict__ quad_row, co
   for (int p0 = 0; p0 < longest; p0 += 8) {
     const bool valid = p0 + sub < len;
     int c = 0, cls = -1;
-    float v = 0.0f;
+    T v = T();
     if (valid) {
       c = __ldg(col_idx + rs + p0 + sub);
-      v = to_f32(__ldg(vals + rs + p0 + sub));
+      v = __ldg(vals + rs + p0 + sub);
       cls = (c - gc) & (G - 1);
     }
     int dest = 0;
@@ -266,22 +271,42 @@ spmm_bstage_prep_kernel(int slots, int gpw, const int* __restrict__ quad_row, co
     }
     if (valid) {
       const long long e = base + (long long)(dest >> 2) * stride + (dest & 3);
-      qoff[e] = c * ROW_BYTES;
+      qoff[e] = (unsigned short)(c * (ROW_BYTES / 16));
       qval[e] = v;
     }
   }
   for (int d = len + sub; d < ((len + 3) & ~3); d += 8) {
     const long long e = base + (long long)(d >> 2) * stride + (d & 3);
     qoff[e] = 0;
-    qval[e] = 0.0f;
+    qval[e] = T();
   }
 }
 
-// acc += the products of one row's quads 0 .. (len + 3) / 4 - 1 with this lane's columns of the slice (at shared address bs).
-// SHARED: the quads sit in shared memory at addresses so / sv, else in global memory at qo / qv; consecutive quads of the
-// row are qstride quads apart.
+// One quad of the re-laid A: the shared-memory addresses of this lane's piece of the four rows of the slice, and the four values.
+template <typename T, bool SHARED> struct QuadLoad;
+template <bool SHARED> struct QuadLoad<float, SHARED> {
+  static __device__ __forceinline__ void ld(const uint2* qo, const float* qv, unsigned so, unsigned sv, unsigned bs, unsigned (&a)[4], float (&v)[4]) {
+    const uint2 o = SHARED ? lds64(so) : __ldg(qo);
+    const float4 x = SHARED ? lds128(sv, (const float4*)nullptr) : __ldg((const float4*)qv);
+    a[0] = bs + ((o.x & 0xFFFFu) << 4); a[1] = bs + ((o.x >> 16) << 4); a[2] = bs + ((o.y & 0xFFFFu) << 4); a[3] = bs + ((o.y >> 16) << 4);
+    v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+  }
+};
+template <bool SHARED> struct QuadLoad<bf16_t, SHARED> {
+  static __device__ __forceinline__ void ld(const uint2* qo, const bf16_t* qv, unsigned so, unsigned sv, unsigned bs, unsigned (&a)[4], float (&v)[4]) {
+    const uint2 o = SHARED ? lds64(so) : __ldg(qo);
+    const uint2 x = SHARED ? lds64(sv) : __ldg((const uint2*)qv);
+    a[0] = bs + ((o.x & 0xFFFFu) << 4); a[1] = bs + ((o.x >> 16) << 4); a[2] = bs + ((o.y & 0xFFFFu) << 4); a[3] = bs + ((o.y >> 16) << 4);
+    v[0] = __uint_as_float(x.x << 16); v[1] = __uint_as_float(x.x & 0xFFFF0000u);
+    v[2] = __uint_as_float(x.y << 16); v[3] = __uint_as_float(x.y & 0xFFFF0000u);
+  }
+};
+
+// acc += the products of one row's quads 0 .. (len + 3) / 4 - 1 with this lane's columns of the slice (whose piece of row 0
+// is at shared address bs).  SHARED: the quads sit in shared memory at addresses so / sv, else in global memory at qo / qv;
+// consecutive quads of the row are qstride quads apart.
 template <typename T, int VEC, bool SHARED>
-__device__ __forceinline__ void bstage_row_quads(const int4* __restrict__ qo, const float4* __restrict__ qv, unsigned so, unsigned sv, int qstride,
+__device__ __forceinline__ void bstage_row_quads(const uint2* __restrict__ qo, const T* __restrict__ qv, unsigned so, unsigned sv, int qstride,
                                                  int len, unsigned bs, float (&acc)[VEC], float (&tot)[VEC]) {
   typedef typename RawVec<T, VEC>::type raw_t;
   const int full = len >> 2, rem = len & 3;
@@ -292,25 +317,27 @@ __device__ __forceinline__ void bstage_row_quads(const int4* __restrict__ qo, co
 #pragma unroll
       for (int j = 0; j < VEC; ++j) { tot[j] += acc[j]; acc[j] = 0.0f; }
     }
-    const int4 o = SHARED ? lds128(so, (const int4*)nullptr) : __ldg(qo);
-    const float4 v = SHARED ? lds128(sv, (const float4*)nullptr) : __ldg(qv);
-    so += 16u * qstride; sv += 16u * qstride; qo += qstride; qv += qstride;
+    unsigned a[4];
+    float v[4];
+    QuadLoad<T, SHARED>::ld(qo, qv, so, sv, bs, a, v);
+    so += 8u * qstride; sv += 4u * (unsigned)sizeof(T) * qstride; qo += qstride; qv += 4 * qstride;
     raw_t b[4];
-    b[0] = lds128(bs + o.x, (const raw_t*)nullptr); b[1] = lds128(bs + o.y, (const raw_t*)nullptr);
-    b[2] = lds128(bs + o.z, (const raw_t*)nullptr); b[3] = lds128(bs + o.w, (const raw_t*)nullptr);
-    RawVec<T, VEC>::fma_mixed(b[0], v.x, acc); RawVec<T, VEC>::fma_mixed(b[1], v.y, acc);
-    RawVec<T, VEC>::fma_mixed(b[2], v.z, acc); RawVec<T, VEC>::fma_mixed(b[3], v.w, acc);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) b[u] = lds128(a[u], (const raw_t*)nullptr);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) RawVec<T, VEC>::fma_mixed(b[u], v[u], acc);
   }
   if (rem) {   // the padded last quad: its padding is never multiplied (0 * inf would be NaN)
-    const int4 o = SHARED ? lds128(so, (const int4*)nullptr) : __ldg(qo);
-    const float4 v = SHARED ? lds128(sv, (const float4*)nullptr) : __ldg(qv);
-    RawVec<T, VEC>::fma_mixed(lds128(bs + o.x, (const raw_t*)nullptr), v.x, acc);
-    if (rem > 1) RawVec<T, VEC>::fma_mixed(lds128(bs + o.y, (const raw_t*)nullptr), v.y, acc);
-    if (rem > 2) RawVec<T, VEC>::fma_mixed(lds128(bs + o.z, (const raw_t*)nullptr), v.z, acc);
+    unsigned a[4];
+    float v[4];
+    QuadLoad<T, SHARED>::ld(qo, qv, so, sv, bs, a, v);
+    RawVec<T, VEC>::fma_mixed(lds128(a[0], (const raw_t*)nullptr), v[0], acc);
+    if (rem > 1) RawVec<T, VEC>::fma_mixed(lds128(a[1], (const raw_t*)nullptr), v[1], acc);
+    if (rem > 2) RawVec<T, VEC>::fma_mixed(lds128(a[2], (const raw_t*)nullptr), v[2], acc);
   }
 }
 
-// Dynamic shared memory: [ slice of B: bslice_bytes | per warp: capq offset quads (16 B each), capq value quads ].
+// Dynamic shared memory: [ slice of B: bslice_bytes | per warp: capq offset quads (8 B each), capq value quads (4 values each) ]; capq is even.
 // CTA `chunk` of a slice takes the blocks chunk, chunk + row_chunks, ... of the sorted list, its warps in turn, so that
 // every CTA gets the same mix of long and short rows.  A block of more than capq quads is read from global memory.
 // (Fetching the next block's quads a step ahead into a second half of the buffer was measured: no gain.)
@@ -318,7 +345,7 @@ template <typename T, int VEC, int LANES, int THREADS>
 __global__ void __launch_bounds__(THREADS)
 spmm_bstage_quads_kernel(const __grid_constant__ CUtensorMap tmapB, int n, int k, int row_chunks, int blocks, int box_rows, int bslice_bytes,
                          int capq, const int* __restrict__ quad_row, const int* __restrict__ quad_len, const int* __restrict__ quad_pos,
-                         const int* __restrict__ qoff, const float* __restrict__ qval, T* __restrict__ Y, float alpha, float beta,
+                         const unsigned short* __restrict__ qoff, const T* __restrict__ qval, T* __restrict__ Y, float alpha, float beta,
                          int* __restrict__ err, int spin_limit, int no_copies) {
   constexpr int KS = LANES * VEC, ROW_BYTES = LANES * 16, GPW = 32 / LANES, WARPS = THREADS / 32;
   constexpr unsigned FULL = 0xFFFFFFFFu;
@@ -343,8 +370,9 @@ spmm_bstage_quads_kernel(const __grid_constant__ CUtensorMap tmapB, int n, int k
   const int col0 = col_base + l * VEC;
   const bool active = col0 < k;
   const unsigned bs = smem_addr(smem) + l * 16;
-  const unsigned woff = smem_addr(smem) + bslice_bytes + warp * capq * 32;   // the warp's buffer: capq quads of offsets, then of values
-  const unsigned wval = woff + capq * 16;
+  constexpr unsigned VQ = 4u * (unsigned)sizeof(T);                          // bytes of a quad's values
+  const unsigned woff = smem_addr(smem) + bslice_bytes + warp * capq * (8u + VQ);   // the warp's buffer: capq quads of offsets, then of values
+  const unsigned wval = woff + capq * 8u;
   const unsigned my_bar = smem_addr(&wbar[warp]);
   const long long step_blocks = (long long)WARPS * row_chunks;
   // one step's description, a value per lane: lanes < GPW the row number (m_row) and length (m_len) of their slot,
@@ -359,9 +387,9 @@ spmm_bstage_quads_kernel(const __grid_constant__ CUtensorMap tmapB, int n, int k
   // the bulk copies that fetch a block's quads (lane 0 issues; the buffer must be free)
   auto issue = [&](int q0, int nq) {
     if (nq > 0 && nq <= capq && lane == 0) {
-      mbar_arrive_expect_tx(my_bar, (unsigned)nq * 32u);
-      bulk_copy_g2s(woff, qoff + (long long)q0 * 4, (unsigned)nq * 16u, my_bar);
-      bulk_copy_g2s(wval, qval + (long long)q0 * 4, (unsigned)nq * 16u, my_bar);
+      mbar_arrive_expect_tx(my_bar, (unsigned)nq * (8u + VQ));
+      bulk_copy_g2s(woff, qoff + (long long)q0 * 4, (unsigned)nq * 8u, my_bar);
+      bulk_copy_g2s(wval, qval + (long long)q0 * 4, (unsigned)nq * VQ, my_bar);
     }
   };
   long long b = chunk + (long long)warp * row_chunks;
@@ -395,9 +423,9 @@ spmm_bstage_quads_kernel(const __grid_constant__ CUtensorMap tmapB, int n, int k
 #pragma unroll
     for (int j = 0; j < VEC; ++j) { acc[j] = 0.0f; tot[j] = 0.0f; }
     if (staged) {
-      bstage_row_quads<T, VEC, true>(nullptr, nullptr, woff + 16u * gl, wval + 16u * gl, GPW, len, bs, acc, tot);
+      bstage_row_quads<T, VEC, true>(nullptr, nullptr, woff + 8u * gl, wval + VQ * gl, GPW, len, bs, acc, tot);
     } else {
-      bstage_row_quads<T, VEC, false>((const int4*)qoff + q0_cur + gl, (const float4*)qval + q0_cur + gl, 0u, 0u, GPW, len, bs, acc, tot);
+      bstage_row_quads<T, VEC, false>((const uint2*)qoff + q0_cur + gl, qval + 4LL * (q0_cur + gl), 0u, 0u, GPW, len, bs, acc, tot);
     }
     __syncwarp();                       // every lane is done with the buffer: the next block's quads may land in it
     issue(q0_next, nq_next);            // (past the last block nq_next is 0)

@@ -16,7 +16,7 @@ DEFAULTS = {
     "row_unroll": 8, "row_threads": 256, "row_stages": 2, "row_ctas": 3, "row_smem_kb": 220,
     "uni_unroll": 0, "uni_ctas": 0, "sub_lanes": 0,
     "merge_items": 2048, "merge_threads": 128, "merge_short": 32, "merge_carve": 45, "merge_empty": 0,
-    "spmm_bstage": 1, "spmm_sliced": 1, "spmm_ranges": 1, "spmm_stage_a": 2, "spmm_flat": 2, "bstage_threads": 1024, "bstage_nnz": 131072, "bstage_stage_a": 1, "bstage_quads": 1,
+    "spmm_bstage": 1, "spmm_sliced": 1, "spmm_ranges": 1, "spmm_stage_a": 2, "spmm_flat": 2, "bstage_threads": 1024, "bstage_nnz": 0, "bstage_stage_a": 1, "bstage_quads": 1,
 }
 
 # (switch, accepted values, SpMV kernel to force so that the switch matters; None = leave the choice to the plan)
@@ -33,7 +33,7 @@ SPMV_SWITCHES = [
 ]
 SPMM_SWITCHES = [
     ("x_l2_window", [0, 1]), ("pdl", [0, 1]), ("spmm_bstage", [0, 1]), ("spmm_sliced", [0, 1]), ("spmm_ranges", [0, 1, 2, 3, 4, 8]), ("spmm_stage_a", [0, 1, 2]), ("spmm_flat", [0, 1, 2]),
-    ("bstage_threads", [256, 512, 1024]), ("bstage_nnz", [16384, 65536, 131072, 524288]), ("bstage_stage_a", [0, 1]), ("bstage_quads", [0, 1]),
+    ("bstage_threads", [256, 512, 1024]), ("bstage_nnz", [0, 16384, 65536, 131072, 524288]), ("bstage_stage_a", [0, 1]), ("bstage_quads", [0, 1]),
 ]
 
 

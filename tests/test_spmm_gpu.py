@@ -269,3 +269,82 @@ def test_nnz_balanced_kernel_is_reproducible_and_keeps_chains_short():
     finally:
         b200sp.b200sp_set_option("spmm_flat", 2)
         b200sp.b200sp_cache_clear()
+
+
+def quad_row_cases():
+    rng = np.random.default_rng(1)
+    return {
+        "every_length_0_to_70": np.tile(np.arange(71), 3),           # every remainder modulo four, lengths changing inside blocks
+        "all_empty_but_few": np.concatenate([np.zeros(500, np.int64), [5000], np.zeros(500, np.int64), [3, 1024, 1025]]),
+        "rows_at_the_long_row_limit": np.array([1023, 1024, 1025, 1026, 4096, 0, 1, 2, 3, 4, 5000, 1024, 1024]),
+        "only_long_rows": np.array([3000, 2000, 1500]),
+        "single_row": np.array([4000]),
+        "one_block_less_one": np.full(7, 24),
+        "one_block_plus_one": np.full(17, 24),
+        "equal_rows": np.full(4096, 20),
+        "binomial": rng.binomial(2048, 0.01, 5000),
+        "more_quads_than_a_warp_buffer": np.concatenate([np.full(40, 900), np.full(900, 40)]),
+    }
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+@pytest.mark.parametrize("n", [120, 2048, 5000])
+@pytest.mark.parametrize("case", sorted(quad_row_cases()))
+def test_b_in_shared_memory_sorted_quads_adversarial_rows(case, n, dtype):
+    """The kernel that holds a slice of B in shared memory, on its re-laid copy of A (rows sorted by length into blocks, quads
+    interleaved, entries ordered by bank class): all three slice widths (8, 4, 2 lanes per row: n = 120, 2048, 5000), every
+    row-length remainder, list lengths around a block, rows on both sides of the long-row limit, blocks larger than a warp's
+    buffer (read from global memory), k that is and is not a multiple of the slice, beta != 0."""
+    lens = quad_row_cases()[case]
+    m = len(lens)
+    if lens.sum() < 4 * n:                        # the kernel is chosen when nnz >= 4 n
+        lens = np.concatenate([lens, np.full((4 * n - lens.sum()) // 16 + 1, 16)])
+        m = len(lens)
+    A = gen.random_csr(m, n, lens, seed=len(case) + n, sort_cols=False, allow_dup=True)
+    rng = np.random.default_rng(3)
+    for k in (64, 72):
+        B = rng.standard_normal(n * k).astype(np.float32)
+        Y0 = rng.standard_normal(m * k).astype(np.float32)
+        Y, Y_ref, S = run_spmm(A, B, k, None, 1.0, 0.0, dtype)
+        assert_within(Y, Y_ref, S, dtype, what="quads %s n=%d k=%d" % (case, n, k))
+        Y, Y_ref, S = run_spmm(A, B, k, Y0, -0.5, 1.25, dtype)
+        y0f = Y0 if dtype == "f32" else gen.bf16_to_f32(gen.to_bf16(Y0))
+        assert_within(Y, Y_ref, S, dtype, 1.0, np.abs(1.25 * y0f.astype(np.float64)).reshape(m, k), what="quads %s n=%d k=%d ab" % (case, n, k))
+    b200sp.b200sp_check()
+
+
+def test_b_in_shared_memory_sorted_quads_reproducible_exact_and_nonfinite():
+    """Small-integer data: every product and sum is exact, so the result equals the oracle's bit for bit whatever the order of a
+    row's products; three runs agree bit for bit; a row whose padded last quad sits next to an infinite entry of B stays
+    infinite (padding is never multiplied); the plan's sorted order is reused by a second call with other values."""
+    import torch
+    from gpu_util import empty_out, to_dev
+    rng = np.random.default_rng(12)
+    n, k = 2048, 128
+    lens = rng.binomial(2048, 0.01, 3000)
+    lens[5] = 1                                   # one entry: three padded slots in its only quad
+    A = gen.random_csr(len(lens), n, lens, seed=8, integer_vals=True)
+    B = rng.integers(-3, 4, n * k).astype(np.float32)
+    Y, Y_ref, S = run_spmm(A, B, k, None, 1.0, 0.0, "f32")
+    assert np.array_equal(Y.astype(np.float64), Y_ref)
+    d = [to_dev(a) for a in (A.row_ptr, A.col_idx, A.vals, B)]
+    outs = []
+    for _ in range(3):
+        Yd = empty_out(A.m * k, "f32")
+        b200sp.spmm_csr(A.m, A.n, A.nnz, k, d[0], d[1], d[2], d[3], Yd, 1.0, 0.0, "f32")
+        torch.cuda.synchronize()
+        outs.append(Yd.cpu().numpy().copy())
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+    assert np.array_equal(outs[0].reshape(A.m, k), Y)
+    # offset 0 (the padding's) is row 0 of B: make it infinite; row 5 (one entry, another column) must not see it
+    c5 = int(A.col_idx[A.row_ptr[5]])
+    if c5 == 0:
+        A.col_idx[A.row_ptr[5]] = c5 = 7
+    B2 = B.copy()
+    B2[:k] = np.inf
+    A.vals[A.row_ptr[5]] = 2.0
+    Y2, Y2_ref, _ = run_spmm(A, B2, k, None, 1.0, 0.0, "f32")
+    assert np.all(np.isfinite(Y2[5])) and np.array_equal(Y2[5].astype(np.float64), Y2_ref[5])
+    rows_with_col0 = np.unique(np.repeat(np.arange(A.m), np.diff(A.row_ptr))[A.col_idx == 0])
+    assert len(rows_with_col0) > 0 and not np.any(np.isfinite(Y2[rows_with_col0]))
+    b200sp.b200sp_check()
