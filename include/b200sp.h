@@ -39,8 +39,10 @@
  *    nothing; a device that is not compute capability 10.x returns B200SP_ERR_ARCH; a failing CUDA
  *    call returns B200SP_ERR_CUDA and its message is kept for b200sp_last_cuda_error().
  *  - Device memory the library needs (plan scratch, the staging buffers of the "host" entry
- *    points, and for SpMM on matrices with very uneven rows a few bytes per 1024 nonzeros and dense
- *    column of per-call scratch, taken and returned in the order of `stream`) comes from a
+ *    points, and per-call scratch for SpMM, taken and returned in the order of `stream`: on matrices
+ *    with very uneven rows a few bytes per 1024 nonzeros and dense column; on matrices with so few
+ *    columns that a slice of B is kept in shared memory a re-laid copy of A, about (2 + bytes per
+ *    value) * (nnz + 3 m) bytes, plus 8 m bytes kept with the plan) comes from a
  *    stream-ordered memory pool of its own, one per device, created at first use.  The pool keeps up to 1 GiB of freed memory for the next call (option "pool_keep_mb",
  *    read when the pool is created); b200sp_cache_clear hands all unused pool memory back.
  *  - There is no CPU fallback: without a B200 the compute entry points fail.
@@ -113,7 +115,8 @@ int spmm_csr(int64_t m, int64_t n, int64_t nnz, int64_t k, const int32_t* row_pt
  * SpMM treats separately, all on the device.  From the same statistics it decides whether SpMM gives every row to a
  * group of eight lanes (even rows) or cuts the nonzeros into equal chunks whatever rows they belong to (uneven rows:
  * many empty rows, or a share of the nonzeros in rows of more than 128); the list of non-empty rows that the second
- * form needs is built on the first SpMM call, in stream order.
+ * form needs is built on the first SpMM call, in stream order, and so is the order of the rows by length that SpMM
+ * uses when A has so few columns that a slice of B is kept in shared memory.
  * When the row statistics select the row-direct SpMV kernel, the first b200sp_spmv / spmv_csr call with a given
  * col_idx additionally samples how local the columns are (one small kernel and one synchronisation of the stream)
  * and falls back to the merge-tile kernel for matrices with scattered columns.
