@@ -424,6 +424,18 @@ def run_probes(dev, l2_bytes):
                 % (gl * 16, gl // 8, "s" if gl > 8 else "", gl, inflight, "to shared memory (cp.async)" if to_smem else "to registers", label),
                 nreads * gl * 16 / t * 1e-12, "TB/s", "%.1f bytes per clock per SM" % (nreads * gl * 16 / t / sms / clock_hz))
         del buf
+    # the gather phase of SpMV on the workloads' own matrices, against the shared memory carved out of the unified cache
+    import gen
+    for name in ("c3", "c3p", "c2"):
+        w = gen.workload(name)
+        A = w.A
+        d_col, d_val, d_x = up(A.col_idx, dev), up(np.ascontiguousarray(A.vals, np.float32), dev), up(np.ascontiguousarray(w.x, np.float32), dev)
+        outv = torch.zeros(sms * 1024, dtype=torch.float32, device=dev)
+        for kb in (0, 8, 16, 32, 64, 100, 164):
+            t = timed(lambda: b200sp.b200sp_probe_spmv_gather(A.nnz, d_col, d_val, d_x, "f32", kb, outv, stream))
+            row("gather phase of SpMV alone on %s (FP32), %d KB of shared memory carved out per SM" % (name, kb), t * 1e6, "us",
+                "%.0f G gathers/s" % (A.nnz / t * 1e-9))
+        del d_col, d_val, d_x, w, A
     return out
 
 

@@ -103,13 +103,20 @@ int b200sp_get_option(const char* name, int* value);
  *   lines (a power of two), each chunk by a group of group_lanes = 8, 16 or 32 lanes with 16 bytes per lane and
  *   in_flight = 4, 8 or 16 chunks in flight per group, into registers or, with to_shared_memory = 1 (group_lanes = 8
  *   only), into shared memory with cp.async: the L2-to-SM rate of SpMM's reads of B (the k-sliced kernel keeps four
- *   lines per group of eight lanes in registers). */
+ *   lines per group of eight lanes in registers).
+ * b200sp_probe_spmv_gather: the gather phase of a CSR SpMV on the caller's arrays and nothing else: sum over all nonzeros
+ *   of vals[p] * x[col_idx[p]] in per-thread partial sums (no rows, no y), one CTA of 1024 threads per SM, with
+ *   unused_smem_kb (0 .. 200) KB of shared memory per SM carved out and left unused.  out receives one float per thread
+ *   (SMs * 1024 floats; their sum is the sum above).  col_idx, vals 16-byte aligned; dtype as for spmv_csr; nnz is rounded
+ *   down to a multiple of four.  It shows how the time of the gathers depends on the L1 that a kernel's shared memory leaves. */
 int b200sp_probe_gather(const float* table, int64_t table_elems, int64_t gathers, float* sink, void* stream);
 int b200sp_probe_gather_ex(const void* table, int64_t table_elems, int64_t gathers, int elem_bytes, int in_shared_memory, float* sink,
                            void* stream);
 int b200sp_probe_stream(const void* buf, int64_t bytes, float* sink, void* stream);
 int b200sp_probe_lines(const void* buf, int64_t lines, int64_t reads, int in_flight, int to_shared_memory, int group_lanes, float* sink,
                        void* stream);
+int b200sp_probe_spmv_gather(int64_t nnz, const int32_t* col_idx, const void* vals, const void* x, int dtype, int unused_smem_kb, float* out,
+                             void* stream);
 
 #ifdef __cplusplus
 }

@@ -21,7 +21,7 @@ EXPORTS = (
     "spmv_csr", "spmm_csr", "b200sp_plan_create", "b200sp_plan_destroy", "b200sp_plan_info", "b200sp_spmv",
     "b200sp_spmm", "spmv_csr_host", "spmm_csr_host", "b200sp_validate_csr", "b200sp_cache_clear",
     "b200sp_status_string", "b200sp_last_cuda_error", "b200sp_version", "b200sp_checked_build", "b200sp_launch_count", "b200sp_set_option", "b200sp_get_option",
-    "b200sp_check", "b200sp_cache_drop", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_probe_gather_ex", "b200sp_probe_stream", "b200sp_probe_lines", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell", "spmv_csc", "spmm_csc", "spmv_csr_vec_host",
+    "b200sp_check", "b200sp_cache_drop", "spmv_csr_noalloc", "b200sp_noalloc_max_items", "b200sp_probe_gather", "b200sp_probe_gather_ex", "b200sp_probe_stream", "b200sp_probe_lines", "b200sp_probe_spmv_gather", "b200sp_spmv_naive", "b200sp_spmm_naive", "spmv_coo", "spmm_coo", "spmv_ell", "spmm_ell", "spmv_csc", "spmm_csc", "spmv_csr_vec_host",
 )
 
 
@@ -88,6 +88,8 @@ def lib() -> ctypes.CDLL:
         L.b200sp_probe_stream.restype = i32
         L.b200sp_probe_lines.argtypes = [p, i64, i64, i32, i32, i32, p, p]
         L.b200sp_probe_lines.restype = i32
+        L.b200sp_probe_spmv_gather.argtypes = [i64, p, p, p, i32, i32, p, p]
+        L.b200sp_probe_spmv_gather.restype = i32
         L.spmm_csr_host.argtypes = L.spmm_csr.argtypes
         L.b200sp_plan_create.argtypes = [ctypes.POINTER(p), i64, i64, i64, p, p]
         L.b200sp_plan_destroy.argtypes = [p]
@@ -308,6 +310,13 @@ def b200sp_probe_stream(buf, nbytes, sink, stream=None):
 def b200sp_probe_lines(buf, lines, reads, sink, in_flight=4, to_shared_memory=0, stream=None, group_lanes=8):
     _ck(lib().b200sp_probe_lines(_dev(buf, lines * 128 // max(buf.element_size(), 1), buf.element_size(), "probe buffer"), lines, reads,
                                  in_flight, to_shared_memory, group_lanes, _dev(sink, 1, 4, "probe sink"), _stream(stream)), "b200sp_probe_lines")
+
+
+def b200sp_probe_spmv_gather(nnz, col_idx, vals, x, dtype, unused_smem_kb, out, stream=None):
+    code = _dt(dtype)
+    esize = 4 if code == 0 else 2
+    _ck(lib().b200sp_probe_spmv_gather(nnz, _dev(col_idx, nnz, 4, "col_idx"), _dev(vals, nnz, esize, "vals"), _dev(x, 1, esize, "x"), code,
+                                       unused_smem_kb, _dev(out, 1, 4, "probe out"), _stream(stream)), "b200sp_probe_spmv_gather")
 
 
 def b200sp_noalloc_max_items() -> int:

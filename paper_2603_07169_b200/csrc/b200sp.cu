@@ -279,6 +279,26 @@ int b200sp_probe_lines(const void* buf, int64_t lines, int64_t reads, int in_fli
 #undef B200SP_PROBE_LINES
 }
 
+int b200sp_probe_spmv_gather(int64_t nnz, const int32_t* col_idx, const void* vals, const void* x, int dtype, int unused_smem_kb, float* out,
+                             void* stream) {
+  if (!col_idx || !vals || !x || !out || nnz < 4 || nnz >= ((int64_t)1 << 31) || !aligned16(col_idx) || !aligned16(vals) ||
+      (dtype != B200SP_F32 && dtype != B200SP_BF16) || unused_smem_kb < 0 || unused_smem_kb > 200)
+    return B200SP_ERR_INVALID_ARG;
+  DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != B200SP_OK) return rc;
+  const size_t smem = (size_t)unused_smem_kb * 1024;
+  const dim3 grid((unsigned)dev->sms), block(1024);
+  if (dtype == B200SP_F32) {
+    CU(cudaFuncSetAttribute(probe_spmv_gather_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    return launch_smem(probe_spmv_gather_kernel<float>, grid, block, smem, (cudaStream_t)stream, nullptr, 0, dev, (const int*)col_idx,
+                       (const float*)vals, (long long)(nnz / 4), (const float*)x, out);
+  }
+  CU(cudaFuncSetAttribute(probe_spmv_gather_kernel<bf16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+  return launch_smem(probe_spmv_gather_kernel<bf16_t>, grid, block, smem, (cudaStream_t)stream, nullptr, 0, dev, (const int*)col_idx,
+                     (const bf16_t*)vals, (long long)(nnz / 4), (const bf16_t*)x, out);
+}
+
 int64_t b200sp_noalloc_max_items(void) { return (int64_t)kNoAllocMaxTiles * kItems; }
 
 int spmv_coo(int64_t m, int64_t n, int64_t nnz, const int32_t* row_idx, const int32_t* col_idx, const void* vals, const void* x,

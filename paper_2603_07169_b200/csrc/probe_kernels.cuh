@@ -4,6 +4,7 @@
 //   probe_gather_kernel   random reads of a table: the rate at which an SM takes L1 misses (table >> L1), L1 hits (table fits L1)
 //                         or shared-memory reads (table staged in shared memory) -- the bound on gathering x
 //   probe_stream_kernel   coalesced 128-bit reads of a buffer: what a pure stream of the CSR arrays can reach at a given size
+//   probe_spmv_gather_kernel  the gather phase of a CSR SpMV on the caller's arrays and nothing else (no row sums, no y)
 //   probe_lines_kernel    random reads of whole 128-byte lines (or two / four consecutive ones) by groups of 8 (16 / 32) lanes: the L2-to-SM path
 //                         that SpMM's reads of B use
 #pragma once
@@ -99,6 +100,31 @@ __global__ void __launch_bounds__(256) probe_lines_kernel(const int4* __restrict
     }
   }
   if (acc == 0x5A5A1234) *sink = (float)acc;
+}
+
+// The gather phase of a CSR SpMV alone: every thread streams groups of four (col, val) pairs (two groups in flight,
+// grid-stride, coalesced 128-bit loads that do not allocate in L1), gathers x and adds the products into one register;
+// one float per thread goes to `out`.  Launched with a given amount of dynamic shared memory that nothing uses, it shows
+// what the gathers cost as a function of the L1 that the carve-out leaves: on a matrix with skewed columns (few entries of
+// x take most of the gathers) that is what decides the time of an SpMV kernel.
+template <typename T>
+__global__ void __launch_bounds__(1024) probe_spmv_gather_kernel(const int* __restrict__ col_idx, const T* __restrict__ vals, long long quads,
+                                                                const T* __restrict__ x, float* __restrict__ out) {
+  float acc = 0.0f;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long q = (long long)blockIdx.x * blockDim.x + threadIdx.x; q < quads; q += 2 * stride) {
+    const int4 c0 = ld_stream_i4(col_idx + 4 * q);
+    float v0[4], v1[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    ld_stream_vals4(vals + 4 * q, v0);
+    const bool two = q + stride < quads;
+    int4 c1 = c0;                        // a valid column when the second group does not exist (its values are zero)
+    if (two) { c1 = ld_stream_i4(col_idx + 4 * (q + stride)); ld_stream_vals4(vals + 4 * (q + stride), v1); }
+    const float x0 = ld_gather(x + c0.x), x1 = ld_gather(x + c0.y), x2 = ld_gather(x + c0.z), x3 = ld_gather(x + c0.w);
+    const float x4 = ld_gather(x + c1.x), x5 = ld_gather(x + c1.y), x6 = ld_gather(x + c1.z), x7 = ld_gather(x + c1.w);
+    acc += v0[0] * x0 + v0[1] * x1 + v0[2] * x2 + v0[3] * x3;
+    if (two) acc += v1[0] * x4 + v1[1] * x5 + v1[2] * x6 + v1[3] * x7;
+  }
+  out[(long long)blockIdx.x * blockDim.x + threadIdx.x] = acc;
 }
 
 }  // namespace b200sp

@@ -295,3 +295,34 @@ print("ok")
     env = dict(os.environ, B200SP_LIBRARY="libb200sp_check.so")
     out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=600, env=env)
     assert out.returncode == 0 and "ok" in out.stdout, out.stdout + out.stderr
+
+
+def test_spmv_gather_probe_adds_every_product_and_refuses_bad_arguments():
+    """The gather-phase probe on the caller's arrays: its per-thread partial sums add up to sum(vals * x[col_idx]) (FP32 and
+    BF16 storage, with and without shared memory carved out), and out-of-range arguments launch nothing."""
+    import torch
+    import gen
+    from gpu_util import to_dev
+    rng = np.random.default_rng(4)
+    A = gen.random_csr(3000, 5000, rng.integers(0, 60, 3000), seed=2)
+    x = rng.standard_normal(A.n).astype(np.float32)
+    nnz4 = A.nnz // 4 * 4
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    for dtype in ("f32", "bf16"):
+        vals = A.vals if dtype == "f32" else gen.to_bf16(A.vals)
+        xs = x if dtype == "f32" else gen.to_bf16(x)
+        vf = A.vals if dtype == "f32" else gen.bf16_to_f32(vals)
+        xf = x if dtype == "f32" else gen.bf16_to_f32(xs)
+        want = float(np.dot(vf[:nnz4].astype(np.float64), xf[A.col_idx[:nnz4]].astype(np.float64)))
+        scale = float(np.dot(np.abs(vf[:nnz4]).astype(np.float64), np.abs(xf[A.col_idx[:nnz4]]).astype(np.float64)))
+        d_col, d_val, d_x = to_dev(A.col_idx), to_dev(vals), to_dev(xs)
+        for kb in (0, 64):
+            out = torch.zeros(sms * 1024, dtype=torch.float32, device="cuda:0")
+            b200sp.b200sp_probe_spmv_gather(A.nnz, d_col, d_val, d_x, dtype, kb, out)
+            torch.cuda.synchronize()
+            got = float(out.double().sum())
+            assert abs(got - want) <= 1e-5 * scale, (dtype, kb, got, want)
+    out = torch.zeros(sms * 1024, dtype=torch.float32, device="cuda:0")
+    for bad in (dict(nnz=2), dict(kb=201), dict(kb=-1)):
+        with pytest.raises(b200sp.B200spError):
+            b200sp.b200sp_probe_spmv_gather(bad.get("nnz", A.nnz), d_col, d_val, d_x, "f32", bad.get("kb", 0), out)
