@@ -365,6 +365,30 @@ def probe_gather_rate(n_elems: int, dev) -> float:
     return 5 * gathers / (a.elapsed_time(b) * 1e-3)
 
 
+def probe_gather_phase(w, dtype, dev, l2_bytes) -> float:
+    """Seconds the gather phase of SpMV alone takes on this workload's own matrix (b200sp_probe_spmv_gather, no shared memory
+    carved out), each repetition started cold (a buffer larger than L2 rewritten before it); median of 5."""
+    import torch
+    import paper_2603_07169_b200 as b200sp
+    A = w.A
+    d_col, d_val, d_x = up(A.col_idx, dev), up(stored(A.vals, dtype), dev), up(stored(w.x, dtype), dev)
+    flush = torch.empty(max(2 * l2_bytes, 256 << 20) // 4, dtype=torch.float32, device=dev)
+    out = torch.zeros(torch.cuda.get_device_properties(dev).multi_processor_count * 1024, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    ts = []
+    for rep in range(6):
+        flush.fill_(1.0)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        b200sp.b200sp_probe_spmv_gather(A.nnz, d_col, d_val, d_x, dtype, 0, out, stream)
+        b.record(stream)
+        b.synchronize()
+        if rep:
+            ts.append(a.elapsed_time(b) * 1e-3)
+    ts.sort()
+    return ts[len(ts) // 2]
+
+
 def run_probes(dev, l2_bytes):
     """The hardware rates that bound the kernels, each measured by a library probe kernel that does nothing else (CUDA events,
     median of 7 repetitions, a buffer larger than L2 rewritten between repetitions so that every repetition starts cold)."""
@@ -775,6 +799,10 @@ def main():
     # max over ranks of the timed region
     ms_step, value = aggregate_over_ranks(head["ms_total"], head["algorithmic_bytes"], steps, world, dist if world > 1 else None, dev)
     gather_rate = probe_gather_rate(w.A.n, dev) if not w.k else None
+    try:
+        gather_alone_ms = probe_gather_phase(w, dtype, dev, l2) * 1e3 if not w.k else None
+    except Exception:  # pragma: no cover
+        gather_alone_ms = None
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     A = w.A
@@ -863,6 +891,8 @@ def main():
                     ex_ = extras["%s_%s" % (name, dt)]
                     ex_["gather_bound_ms"] = round(ww.A.nnz / rate * 1e3, 5)
                     ex_.update(request_bound(ncu_record(name, dt), ww, dt, rate))
+                    if name in ("c2", "c3", "c3p"):   # the floor on the matrix itself: a loop that only gathers (no rows, no y)
+                        ex_["gather_phase_alone_ms"] = round(probe_gather_phase(ww, dt, dev, l2) * 1e3, 5)
                 else:          # SpMM: time of its reads of B (nnz * k * e bytes, one 128-byte line per nonzero and slice) at the measured rate of such reads
                     lr = probe_lines_rate(dev)
                     ex_ = extras["%s_%s" % (name, dt)]
@@ -972,7 +1002,9 @@ def main():
                              "secondary": None if gather_rate is None else {
                                  "bound": "L1-miss gather (one L2 request per random x read)", "gathers_per_s": gather_rate,
                                  "ms_at_bound": A.nnz / gather_rate * 1e3, "frac_of_bound": (A.nnz / gather_rate * 1e3) / (head["ms_total"] / steps),
-                                 "note": "measured live with b200sp_probe_gather on a table the size of x"}},
+                                 "note": "measured live with b200sp_probe_gather on a table the size of x",
+                                 "gather_phase_alone_ms": gather_alone_ms,
+                                 "gather_phase_note": "b200sp_probe_spmv_gather on this workload's own col_idx / vals / x, started cold: a loop that only gathers (no row sums, no y)"}},
                 "cusparse": {"ms_per_step": head["cusparse_ms"], "note": "cusparseSpMV/SpMM, default algorithm, preprocess excluded, over the same rotated operand copies (cold L2); comparison point only"},
                 "cpu_baseline": cpu, "extra": extras}
         print(json.dumps(line))
